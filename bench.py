@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the HGRN2 hot path on B200.
+
+A step is one forward + one backward of the recurrence over the `lm_2048` workload (model
+d = 2048: H = 16 heads of d_k = d_v = 128, B = 8 sequences of N = 2048 tokens, bf16 I/O, fp32
+state).  The decode workload (`decode`: 256 x 16 states, one token per call, 512 consecutive
+calls) is timed separately and reported in the same JSON line under "decode".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 the script expects to be launched by torch.distributed.run, one rank per GPU; the
+(batch, head) units are independent, so every rank runs the same per-GPU workload (weak
+scaling) and no collective touches the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (None until a capture of that kernel exists).
+NCU_TRAFFIC_BYTES = {"fwd": None, "bwd": None, "step": None}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            d = json.load(fh)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work (what the method must move / compute, independent of the implementation)
+# ------------------------------------------------------------------------------------------------
+def train_bytes(w, esize=2):
+    """fwd reads o, f, i and writes y; bwd reads o, f, i, dy and writes d_o, d_f, d_i: each once."""
+    per_tensor = w.B * w.H * w.N * w.dk * esize
+    return {"fwd": 4 * per_tensor, "bwd": 7 * per_tensor}
+
+
+def train_flops(w, C=64):
+    """Causal count of the chunked form per token-head (intra-chunk blocks counted (C+1)/2C)."""
+    th = w.B * w.H * w.N
+    fwd = 4 * w.dk * w.dv + 2 * w.dk * (C + 1)
+    bwd = 8 * w.dk * w.dv + 5 * w.dk * (C + 1)
+    return {"fwd": th * fwd, "bwd": th * bwd}
+
+
+def decode_bytes(w, esize=2):
+    units = w.B * w.H
+    return units * (2 * w.dk * w.dv * 4 + (2 * w.dk + 2 * w.dv) * esize)
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks sampling during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=5)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for p in self.samples:
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, val in zip(self.NAMES, p[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle arm (CPU): used for --impl reference and for the cpu_baseline object
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_step(inp_units):
+    from oracle import ref
+    ref.hgrn2_fwd(inp_units["o"], inp_units["f"], inp_units["i"], inp_units["S0"])
+    ref.hgrn2_bwd(inp_units["o"], inp_units["f"], inp_units["i"], inp_units["S0"], inp_units["dy"], inp_units["dSN"])
+
+
+def oracle_sample_inputs(w, n_units):
+    """The first n_units (b, h) units of the workload, as one [1, n_units, N, d] problem in fp64."""
+    from paper_2404_07904_b200 import workloads as W
+    small = W.scaled(w, B=1, H=n_units)
+    inp = W.make_inputs(small)
+    return {k: (None if v is None else v.astype(np.float64)) for k, v in inp.items()}
+
+
+def time_oracle(w, steps, warmup, n_units):
+    from oracle import ref
+    ref.build()
+    cores = ref.num_threads()
+    inp = oracle_sample_inputs(w, n_units)
+    for _ in range(warmup):
+        oracle_sample_step(inp)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_sample_step(inp)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    tokens = n_units * w.N / w.H          # a token spans all H heads
+    return tokens / dt, dt, cores
+
+
+def run_reference(args):
+    from paper_2404_07904_b200 import workloads as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = W.CONFIGS["lm_2048"]
+    from oracle import ref
+    ref.build()
+    n_units = max(1, min(ref.num_threads(), w.B * w.H))
+    value, dt, cores = time_oracle(w, args.steps, args.warmup, n_units)
+    sample = (f"{n_units} of {w.B * w.H} (batch, head) units of lm_2048 per step (N={w.N}, d_k=d_v={w.dk}), "
+              f"fwd+bwd, fp64, scaled by tokens")
+    line = {
+        "impl": "reference", "metric": "HGRN2 layer fwd+bwd tokens/s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, None),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def workload_config(w, path):
+    return {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d_k": w.dk, "d_v": w.dv, "d_model": w.H * w.dk,
+            "io": w.io, "state": "f32", "gamma": w.gamma, "path": path,
+            "l2": "inputs larger than L2 (each pass streams > 250 MB; no flush needed)"}
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2404_07904_b200 import binding, workloads as W
+    import __graft_entry__ as entry
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("for --gpus N > 1 launch with: python -m torch.distributed.run --nproc-per-node N bench.py --gpus N ...")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    if rank == 0:
+        entry.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+    binding.load()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return ms
+
+    peaks, peak_kind = load_peaks()
+    w = W.CONFIGS["lm_2048"]
+    # every rank holds its own batch of the same shape (weak scaling); a different seed per rank
+    inp = W.make_inputs(w, seed=w.seed + 1000 * rank)
+    bf = torch.bfloat16
+    host = {k: torch.from_numpy(inp[k]).to(bf).pin_memory() for k in ("o", "f", "i", "dy")}
+    d = {k: v.to(dev, non_blocking=True) for k, v in host.items()}
+    desc = binding.make_desc(w.B, w.H, w.N, w.dk, w.dv, binding.HGRN2_BF16, w.chunk, 0)
+    path = binding.path_of(desc)
+    shape_k, shape_v = (w.B, w.H, w.N, w.dk), (w.B, w.H, w.N, w.dv)
+    y = torch.empty(shape_v, dtype=bf, device=dev)
+    d_o = torch.empty(shape_k, dtype=bf, device=dev)
+    d_f = torch.empty(shape_k, dtype=bf, device=dev)
+    d_i = torch.empty(shape_v, dtype=bf, device=dev)
+    saved = binding.alloc_saved(desc, dev)
+    ws = binding.alloc_workspace(desc, dev)
+    host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in (("y", y), ("d_o", d_o), ("d_f", d_f), ("d_i", d_i))}
+    stream = torch.cuda.current_stream()
+
+    def fwd():
+        binding.hgrn2_fwd(d["o"], d["f"], d["i"], None, y=y, saved=saved, ws=ws, want_final_state=False)
+
+    def bwd():
+        binding.hgrn2_bwd(d["o"], d["f"], d["i"], None, d["dy"], None, saved, d_o=d_o, d_f=d_f, d_i=d_i, ws=ws,
+                          want_dS0=False)
+
+    def step():
+        fwd(); bwd()
+
+    def e2e_step():
+        for k in ("o", "f", "i", "dy"):
+            d[k].copy_(host[k], non_blocking=True)
+        fwd(); bwd()
+        for k, t in (("y", y), ("d_o", d_o), ("d_f", d_f), ("d_i", d_i)):
+            host_out[k].copy_(t, non_blocking=True)
+
+    def timed(fn, n):
+        """n calls between two events on the launching stream; ms for the n calls."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
+    K, Wm = args.steps, max(args.warmup, 3)
+    for _ in range(Wm):
+        step()
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws) == 0, "device-side error during warm-up"
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_total = max_over_ranks(timed(step, K))
+    ms_fwd = max_over_ranks(timed(fwd, K))
+    ms_bwd = max_over_ranks(timed(bwd, K))
+    if rank == 0:
+        sampler.stop()
+    for _ in range(2):
+        e2e_step()
+    ms_e2e = max_over_ranks(timed(e2e_step, max(3, min(K, 10)))) / max(3, min(K, 10))
+    assert binding.hgrn2_poll(ws) == 0, "device-side error during the timed region"
+
+    ms_step = ms_total / K
+    tokens_per_step = world * w.tokens
+    value = tokens_per_step / (ms_step * 1e-3)
+    e2e_value = tokens_per_step / (ms_e2e * 1e-3)
+    ab = train_bytes(w)
+    fl = train_flops(w)
+    kern = {}
+    for name, ms in (("fwd", ms_fwd / K), ("bwd", ms_bwd / K)):
+        kern[name] = {"ms": ms, "GBps": ab[name] / (ms * 1e-3) / 1e9, "TFLOPs": fl[name] / (ms * 1e-3) / 1e12}
+    dom = "bwd" if kern["bwd"]["ms"] >= kern["fwd"]["ms"] else "fwd"
+    # roofline of the whole step: the slower of bytes at HBM bandwidth and FLOPs at dense bf16 peak
+    t_hbm = (ab["fwd"] + ab["bwd"]) / (peaks["hbm_gbs"] * 1e9)
+    t_tc = (fl["fwd"] + fl["bwd"]) / (peaks["bf16_tflops_sustained"] * 1e12)
+    roof_tokens = w.tokens / max(t_hbm, t_tc)
+    roofline = {
+        "bound": "hbm", "kernel": f"hgrn2_{dom} ({path})", "achieved": kern[dom]["GBps"], "peak": peaks["hbm_gbs"],
+        "unit": "GB/s", "frac": kern[dom]["GBps"] / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES[dom],
+        "peak_source": f"of {peak_kind}", "algorithmic_bytes_per_launch": ab[dom],
+        "frac_nominal": kern[dom]["GBps"] / NOMINAL["hbm_gbs"],
+        "step": {"roofline_tokens_per_s": roof_tokens, "frac": (value / world) / roof_tokens,
+                 "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6},
+        "kernels": kern,
+    }
+
+    # ---- decode: 512 consecutive one-token calls on the decode workload -------------------------
+    wd = W.CONFIGS["decode"]
+    T = wd.N
+    blk = 64
+    gates = {"o": [], "f": [], "i": []}
+    S0 = None
+    for b0 in range(0, T, blk):
+        dd = W.make_decode_inputs(wd, steps=min(blk, T - b0), seed=wd.seed + 1000 * rank + 7 * (b0 // blk))
+        if S0 is None:
+            S0 = dd["S0"]
+        for k in gates:
+            gates[k].append(torch.from_numpy(dd[k]).to(bf))
+    gates = {k: torch.cat(v, 0).to(dev) for k, v in gates.items()}
+    S = torch.from_numpy(S0).to(dev)
+    yd = torch.empty((T, wd.B, wd.H, wd.dv), dtype=bf, device=dev)
+
+    def decode_all():
+        for t in range(T):
+            binding.hgrn2_step(gates["o"][t], gates["f"][t], gates["i"][t], S, y=yd[t])
+
+    for t in range(8):
+        binding.hgrn2_step(gates["o"][t], gates["f"][t], gates["i"][t], S, y=yd[t])
+    S.copy_(torch.from_numpy(S0))
+    ms_dec = max_over_ranks(timed(decode_all, 1)) / T
+    db = decode_bytes(wd)
+    dec_gbps = db / (ms_dec * 1e-3) / 1e9
+    decode = {"workload": wd.name, "B": wd.B, "H": wd.H, "steps": T, "us_per_step": ms_dec * 1e3,
+              "value": dec_gbps, "unit": "GB/s", "tokens_per_s": world * wd.B / (ms_dec * 1e-3),
+              "roofline": {"bound": "hbm", "kernel": "hgrn2_step", "achieved": dec_gbps, "peak": peaks["hbm_gbs"],
+                           "unit": "GB/s", "frac": dec_gbps / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES["step"],
+                           "peak_source": f"of {peak_kind}", "frac_nominal": dec_gbps / NOMINAL["hbm_gbs"]}}
+
+    if world > 1:
+        dist.barrier()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- oracle on the host cores, bounded sample -------------------------------------------------
+    from oracle import ref
+    ref.build()
+    cores = ref.num_threads()
+    n_units = max(1, min(cores, w.B * w.H))
+    reps = 2
+    cpu_value, cpu_dt, cores = time_oracle(w, reps, 1, n_units)
+    cpu_baseline = {"value": cpu_value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                    "sample": f"{n_units} of {w.B * w.H} (batch, head) units of lm_2048 (N={w.N}), fwd+bwd in fp64, "
+                              f"{reps} timed repetitions of {cpu_dt:.2f} s, scaled by tokens"}
+
+    line = {
+        "metric": "HGRN2 layer fwd+bwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(w, path),
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "decode": decode,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in host.values()),
+                "d2h_bytes_per_step": sum(v.numel() * v.element_size() for v in host_out.values())},
+        "gpu_launches": 2 * K,
+        "clocks": sampler.summary(),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,136 @@
+/*
+ * hgrn2.h -- C ABI of the B200 (sm_100a) HGRN2 recurrence library.
+ *
+ * The library computes, per independent (batch, head) unit, the outer-product
+ * state-expanded gated linear recurrence of the paper's Eq. 3 (multi-head variant,
+ * Section 3.2), written with the state transposed (rows = gate dimension k,
+ * columns = input dimension v):
+ *
+ *     S_t = Diag(f_t) S_{t-1} + (1 - f_t)^T i_t          S_t in R^{dk x dv}
+ *     y_t = o_t S_t                                       (the updated state feeds y_t)
+ *
+ * i.e. linear attention with q = o, k = 1 - f, v = i and a per-key-dimension decay f
+ * (Table 4).  Eq. 3 carries no 1/sqrt(d) scale and none is applied.
+ *
+ * Conventions common to every call
+ *   - All data pointers are DEVICE pointers, 16-byte aligned, to dense row-major
+ *     tensors; the library never allocates, frees or copies host memory, never
+ *     synchronises, and enqueues work only on `cuda_stream` (a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream).  The caller owns every buffer and
+ *     must keep it alive until the stream has passed the call.
+ *   - Sequence tensors are [B][H][N][d] with d innermost; o and f have d = dk, i, y
+ *     and dy have d = dv.  Their element type is desc->io (float or bf16).
+ *   - State tensors S0, SN, dS0, dSN, S are [B][H][dk][dv] float32, dv innermost.
+ *   - f must lie in [0, 1].  The chunked kernels work with in-chunk cumulative decay
+ *     and treat f below 2^-100 as 2^-100; d_f divides by f and loses accuracy as
+ *     f -> 0 (it stays finite).
+ *   - Errors detected on the host (bad sizes, NULL or misaligned pointers, unsupported
+ *     shapes, too small a workspace) are returned at once and nothing is launched.
+ *     A failed launch returns HGRN2_ERR_CUDA.  Device-side problems (a bounded wait
+ *     that ran out) are written to the status word at the start of `ws` and reported
+ *     by hgrn2_poll after the caller has synchronised the stream.  Nothing aborts,
+ *     traps or throws.
+ *   - When B * H * N = 0 the sequence tensors have no elements and their pointers may be
+ *     NULL; with N = 0 the calls copy S0 to SN (and dSN to dS0).
+ *   - Supported shapes: dk, dv in {16, 32, 64, 128}; any B, H, N >= 1 (N = 0 is
+ *     accepted and does nothing).  bf16 I/O with dk = dv = 128 runs on the tcgen05
+ *     tensor-core kernels; everything else, and anything with
+ *     HGRN2_FLAG_FORCE_ALU, runs on the fp32 CUDA-core kernels.
+ */
+#ifndef HGRN2_H_
+#define HGRN2_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HGRN2_OK = 0,
+    HGRN2_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, negative size, bad enum */
+    HGRN2_ERR_UNSUPPORTED = 2,   /* shape / dtype / chunk the kernels do not cover            */
+    HGRN2_ERR_ALIGNMENT   = 3,   /* a pointer is not 16-byte aligned                          */
+    HGRN2_ERR_WORKSPACE   = 4,   /* workspace missing                                         */
+    HGRN2_ERR_CUDA        = 5,   /* a CUDA runtime call or launch failed                      */
+    HGRN2_ERR_TIMEOUT     = 6,   /* device side: a bounded wait expired (status word)         */
+    HGRN2_ERR_DOMAIN      = 7    /* device side: input outside the supported domain           */
+} hgrn2_status;
+
+typedef enum { HGRN2_F32 = 0, HGRN2_BF16 = 1 } hgrn2_dtype;
+
+/* desc->flags */
+#define HGRN2_FLAG_FORCE_ALU 1u  /* use the fp32 CUDA-core kernels even where tensor-core ones exist */
+
+/* Problem description shared by all calls.  `chunk` is the chunk length C of the
+ * chunkwise-parallel form (an implementation parameter: results agree for every
+ * supported value up to rounding); 0 selects the default. */
+typedef struct hgrn2_desc {
+    int32_t  B, H, N, dk, dv;
+    int32_t  io;      /* hgrn2_dtype of o, f, i, y, dy, d_o, d_f, d_i */
+    int32_t  chunk;
+    uint32_t flags;
+} hgrn2_desc;
+
+/* Bytes of the `saved` buffer that hgrn2_fwd fills for hgrn2_bwd: the state at the
+ * start of every chunk (derived from Eq. 3 by unrolling C steps).  0 on a bad desc. */
+size_t hgrn2_saved_bytes(const hgrn2_desc *desc);
+
+/* Bytes of the workspace `ws` every call takes: a 256-byte status block followed by
+ * room for the chunk states that hgrn2_bwd re-creates when it is given saved = NULL.
+ * 0 on a bad desc. */
+size_t hgrn2_workspace_bytes(const hgrn2_desc *desc);
+
+/* Forward over a whole sequence (Eq. 3 unrolled chunk by chunk; training and prefill).
+ *   o, f [B][H][N][dk], i [B][H][N][dv]  in   (desc->io)
+ *   S0   [B][H][dk][dv] float32          in,  NULL = zero initial state
+ *   y    [B][H][N][dv]                   out  (desc->io)
+ *   SN   [B][H][dk][dv] float32          out, NULL = not wanted
+ *   saved  hgrn2_saved_bytes(desc) bytes out, NULL = inference (nothing kept for backward)
+ *   ws     hgrn2_workspace_bytes(desc) bytes, scratch; its first word is the status word,
+ *          which this call clears on the stream before the kernel. */
+hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                       const float *S0, void *y, float *SN, void *saved, void *ws,
+                       void *cuda_stream);
+
+/* Backward of hgrn2_fwd: the vector-Jacobian product for L = <dy, y> + <dSN, S_N>
+ * (the paper delegates training to prior work and prints no backward; this is the
+ * reverse-mode derivative of Eq. 3, run chunk by chunk in reverse).
+ *   o, f, i, S0   as given to hgrn2_fwd
+ *   dy  [B][H][N][dv] in;  dSN [B][H][dk][dv] float32 in, NULL = zero
+ *   saved  the buffer hgrn2_fwd filled with the same desc, or NULL: the chunk states
+ *          are then re-created inside `ws`
+ *   d_o, d_f [B][H][N][dk], d_i [B][H][N][dv] out (desc->io).  d_f folds both paths of
+ *          f: the decay and the tied input gate k = 1 - f.
+ *   dS0 [B][H][dk][dv] float32 out, NULL = not wanted */
+hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                       const float *S0, const void *dy, const float *dSN, const void *saved,
+                       void *d_o, void *d_f, void *d_i, float *dS0, void *ws,
+                       void *cuda_stream);
+
+/* One decode step for every unit (Eq. 3 once; constant-size state, Section 1).
+ *   o, f [B][H][dk], i [B][H][dv] in (desc->io); desc->N is ignored
+ *   S    [B][H][dk][dv] float32, updated in place
+ *   y    [B][H][dv] out (desc->io), computed from the updated state */
+hgrn2_status hgrn2_step(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                        float *S, void *y, void *cuda_stream);
+
+/* Reads the device status word of `ws` (a device pointer) with a blocking copy.  Call it
+ * after synchronising the stream the work ran on.  Returns HGRN2_OK, HGRN2_ERR_TIMEOUT,
+ * HGRN2_ERR_DOMAIN, or HGRN2_ERR_CUDA if the copy itself failed. */
+hgrn2_status hgrn2_poll(const void *ws);
+
+/* Static, human-readable name of a status code. */
+const char *hgrn2_status_string(hgrn2_status s);
+
+/* Chunk length the library will use for this desc (resolves chunk = 0); 0 on a bad desc. */
+int32_t hgrn2_chunk(const hgrn2_desc *desc);
+
+/* Name of the kernel family that serves this desc: "alu" or "tcgen05"; "" on a bad desc. */
+const char *hgrn2_path(const hgrn2_desc *desc);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HGRN2_H_ */

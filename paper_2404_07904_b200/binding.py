@@ -1,0 +1,200 @@
+"""Thin Python binding of the C-ABI library (``include/hgrn2.h``): argument marshalling only.
+
+Tensors are ``torch`` CUDA tensors used purely as device memory; every step of the
+recurrence runs inside ``libhgrn2.so``.  There is no CPU or eager fallback: if the library
+is missing or fails to load, importing this module's functions raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libhgrn2.so")
+
+HGRN2_F32, HGRN2_BF16 = 0, 1
+FLAG_FORCE_ALU = 1
+
+STATUS_NAMES = {
+    0: "HGRN2_OK", 1: "HGRN2_ERR_INVALID_ARG", 2: "HGRN2_ERR_UNSUPPORTED", 3: "HGRN2_ERR_ALIGNMENT",
+    4: "HGRN2_ERR_WORKSPACE", 5: "HGRN2_ERR_CUDA", 6: "HGRN2_ERR_TIMEOUT", 7: "HGRN2_ERR_DOMAIN",
+}
+
+# Every symbol include/hgrn2.h declares.
+EXPORTS = (
+    "hgrn2_saved_bytes", "hgrn2_workspace_bytes", "hgrn2_fwd", "hgrn2_bwd", "hgrn2_step",
+    "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path",
+)
+
+
+class Hgrn2Error(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {STATUS_NAMES.get(code, code)} ({status_string(code)})")
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32),
+                ("dk", ctypes.c_int32), ("dv", ctypes.c_int32), ("io", ctypes.c_int32),
+                ("chunk", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libhgrn2.so (built in-tree by ``paper_2404_07904_b200.build``); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2404_07904_b200.build` "
+            "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, dp = ctypes.c_void_p, ctypes.POINTER(Desc)
+    lib.hgrn2_saved_bytes.restype = ctypes.c_size_t
+    lib.hgrn2_saved_bytes.argtypes = [dp]
+    lib.hgrn2_workspace_bytes.restype = ctypes.c_size_t
+    lib.hgrn2_workspace_bytes.argtypes = [dp]
+    lib.hgrn2_chunk.restype = ctypes.c_int32
+    lib.hgrn2_chunk.argtypes = [dp]
+    lib.hgrn2_path.restype = ctypes.c_char_p
+    lib.hgrn2_path.argtypes = [dp]
+    lib.hgrn2_status_string.restype = ctypes.c_char_p
+    lib.hgrn2_status_string.argtypes = [ctypes.c_int]
+    lib.hgrn2_poll.restype = ctypes.c_int
+    lib.hgrn2_poll.argtypes = [vp]
+    lib.hgrn2_fwd.restype = ctypes.c_int
+    lib.hgrn2_fwd.argtypes = [dp] + [vp] * 9
+    lib.hgrn2_bwd.restype = ctypes.c_int
+    lib.hgrn2_bwd.argtypes = [dp] + [vp] * 13
+    lib.hgrn2_step.restype = ctypes.c_int
+    lib.hgrn2_step.argtypes = [dp] + [vp] * 6
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load().hgrn2_status_string(int(code)).decode()
+
+
+def _io_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return HGRN2_F32
+    if t.dtype == torch.bfloat16:
+        return HGRN2_BF16
+    raise TypeError(f"unsupported I/O dtype {t.dtype}")
+
+
+def make_desc(B, H, N, dk, dv, io, chunk=0, flags=0) -> Desc:
+    return Desc(int(B), int(H), int(N), int(dk), int(dv), int(io), int(chunk), int(flags))
+
+
+def saved_bytes(desc: Desc) -> int:
+    return int(load().hgrn2_saved_bytes(ctypes.byref(desc)))
+
+
+def workspace_bytes(desc: Desc) -> int:
+    return int(load().hgrn2_workspace_bytes(ctypes.byref(desc)))
+
+
+def chunk_of(desc: Desc) -> int:
+    return int(load().hgrn2_chunk(ctypes.byref(desc)))
+
+
+def path_of(desc: Desc) -> str:
+    return load().hgrn2_path(ctypes.byref(desc)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("the library takes device pointers: tensor is not on a CUDA device")
+    if not t.is_contiguous():
+        raise ValueError("tensors must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise Hgrn2Error(code, what)
+
+
+def alloc_workspace(desc: Desc, device) -> torch.Tensor:
+    n = workspace_bytes(desc)
+    if n == 0:
+        raise Hgrn2Error(2, "hgrn2_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def alloc_saved(desc: Desc, device) -> torch.Tensor:
+    return torch.empty(max(saved_bytes(desc), 16), dtype=torch.uint8, device=device)
+
+
+def hgrn2_fwd(o, f, i, S0=None, *, y=None, SN=None, saved=None, ws=None, want_final_state=True,
+              save_for_backward=True, chunk=0, flags=0, stream=None):
+    """Forward over [B, H, N, d] tensors.  Returns (y, SN, saved, ws, desc); buffers that are not passed in
+    are allocated with torch (device memory only)."""
+    B, H, N, dk = o.shape
+    dv = i.shape[-1]
+    desc = make_desc(B, H, N, dk, dv, _io_code(o), chunk, flags)
+    dev = o.device
+    if y is None:
+        y = torch.empty((B, H, N, dv), dtype=o.dtype, device=dev)
+    if SN is None and want_final_state:
+        SN = torch.empty((B, H, dk, dv), dtype=torch.float32, device=dev)
+    if saved is None and save_for_backward:
+        saved = alloc_saved(desc, dev)
+    if ws is None:
+        ws = alloc_workspace(desc, dev)
+    code = load().hgrn2_fwd(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S0), _ptr(y), _ptr(SN),
+                            _ptr(saved), _ptr(ws), _stream(stream))
+    _check(code, "hgrn2_fwd")
+    return y, SN, saved, ws, desc
+
+
+def hgrn2_bwd(o, f, i, S0, dy, dSN=None, saved=None, *, d_o=None, d_f=None, d_i=None, dS0=None, ws=None,
+              want_dS0=True, chunk=0, flags=0, stream=None):
+    """Backward of hgrn2_fwd.  Returns (d_o, d_f, d_i, dS0, ws)."""
+    B, H, N, dk = o.shape
+    dv = i.shape[-1]
+    desc = make_desc(B, H, N, dk, dv, _io_code(o), chunk, flags)
+    dev = o.device
+    d_o = torch.empty_like(o) if d_o is None else d_o
+    d_f = torch.empty_like(f) if d_f is None else d_f
+    d_i = torch.empty_like(i) if d_i is None else d_i
+    if dS0 is None and want_dS0:
+        dS0 = torch.empty((B, H, dk, dv), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = alloc_workspace(desc, dev)
+    code = load().hgrn2_bwd(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S0), _ptr(dy), _ptr(dSN),
+                            _ptr(saved), _ptr(d_o), _ptr(d_f), _ptr(d_i), _ptr(dS0), _ptr(ws), _stream(stream))
+    _check(code, "hgrn2_bwd")
+    return d_o, d_f, d_i, dS0, ws
+
+
+def hgrn2_step(o, f, i, S, *, y=None, stream=None):
+    """One decode step on [B, H, d] gates; S [B, H, dk, dv] float32 is updated in place.  Returns y."""
+    B, H, dk = o.shape
+    dv = i.shape[-1]
+    desc = make_desc(B, H, 1, dk, dv, _io_code(o))
+    if y is None:
+        y = torch.empty((B, H, dv), dtype=o.dtype, device=o.device)
+    code = load().hgrn2_step(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S), _ptr(y), _stream(stream))
+    _check(code, "hgrn2_step")
+    return y
+
+
+def hgrn2_poll(ws: torch.Tensor) -> int:
+    """Device-side status of the last call that used `ws` (synchronise its stream first)."""
+    return int(load().hgrn2_poll(_ptr(ws)))

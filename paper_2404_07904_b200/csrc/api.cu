@@ -1,0 +1,222 @@
+// C ABI of the HGRN2 library: argument checks and dispatch.  Every step of the path runs in
+// the kernels of this directory; nothing here computes on the host.
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace hgrn2;
+
+namespace hgrn2 {
+// tensor-core family (chunk_tc.cu)
+bool        tc_supported(const hgrn2_desc *d);
+int         tc_default_chunk();
+bool        tc_chunk_supported(int C);
+size_t      tc_saved_bytes(const hgrn2_desc *d, int C);
+cudaError_t launch_tc_fwd(const SeqArgs &a);
+cudaError_t launch_tc_bwd(const SeqArgs &a);
+}  // namespace hgrn2
+
+namespace {
+
+bool dim_ok(int d) { return d == 16 || d == 32 || d == 64 || d == 128; }
+
+bool desc_ok(const hgrn2_desc *d)
+{
+    if (!d) return false;
+    if (d->B < 0 || d->H < 0 || d->N < 0) return false;
+    if (d->io != HGRN2_F32 && d->io != HGRN2_BF16) return false;
+    if (d->chunk < 0) return false;
+    return true;
+}
+
+bool use_tc(const hgrn2_desc *d)
+{
+    return !(d->flags & HGRN2_FLAG_FORCE_ALU) && tc_supported(d);
+}
+
+// 0 = unsupported
+int resolve_chunk(const hgrn2_desc *d)
+{
+    if (!desc_ok(d) || !dim_ok(d->dk) || !dim_ok(d->dv)) return 0;
+    if (use_tc(d)) {
+        if (d->chunk == 0) return tc_default_chunk();
+        return tc_chunk_supported(d->chunk) ? d->chunk : 0;
+    }
+    if (d->chunk == 0) return alu_default_chunk(d->dk, d->dv);
+    return alu_chunk_supported(d->dk, d->dv, d->chunk) ? d->chunk : 0;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+hgrn2_status check_ptrs(const void *const *req, int nreq, const void *const *opt, int nopt)
+{
+    for (int j = 0; j < nreq; ++j)
+        if (!req[j]) return HGRN2_ERR_INVALID_ARG;
+    for (int j = 0; j < nreq; ++j)
+        if (!aligned16(req[j])) return HGRN2_ERR_ALIGNMENT;
+    for (int j = 0; j < nopt; ++j)
+        if (opt[j] && !aligned16(opt[j])) return HGRN2_ERR_ALIGNMENT;
+    return HGRN2_OK;
+}
+
+size_t state_bytes(const hgrn2_desc *d) { return (size_t)d->B * d->H * d->dk * d->dv * sizeof(float); }
+
+size_t saved_bytes_for(const hgrn2_desc *d, int C)
+{
+    if (use_tc(d)) return tc_saved_bytes(d, C);
+    const size_t NC = ((size_t)d->N + C - 1) / C;
+    return (size_t)d->B * d->H * NC * d->dk * d->dv * sizeof(float);
+}
+
+void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream)
+{
+    memset(&a, 0, sizeof(a));
+    a.B = d->B; a.H = d->H; a.N = d->N; a.dk = d->dk; a.dv = d->dv; a.C = C;
+    a.NC = (d->N + C - 1) / C;
+    a.io = d->io;
+    a.stream = static_cast<cudaStream_t>(stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t hgrn2_chunk(const hgrn2_desc *desc) { return resolve_chunk(desc); }
+
+const char *hgrn2_path(const hgrn2_desc *desc)
+{
+    if (resolve_chunk(desc) == 0) return "";
+    return use_tc(desc) ? "tcgen05" : "alu";
+}
+
+size_t hgrn2_saved_bytes(const hgrn2_desc *desc)
+{
+    const int C = resolve_chunk(desc);
+    if (C == 0) return 0;
+    return saved_bytes_for(desc, C);
+}
+
+size_t hgrn2_workspace_bytes(const hgrn2_desc *desc)
+{
+    const int C = resolve_chunk(desc);
+    if (C == 0) return 0;
+    return sizeof(StatusBlock) + saved_bytes_for(desc, C);
+}
+
+const char *hgrn2_status_string(hgrn2_status s)
+{
+    switch (s) {
+        case HGRN2_OK:              return "ok";
+        case HGRN2_ERR_INVALID_ARG: return "invalid argument";
+        case HGRN2_ERR_UNSUPPORTED: return "unsupported shape, dtype or chunk";
+        case HGRN2_ERR_ALIGNMENT:   return "pointer not 16-byte aligned";
+        case HGRN2_ERR_WORKSPACE:   return "workspace missing";
+        case HGRN2_ERR_CUDA:        return "CUDA runtime error";
+        case HGRN2_ERR_TIMEOUT:     return "device-side wait timed out";
+        case HGRN2_ERR_DOMAIN:      return "input outside the supported domain";
+    }
+    return "unknown status";
+}
+
+hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                       const float *S0, void *y, float *SN, void *saved, void *ws, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    const int C = resolve_chunk(desc);
+    if (C == 0) return HGRN2_ERR_UNSUPPORTED;
+    if (!ws) return HGRN2_ERR_WORKSPACE;
+    const bool empty = (size_t)desc->B * desc->H * desc->N == 0;   // sequence tensors have no elements
+    const void *req[] = {ws, o, f, i, y};
+    const void *opt[] = {S0, SN, saved, o, f, i, y};
+    hgrn2_status st = check_ptrs(req, empty ? 1 : 5, opt, empty ? 7 : 3);
+    if (st != HGRN2_OK) return st;
+
+    SeqArgs a;
+    fill_args(a, desc, C, cuda_stream);
+    a.o = o; a.f = f; a.i = i; a.S0 = S0; a.y = y; a.SN = SN;
+    a.states = static_cast<float *>(saved);
+    a.status = static_cast<StatusBlock *>(ws);
+    if (cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+    if ((size_t)desc->B * desc->H == 0) return HGRN2_OK;
+    if (desc->N == 0) {
+        if (SN) {
+            cudaError_t e = S0 ? cudaMemcpyAsync(SN, S0, state_bytes(desc), cudaMemcpyDeviceToDevice, a.stream)
+                               : cudaMemsetAsync(SN, 0, state_bytes(desc), a.stream);
+            if (e != cudaSuccess) return HGRN2_ERR_CUDA;
+        }
+        return HGRN2_OK;
+    }
+    cudaError_t e = use_tc(desc) ? launch_tc_fwd(a) : launch_alu_fwd(a);
+    return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                       const float *S0, const void *dy, const float *dSN, const void *saved,
+                       void *d_o, void *d_f, void *d_i, float *dS0, void *ws, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    const int C = resolve_chunk(desc);
+    if (C == 0) return HGRN2_ERR_UNSUPPORTED;
+    if (!ws) return HGRN2_ERR_WORKSPACE;
+    const bool empty = (size_t)desc->B * desc->H * desc->N == 0;
+    const void *req[] = {ws, o, f, i, dy, d_o, d_f, d_i};
+    const void *opt[] = {S0, dSN, saved, dS0, o, f, i, dy, d_o, d_f, d_i};
+    hgrn2_status st = check_ptrs(req, empty ? 1 : 8, opt, empty ? 11 : 4);
+    if (st != HGRN2_OK) return st;
+
+    SeqArgs a;
+    fill_args(a, desc, C, cuda_stream);
+    a.o = o; a.f = f; a.i = i; a.S0 = S0; a.dy = dy; a.dSN = dSN;
+    a.d_o = d_o; a.d_f = d_f; a.d_i = d_i; a.dS0 = dS0;
+    a.status = static_cast<StatusBlock *>(ws);
+    if (cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+    if ((size_t)desc->B * desc->H == 0) return HGRN2_OK;
+    if (desc->N == 0) {
+        if (dS0) {
+            cudaError_t e = dSN ? cudaMemcpyAsync(dS0, dSN, state_bytes(desc), cudaMemcpyDeviceToDevice, a.stream)
+                                : cudaMemsetAsync(dS0, 0, state_bytes(desc), a.stream);
+            if (e != cudaSuccess) return HGRN2_ERR_CUDA;
+        }
+        return HGRN2_OK;
+    }
+    const bool tc = use_tc(desc);
+    if (saved) {
+        a.states = const_cast<float *>(static_cast<const float *>(saved));
+    } else {
+        // re-create the chunk-start states inside the workspace with a states-only forward
+        SeqArgs r = a;
+        r.y = nullptr; r.SN = nullptr;
+        r.states = reinterpret_cast<float *>(static_cast<char *>(ws) + sizeof(StatusBlock));
+        cudaError_t e = tc ? launch_tc_fwd(r) : launch_alu_fwd(r);
+        if (e != cudaSuccess) return HGRN2_ERR_CUDA;
+        a.states = r.states;
+    }
+    cudaError_t e = tc ? launch_tc_bwd(a) : launch_alu_bwd(a);
+    return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+hgrn2_status hgrn2_step(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                        float *S, void *y, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    if (!dim_ok(desc->dk) || !dim_ok(desc->dv)) return HGRN2_ERR_UNSUPPORTED;
+    const void *req[] = {o, f, i, S, y};
+    hgrn2_status st = check_ptrs(req, 5, nullptr, 0);
+    if (st != HGRN2_OK) return st;
+    StepArgs a;
+    a.B = desc->B; a.H = desc->H; a.dk = desc->dk; a.dv = desc->dv; a.io = desc->io;
+    a.o = o; a.f = f; a.i = i; a.S = S; a.y = y;
+    a.stream = static_cast<cudaStream_t>(cuda_stream);
+    return launch_step(a) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+hgrn2_status hgrn2_poll(const void *ws)
+{
+    if (!ws) return HGRN2_ERR_INVALID_ARG;
+    int32_t code = 0;
+    if (cudaMemcpy(&code, ws, sizeof(code), cudaMemcpyDeviceToHost) != cudaSuccess) return HGRN2_ERR_CUDA;
+    if (code < 0 || code > HGRN2_ERR_DOMAIN) return HGRN2_ERR_CUDA;
+    return static_cast<hgrn2_status>(code);
+}
+
+}  // extern "C"

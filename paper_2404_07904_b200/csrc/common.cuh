@@ -1,0 +1,75 @@
+// Shared device/host helpers of the HGRN2 library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hgrn2.h"
+
+namespace hgrn2 {
+
+// Smallest forget-gate value the chunked kernels distinguish from zero: below it the
+// in-chunk cumulative decay is formed as if f were this value.
+constexpr float kFMin = 7.888609052210118e-31f;   // 2^-100
+
+// Layout of the 256-byte status block at the start of every workspace.
+struct StatusBlock {
+    int32_t code;      // hgrn2_status, 0 = ok; first error wins
+    int32_t where;     // kernel-specific location tag of the first error
+    int32_t pad[62];
+};
+static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
+
+template <typename T> __device__ __forceinline__ float load_f(const T *p);
+template <> __device__ __forceinline__ float load_f<float>(const float *p) { return *p; }
+template <> __device__ __forceinline__ float load_f<__nv_bfloat16>(const __nv_bfloat16 *p)
+{
+    return __bfloat162float(*p);
+}
+
+template <typename T> __device__ __forceinline__ void store_f(T *p, float x);
+template <> __device__ __forceinline__ void store_f<float>(float *p, float x) { *p = x; }
+template <> __device__ __forceinline__ void store_f<__nv_bfloat16>(__nv_bfloat16 *p, float x)
+{
+    *p = __float2bfloat16_rn(x);
+}
+
+__device__ __forceinline__ void report_error(StatusBlock *sb, int code, int where)
+{
+    if (sb != nullptr && atomicCAS(&sb->code, 0, code) == 0) sb->where = where;
+}
+
+// ---- internal launchers (defined in the .cu files, called from api.cu) ----------------------
+
+struct SeqArgs {
+    int B, H, N, dk, dv, C, NC;
+    int io;                       // hgrn2_dtype
+    const void *o, *f, *i;        // inputs
+    const float *S0;              // nullable
+    void *y;                      // fwd out (nullable: states only)
+    float *SN;                    // nullable
+    float *states;                // [B*H][NC][dk][dv] chunk-start states: fwd writes (nullable), bwd reads
+    const void *dy;               // bwd
+    const float *dSN;             // nullable
+    void *d_o, *d_f, *d_i;        // bwd out
+    float *dS0;                   // nullable
+    StatusBlock *status;
+    cudaStream_t stream;
+};
+
+struct StepArgs {
+    int B, H, dk, dv, io;
+    const void *o, *f, *i;
+    float *S;
+    void *y;
+    cudaStream_t stream;
+};
+
+cudaError_t launch_step(const StepArgs &a);
+int         alu_default_chunk(int dk, int dv);
+bool        alu_chunk_supported(int dk, int dv, int C);
+cudaError_t launch_alu_fwd(const SeqArgs &a);
+cudaError_t launch_alu_bwd(const SeqArgs &a);
+
+}  // namespace hgrn2

@@ -1,0 +1,206 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle element by element.
+
+Tolerances (max-norm relative error per output tensor): 1e-4 for float32 I/O, 2e-2 for bf16 I/O with
+float32 state.  bf16 inputs are rounded once and both sides consume the rounded values.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2404_07904_b200 import binding, workloads as W
+from oracle import ref
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+# ---------------------------------------------------------------- decode step
+@pytest.mark.parametrize("B,H,dk,dv,io", [(3, 2, 128, 128, "bf16"), (2, 3, 64, 64, "f32"), (1, 1, 16, 128, "f32"),
+                                          (2, 1, 128, 16, "bf16"), (5, 4, 32, 64, "bf16"), (1, 2, 64, 32, "f32")])
+def test_step_matches_oracle(B, H, dk, dv, io):
+    w = W.scaled(W.CONFIGS["decode"], B=B, H=H, dk=dk, dv=dv, io=io)
+    d = W.make_decode_inputs(w, steps=6)
+    tdt = torch.float32 if io == "f32" else torch.bfloat16
+    Sbuf, S = G.canary((B, H, dk, dv), torch.float32)
+    S.copy_(torch.from_numpy(d["S0"]))
+    S_ref = d["S0"].astype(np.float64)
+    for t in range(6):
+        o, f, i = (torch.from_numpy(d[k][t]).cuda().to(tdt) for k in ("o", "f", "i"))
+        ybuf, y = G.canary((B, H, dv), tdt)
+        binding.hgrn2_step(o, f, i, S, y=y)
+        y_ref = ref.hgrn2_step(d["o"][t], d["f"][t], d["i"][t], S_ref)
+        assert G.rel_err(y.float().cpu().numpy(), y_ref) <= G.TOL[io]
+        assert G.canary_ok(ybuf)
+    assert G.rel_err(S.cpu().numpy(), S_ref) <= 1e-5
+    assert G.canary_ok(Sbuf)
+
+
+def test_step_continues_prefill_state():
+    # forward over N tokens, then decode steps from its S_N == forward over N + T tokens
+    w = W.scaled(W.CONFIGS["lm_2048"], B=2, H=2, N=200, has_S0=True)
+    inp = W.make_inputs(w)
+    t = G.to_dev(inp, "bf16")
+    m = 150
+    _, Sm, _, ws, _ = binding.hgrn2_fwd(t["o"][:, :, :m].contiguous(), t["f"][:, :, :m].contiguous(),
+                                        t["i"][:, :, :m].contiguous(), t["S0"], save_for_backward=False)
+    ys = []
+    for s in range(m, 200):
+        ys.append(binding.hgrn2_step(t["o"][:, :, s].contiguous(), t["f"][:, :, s].contiguous(),
+                                     t["i"][:, :, s].contiguous(), Sm))
+    torch.cuda.synchronize()
+    y_ref, SN_ref = ref.hgrn2_fwd(inp["o"], inp["f"], inp["i"], inp["S0"])
+    got = torch.stack(ys, dim=2).float().cpu().numpy()
+    assert G.rel_err(got, y_ref[:, :, m:]) <= 2e-2
+    assert G.rel_err(Sm.cpu().numpy(), SN_ref) <= 2e-2
+
+
+# ---------------------------------------------------------------- config 1 and the fp32 path
+def test_config1_tiny_f32():
+    w = W.CONFIGS["tiny_f32"]
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "f32", chunk=w.chunk)
+    errs = G.assert_close(got, G.oracle_fwd_bwd(inp), 1e-4, "config 1")
+    print("config1 errs", errs)
+
+
+@pytest.mark.parametrize("N", [1, 2, 63, 64, 65, 129])
+@pytest.mark.parametrize("d,chunk", [(64, 0), (64, 16), (128, 0), (16, 32)])
+def test_f32_shape_sweep(N, d, chunk):
+    w = W.scaled(W.CONFIGS["tiny_f32"], B=2, H=1, N=N, dk=d, dv=d, has_S0=(N % 2 == 1), has_dSN=(N % 2 == 1),
+                 seed=N + d, gamma=0.3)
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "f32", chunk=chunk)
+    G.assert_close(got, G.oracle_fwd_bwd(inp), 1e-4, f"N={N} d={d} chunk={chunk}")
+
+
+def test_f32_rectangular_state_and_recompute():
+    w = W.scaled(W.CONFIGS["tiny_f32"], B=1, H=3, N=100, dk=32, dv=128, has_S0=True, has_dSN=True, seed=7)
+    inp = W.make_inputs(w)
+    want = G.oracle_fwd_bwd(inp)
+    G.assert_close(G.gpu_fwd_bwd(inp, "f32"), want, 1e-4, "saved")
+    G.assert_close(G.gpu_fwd_bwd(inp, "f32", use_saved=False), want, 1e-4, "recomputed")
+
+
+def test_alu_path_bf16_io():
+    w = W.scaled(W.CONFIGS["lm_2048"], B=1, H=2, N=300, has_S0=True, has_dSN=True)
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "bf16", flags=binding.FLAG_FORCE_ALU)
+    G.assert_close(got, G.oracle_fwd_bwd(inp), 2e-2, "alu bf16")
+
+
+def test_f_zero_and_f_one_forward():
+    # f == 0: y_t = (sum_k o_tk) i_t whatever S0 is; f == 1: the state never moves.
+    w = W.scaled(W.CONFIGS["tiny_f32"], N=70, has_S0=True)
+    inp = W.make_inputs(w)
+    for fv in (0.0, 1.0):
+        inp["f"][:] = fv
+        t = G.to_dev(inp, "f32")
+        y, SN, _, ws, _ = binding.hgrn2_fwd(t["o"], t["f"], t["i"], t["S0"], save_for_backward=False)
+        torch.cuda.synchronize()
+        y_ref, SN_ref = ref.hgrn2_fwd(inp["o"], inp["f"], inp["i"], inp["S0"])
+        assert G.rel_err(y.cpu().numpy(), y_ref) <= 1e-4
+        assert G.rel_err(SN.cpu().numpy(), SN_ref) <= 1e-4
+
+
+def test_empty_sequence_and_empty_batch():
+    dev = "cuda"
+    S0 = torch.randn(2, 2, 64, 64, device=dev)
+    o = torch.empty(2, 2, 0, 64, device=dev); i = torch.empty(2, 2, 0, 64, device=dev)
+    y, SN, saved, ws, _ = binding.hgrn2_fwd(o, o, i, S0)
+    d_o, d_f, d_i, dS0, _ = binding.hgrn2_bwd(o, o, i, S0, i, S0, saved)
+    torch.cuda.synchronize()
+    assert torch.equal(SN, S0) and torch.equal(dS0, S0)
+    o = torch.empty(0, 2, 8, 64, device=dev)
+    binding.hgrn2_fwd(o, o, o, None)
+    torch.cuda.synchronize()
+
+
+def test_run_to_run_determinism():
+    w = W.scaled(W.CONFIGS["lm_2048"], B=1, H=3, N=257, has_S0=True, has_dSN=True)
+    inp = W.make_inputs(w)
+    a = G.gpu_fwd_bwd(inp, "bf16")
+    b = G.gpu_fwd_bwd(inp, "bf16")
+    for k in a:
+        np.testing.assert_array_equal(a[k], b[k])
+
+
+# ---------------------------------------------------------------- the library's default path for the LM configs
+def _check_units(inp, got, units, tol, what):
+    want = G.oracle_fwd_bwd(inp, units)
+    worst = {}
+    for (b, h), wu in want.items():
+        gu = {k: got[k][b:b + 1, h:h + 1] for k in wu}
+        errs = G.assert_close(gu, wu, tol, f"{what} unit {(b, h)}")
+        for k, v in errs.items():
+            worst[k] = max(worst.get(k, 0.0), v)
+    print(what, {k: f"{v:.2e}" for k, v in worst.items()})
+
+
+@pytest.mark.parametrize("N", [1, 63, 64, 65, 200, 512])
+def test_bf16_default_path_shape_sweep(N):
+    w = W.scaled(W.CONFIGS["lm_2048"], B=2, H=2, N=N, has_S0=(N % 2 == 0), has_dSN=(N % 2 == 0), seed=50 + N)
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "bf16")
+    G.assert_close(got, G.oracle_fwd_bwd(inp), 2e-2, f"bf16 N={N}")
+
+
+@pytest.mark.parametrize("gamma", [0.0, 0.5, 0.9, 0.99])
+def test_bf16_decay_sweep(gamma):
+    w = W.scaled(W.CONFIGS["lm_2560"], B=1, H=3, N=640)
+    inp = W.make_inputs(w, gamma=gamma)
+    got = G.gpu_fwd_bwd(inp, "bf16")
+    G.assert_close(got, G.oracle_fwd_bwd(inp), 2e-2, f"gamma={gamma}")
+
+
+def test_bf16_recompute_matches_saved():
+    w = W.scaled(W.CONFIGS["lm_2048"], B=1, H=2, N=400, has_S0=True, has_dSN=True)
+    inp = W.make_inputs(w)
+    a = G.gpu_fwd_bwd(inp, "bf16")
+    b = G.gpu_fwd_bwd(inp, "bf16", use_saved=False)
+    for k in a:
+        np.testing.assert_array_equal(a[k], b[k])
+
+
+def test_config2_full_size_sampled_units():
+    w = W.CONFIGS["lm_2048"]
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "bf16", check_canaries=True)
+    _check_units(inp, got, [(0, 0), (3, 7), (7, 15)], 2e-2, "config 2")
+    for k, v in got.items():
+        assert np.isfinite(v).all(), k
+
+
+def test_config3_long_context_sampled_units():
+    w = W.CONFIGS["long_16k"]
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "bf16")
+    _check_units(inp, got, [(0, 0), (1, 15)], 2e-2, "config 3")
+    for k, v in got.items():
+        assert np.isfinite(v).all(), k
+
+
+@pytest.mark.parametrize("gamma", W.LM_2560_GAMMAS)
+def test_config4_sampled_units(gamma):
+    w = W.scaled(W.CONFIGS["lm_2560"], B=2)          # 2 of the 8 sequences: every unit is independent
+    inp = W.make_inputs(w, gamma=gamma)
+    got = G.gpu_fwd_bwd(inp, "bf16")
+    _check_units(inp, got, [(0, 0), (1, 19)], 2e-2, f"config 4 gamma={gamma}")
+
+
+def test_config5_decode_full_batch():
+    w = W.CONFIGS["decode"]
+    T = 16
+    d = W.make_decode_inputs(w, steps=T)
+    S = torch.from_numpy(d["S0"]).cuda()
+    units = [(0, 0), (100, 7), (255, 15)]
+    S_ref = {u: d["S0"][u[0]:u[0] + 1, u[1]:u[1] + 1].astype(np.float64) for u in units}
+    for t in range(T):
+        o, f, i = (torch.from_numpy(d[k][t]).cuda().to(torch.bfloat16) for k in ("o", "f", "i"))
+        y = binding.hgrn2_step(o, f, i, S).float().cpu().numpy()
+        for (b, h) in units:
+            y_ref = ref.hgrn2_step(d["o"][t][b:b + 1, h:h + 1], d["f"][t][b:b + 1, h:h + 1],
+                                   d["i"][t][b:b + 1, h:h + 1], S_ref[(b, h)])
+            assert G.rel_err(y[b:b + 1, h:h + 1], y_ref) <= 2e-2
+    Sh = S.cpu().numpy()
+    for (b, h) in units:
+        assert G.rel_err(Sh[b:b + 1, h:h + 1], S_ref[(b, h)]) <= 1e-5
