@@ -193,6 +193,44 @@ def workload_config(w, path):
 # ------------------------------------------------------------------------------------------------
 # the CUDA arm
 # ------------------------------------------------------------------------------------------------
+def run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks, peak_kind, bf):
+    import torch
+    # ---- decode: 512 consecutive one-token calls on the decode workload -------------------------
+    wd = W.CONFIGS["decode"]
+    T = args.decode_steps if args.decode_steps > 0 else wd.N
+    blk = 64
+    gates = {"o": [], "f": [], "i": []}
+    S0 = None
+    for b0 in range(0, T, blk):
+        dd = W.make_decode_inputs(wd, steps=min(blk, T - b0), seed=wd.seed + 1000 * rank + 7 * (b0 // blk))
+        if S0 is None:
+            S0 = dd["S0"]
+        for k in gates:
+            gates[k].append(torch.from_numpy(dd[k]).to(bf))
+    gates = {k: torch.cat(v, 0).to(dev) for k, v in gates.items()}
+    S = torch.from_numpy(S0).to(dev)
+    yd = torch.empty((T, wd.B, wd.H, wd.dv), dtype=bf, device=dev)
+
+    def decode_all():
+        for t in range(T):
+            binding.hgrn2_step(gates["o"][t], gates["f"][t], gates["i"][t], S, y=yd[t])
+
+    for t in range(min(8, T)):
+        binding.hgrn2_step(gates["o"][t], gates["f"][t], gates["i"][t], S, y=yd[t])
+    S.copy_(torch.from_numpy(S0))
+    ms_dec = max_over_ranks(timed(decode_all, 1)) / T
+    db = decode_bytes(wd)
+    dec_gbps = db / (ms_dec * 1e-3) / 1e9
+    decode = {"workload": wd.name, "B": wd.B, "H": wd.H, "steps": T, "us_per_step": ms_dec * 1e3,
+              "value": dec_gbps, "unit": "GB/s", "tokens_per_s": world * wd.B / (ms_dec * 1e-3),
+              "roofline": {"bound": "hbm", "kernel": "hgrn2_step", "achieved": dec_gbps, "peak": peaks["hbm_gbs"],
+                           "unit": "GB/s", "frac": dec_gbps / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES["step"],
+                           "peak_source": f"of {peak_kind}", "frac_nominal": dec_gbps / NOMINAL["hbm_gbs"]}}
+    if args.only == "decode" and rank == 0:
+        print(json.dumps({"only": "decode", "decode": decode}), flush=True)
+    return decode
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -276,6 +314,9 @@ def run_cuda(args):
         return e0.elapsed_time(e1)
 
     K, Wm = args.steps, max(args.warmup, 3)
+    if args.only == "decode":
+        run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks, peak_kind, bf)
+        return 0
     for _ in range(Wm):
         step()
     torch.cuda.synchronize()
@@ -318,37 +359,11 @@ def run_cuda(args):
         "kernels": kern,
     }
 
-    # ---- decode: 512 consecutive one-token calls on the decode workload -------------------------
-    wd = W.CONFIGS["decode"]
-    T = wd.N
-    blk = 64
-    gates = {"o": [], "f": [], "i": []}
-    S0 = None
-    for b0 in range(0, T, blk):
-        dd = W.make_decode_inputs(wd, steps=min(blk, T - b0), seed=wd.seed + 1000 * rank + 7 * (b0 // blk))
-        if S0 is None:
-            S0 = dd["S0"]
-        for k in gates:
-            gates[k].append(torch.from_numpy(dd[k]).to(bf))
-    gates = {k: torch.cat(v, 0).to(dev) for k, v in gates.items()}
-    S = torch.from_numpy(S0).to(dev)
-    yd = torch.empty((T, wd.B, wd.H, wd.dv), dtype=bf, device=dev)
-
-    def decode_all():
-        for t in range(T):
-            binding.hgrn2_step(gates["o"][t], gates["f"][t], gates["i"][t], S, y=yd[t])
-
-    for t in range(8):
-        binding.hgrn2_step(gates["o"][t], gates["f"][t], gates["i"][t], S, y=yd[t])
-    S.copy_(torch.from_numpy(S0))
-    ms_dec = max_over_ranks(timed(decode_all, 1)) / T
-    db = decode_bytes(wd)
-    dec_gbps = db / (ms_dec * 1e-3) / 1e9
-    decode = {"workload": wd.name, "B": wd.B, "H": wd.H, "steps": T, "us_per_step": ms_dec * 1e3,
-              "value": dec_gbps, "unit": "GB/s", "tokens_per_s": world * wd.B / (ms_dec * 1e-3),
-              "roofline": {"bound": "hbm", "kernel": "hgrn2_step", "achieved": dec_gbps, "peak": peaks["hbm_gbs"],
-                           "unit": "GB/s", "frac": dec_gbps / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES["step"],
-                           "peak_source": f"of {peak_kind}", "frac_nominal": dec_gbps / NOMINAL["hbm_gbs"]}}
+    if args.only == "train":
+        if rank == 0:
+            print(json.dumps({"only": "train", "ms_per_step": ms_step, "kernels": kern}), flush=True)
+        return 0
+    decode = run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks, peak_kind, bf)
 
     if world > 1:
         dist.barrier()
@@ -392,6 +407,9 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--only", default="all", choices=["all", "train", "decode"],
+                    help="restrict the run to one part (for profiling); the JSON line is printed for 'all' only")
+    ap.add_argument("--decode-steps", type=int, default=0, help="decode calls to time (0 = the workload's 512)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
