@@ -1,11 +1,427 @@
-// tcgen05 tensor-core family: placeholder until the kernels land (nothing is served from here yet).
-#include "common.cuh"
+// Chunkwise HGRN2 forward / backward on the Blackwell tensor cores (tcgen05 + TMEM + TMA),
+// bf16 I/O, fp32 state, d_k = d_v = 128, chunk length C = 64.  One CTA per (batch, head) unit walks
+// the chunks in order with the running state resident in tensor memory.
+//
+// Mid-chunk reference frame.  Within a chunk let b_j = sum_{r<=j} log f_r (per key dimension) and
+// let m be the middle of the chunk (after local row 31).  Only two rescaled operands are formed:
+//
+//     Qs_t = q_t * exp(b_t - b_m)          Ks_s = k_s * exp(b_m - b_s)          (q = o, k = 1 - f)
+//
+// so that Qs_t . Ks_s = q_t k_s exp(b_t - b_s) for every pair, and with Pm = exp(b_m),
+// E = exp(b_C - b_m) (per key dimension):
+//
+//     A  = tril(Qs Ks^T)                       S' = Diag(Pm) S_in      (state in the mid frame)
+//     Y  = A V + Qs S'                         S_out = Diag(E) (S' + Ks^T V)
+//
+// The factors exp(b_t - b_m) are in-chunk cumulative PRODUCTS of f taken outward from the middle
+// (the linear-space image of the log-space cumulative sum): rows after m multiply by prod f, rows
+// before m divide by it.  Products are floored at 2^-100, so extreme decay inside half a chunk
+// (more than 2^100 across 32 steps) loses accuracy but never produces Inf or NaN.
+// Per chunk the state accumulator in TMEM is rescaled once, by E(previous chunk) * Pm(this chunk).
+//
+// Tensor-memory plan (512 columns): S' at columns [0,128) (lane = key dim, column = value dim),
+// Y at [128,256) and A at [256,320) in the M = 64 accumulator layout (row r -> lane 32*(r/16) + r%16).
+#include <cstdlib>
+
+#include "tc_common.cuh"
 
 namespace hgrn2 {
-bool        tc_supported(const hgrn2_desc *) { return false; }
-int         tc_default_chunk() { return 64; }
-bool        tc_chunk_supported(int C) { return C == 64; }
-size_t      tc_saved_bytes(const hgrn2_desc *, int) { return 0; }
-cudaError_t launch_tc_fwd(const SeqArgs &) { return cudaErrorNotSupported; }
+
+namespace {
+
+using namespace tc;
+
+constexpr int kC = 64;
+constexpr int kD = 128;
+constexpr int kThreads = 256;
+constexpr uint32_t kSlab = kC * 128;            // bytes of one slab of a [64][128] tile
+constexpr uint32_t kTile = 2 * kSlab;           // one [64][128] bf16 tile
+constexpr uint32_t kStateSlab = kD * 128;       // bytes of one slab of the [128][128] state copy
+constexpr uint32_t kStateTile = 2 * kStateSlab;
+constexpr float kProdFloor = 7.888609052210118e-31f;   // 2^-100
+
+constexpr uint32_t kColS = 0, kColY = 128, kColA = 256;
+constexpr uint32_t kTmemCols = 512;
+
+// ---- shared-memory map of the forward kernel (offsets from a 1024-byte aligned base) -------------
+constexpr int kFwdStages = 2;
+constexpr uint32_t kFwdStageBytes = 3 * kTile;                        // q, f, v
+constexpr uint32_t kFwdOffS = kFwdStages * kFwdStageBytes;            // bf16 copy of S'
+constexpr uint32_t kFwdOffP = kFwdOffS + kStateTile;                  // bf16 tril(A), one slab
+constexpr uint32_t kFwdOffTot = kFwdOffP + kSlab;                     // float tot[4][128]
+constexpr uint32_t kFwdOffPm = kFwdOffTot + 4 * 128 * 4;              // float pm[128]
+constexpr uint32_t kFwdOffE = kFwdOffPm + 128 * 4;                    // float ee[128]
+constexpr uint32_t kFwdOffBar = kFwdOffE + 128 * 4;                   // mbarriers etc.
+constexpr uint32_t kFwdSmemBytes = kFwdOffBar + 128 + 1024;           // + alignment slack
+
+struct FwdCtl {
+    uint64_t full[kFwdStages];
+    uint64_t barA, barY;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// In-place rescaling of the raw o and f tiles of one chunk into Qs and Ks (see the file header).
+// Thread layout: 64 column pairs x 4 row quarters; quarter q owns rows 16q..16q+15.
+__device__ __forceinline__ void transform_chunk(uint8_t *qbuf, uint8_t *fbuf, float *tot, float *pm, float *ee,
+                                                int n_valid, int tid)
+{
+    const int quarter = tid >> 6, p = tid & 63;
+    const int col = 2 * p;
+    const uint32_t slab_off = (col >> 6) * kSlab;
+    const int jch = (col & 63) >> 3;
+    const uint32_t bic = (col & 7) * 2;
+    uint32_t qw[16];
+    float f0[16], f1[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int r = quarter * 16 + j;
+        const uint32_t off = slab_off + slab_chunk_off(r, jch) + bic;
+        uint32_t fw = *reinterpret_cast<const uint32_t *>(fbuf + off);
+        qw[j] = *reinterpret_cast<const uint32_t *>(qbuf + off);
+        if (r >= n_valid) {               // neutral padding token: f = 1, o = 0
+            fw = 0x3F803F80u;
+            qw[j] = 0u;
+        }
+        f0[j] = bf16_lo(fw);
+        f1[j] = bf16_hi(fw);
+    }
+    // m0[j], m1[j]: product of f over the rows strictly between row j and the middle of the chunk
+    // (quarters 0, 1: rows j+1 .. 31; quarters 2, 3: rows 32 .. j), restricted to this quarter.
+    float m0[16], m1[16];
+    float t0, t1;
+    if (quarter < 2) {
+        float a0 = 1.f, a1 = 1.f;
+#pragma unroll
+        for (int j = 15; j >= 0; --j) {
+            m0[j] = a0; m1[j] = a1;
+            a0 *= f0[j]; a1 *= f1[j];
+        }
+        t0 = a0; t1 = a1;
+    } else {
+        float a0 = 1.f, a1 = 1.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            a0 *= f0[j]; a1 *= f1[j];
+            m0[j] = a0; m1[j] = a1;
+        }
+        t0 = a0; t1 = a1;
+    }
+    tot[quarter * 128 + col] = t0;
+    tot[quarter * 128 + col + 1] = t1;
+    __syncthreads();
+    float o0 = 1.f, o1 = 1.f;
+    if (quarter == 0) { o0 = tot[128 + col]; o1 = tot[128 + col + 1]; }
+    if (quarter == 3) { o0 = tot[256 + col]; o1 = tot[256 + col + 1]; }
+    if (quarter == 0) { pm[col] = fmaxf(t0 * o0, kProdFloor); pm[col + 1] = fmaxf(t1 * o1, kProdFloor); }
+    if (quarter == 3) { ee[col] = fmaxf(t0 * o0, kProdFloor); ee[col + 1] = fmaxf(t1 * o1, kProdFloor); }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int r = quarter * 16 + j;
+        const uint32_t off = slab_off + slab_chunk_off(r, jch) + bic;
+        const float mm0 = fmaxf(m0[j] * o0, kProdFloor), mm1 = fmaxf(m1[j] * o1, kProdFloor);
+        const float i0 = __frcp_rn(mm0), i1 = __frcp_rn(mm1);
+        const float sq0 = quarter < 2 ? i0 : mm0, sq1 = quarter < 2 ? i1 : mm1;
+        const float sk0 = quarter < 2 ? mm0 : i0, sk1 = quarter < 2 ? mm1 : i1;
+        const float q0 = bf16_lo(qw[j]), q1 = bf16_hi(qw[j]);
+        *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(q0 * sq0, q1 * sq1);
+        *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0[j]) * sk0, (1.f - f1[j]) * sk1);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
+              const __grid_constant__ CUtensorMap map_i, const float *__restrict__ S0,
+              __nv_bfloat16 *__restrict__ y, float *__restrict__ SN, __nv_bfloat16 *__restrict__ saved, int N,
+              int NC, StatusBlock *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *sbuf = smem + kFwdOffS;
+    uint8_t *pbuf = smem + kFwdOffP;
+    float *tot = reinterpret_cast<float *>(smem + kFwdOffTot);
+    float *pm = reinterpret_cast<float *>(smem + kFwdOffPm);
+    float *ee = reinterpret_cast<float *>(smem + kFwdOffE);
+    FwdCtl *ctl = reinterpret_cast<FwdCtl *>(smem + kFwdOffBar);
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int u = blockIdx.x;
+    const int sub = warp & 3, half = warp >> 2;          // TMEM sub-partition and column half of this warp
+    const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
+
+    if (tid == 0) {
+        for (int s = 0; s < kFwdStages; ++s) mbar_init(&ctl->full[s], 1);
+        mbar_init(&ctl->barA, 1);
+        mbar_init(&ctl->barY, 1);
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&map_o);
+        tma_prefetch_desc(&map_f);
+        tma_prefetch_desc(&map_i);
+    }
+    if (warp == 0) tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+
+    auto issue_loads = [&](int c) {
+        const int s = c % kFwdStages;
+        uint8_t *st = smem + s * kFwdStageBytes;
+        mbar_arrive_expect_tx(&ctl->full[s], kFwdStageBytes);
+        for (int b = 0; b < 2; ++b) {
+            tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
+            tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
+            tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
+        }
+    };
+    if (tid == 0) {
+        for (int c = 0; c < kFwdStages && c < NC; ++c) issue_loads(c);
+    }
+
+    // S'' <- S0 (the accumulator holds the state of the previous frame, to be rescaled per chunk)
+    const int krow = 32 * sub + lane;
+    {
+        uint32_t r[32];
+        for (int part = 0; part < 2; ++part) {
+            const int v0 = 64 * half + 32 * part;
+            if (S0) {
+                const float4 *src = reinterpret_cast<const float4 *>(S0 + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 x = __ldg(src + j);
+                    r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
+                    r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
+            }
+            tmem_st32(tmem + lane_base + kColS + v0, r);
+        }
+        tmem_wait_st();
+    }
+    float e_prev = 1.f;
+
+    constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
+    constexpr uint32_t idescY1 = idesc_bf16(64, 128, 0, 1);    // Qs (K-major) x S' (MN-major)
+    constexpr uint32_t idescY2 = idesc_bf16(64, 128, 0, 1);    // P  (K-major) x V  (MN-major)
+    constexpr uint32_t idescS = idesc_bf16(128, 128, 1, 1);    // Ks^T (MN-major) x V (MN-major)
+
+    for (int c = 0; c < NC; ++c) {
+        const int s = c % kFwdStages;
+        uint8_t *qbuf = smem + s * kFwdStageBytes;
+        uint8_t *fbuf = qbuf + kTile;
+        uint8_t *vbuf = qbuf + 2 * kTile;
+        const int n_valid = min(kC, N - c * kC);
+        mbar_wait(&ctl->full[s], (c / kFwdStages) & 1, abort_flag);
+
+        transform_chunk(qbuf, fbuf, tot, pm, ee, n_valid, tid);
+        fence_proxy_async_smem();
+        __syncthreads();
+
+        // state maintenance: S' = (E_prev * Pm) S'', bf16 copy to shared memory (+ saved for backward)
+        {
+            const float factor = e_prev * pm[krow];
+            e_prev = ee[krow];
+            uint32_t r[32];
+            for (int part = 0; part < 2; ++part) {
+                const int v0 = 64 * half + 32 * part;
+                tmem_ld32(tmem + lane_base + kColS + v0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
+                tmem_st32(tmem + lane_base + kColS + v0, r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
+                    w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+                    w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+                    w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+                    const int jch = 4 * part + j;       // 16-byte chunk inside this half's slab row
+                    *reinterpret_cast<uint4 *>(sbuf + half * kStateSlab + slab_chunk_off(krow, jch)) = w;
+                    if (saved)
+                        *reinterpret_cast<uint4 *>(saved + (((size_t)u * NC + c) * kD + krow) * kD + v0 + 8 * j) = w;
+                }
+            }
+            tmem_wait_st();
+        }
+        tc_fence_before_sync();
+        fence_proxy_async_smem();
+        __syncthreads();
+
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const uint32_t qa = smem_u32(qbuf), fa = smem_u32(fbuf), va = smem_u32(vbuf), sa = smem_u32(sbuf);
+            if (y) {
+                for (int kk = 0; kk < 8; ++kk) {        // A = Qs Ks^T
+                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                    mma_bf16_ss(tmem + kColA, smem_desc_sw128(qa + koff, 16, 1024), smem_desc_sw128(fa + koff, 16, 1024),
+                                idescA, kk > 0);
+                }
+                mma_commit(&ctl->barA);
+                for (int kk = 0; kk < 8; ++kk) {        // Y = Qs S'
+                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                    mma_bf16_ss(tmem + kColY, smem_desc_sw128(qa + koff, 16, 1024),
+                                smem_desc_sw128(sa + kk * 2048, kStateSlab, 1024), idescY1, kk > 0);
+                }
+            }
+            for (int kk = 0; kk < 4; ++kk)              // S' += Ks^T V
+                mma_bf16_ss(tmem + kColS, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
+                            smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescS, 1);
+            if (!y) mma_commit(&ctl->barY);
+        }
+
+        if (y) {
+            // A epilogue: causal mask, bf16, K-major tile for the second product
+            mbar_wait(&ctl->barA, c & 1, abort_flag);
+            tc_fence_after_sync();
+            {
+                uint32_t r[32];
+                tmem_ld32(tmem + lane_base + kColA + 32 * half, r);
+                tmem_wait_ld();
+                if (lane < 16) {
+                    const int t = 16 * sub + lane;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int s0 = 32 * half + 8 * j;
+                        float x[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? __uint_as_float(r[8 * j + q]) : 0.f;
+                        uint4 w;
+                        w.x = pack_bf16(x[0], x[1]); w.y = pack_bf16(x[2], x[3]);
+                        w.z = pack_bf16(x[4], x[5]); w.w = pack_bf16(x[6], x[7]);
+                        *reinterpret_cast<uint4 *>(pbuf + slab_chunk_off(t, 4 * half + j)) = w;
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after_sync();
+                const uint32_t pa = smem_u32(pbuf), va = smem_u32(vbuf);
+                for (int kk = 0; kk < 4; ++kk)          // Y += P V
+                    mma_bf16_ss(tmem + kColY, smem_desc_sw128(pa + kk * 32, 16, 1024),
+                                smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescY2, 1);
+                mma_commit(&ctl->barY);
+            }
+        }
+
+        mbar_wait(&ctl->barY, c & 1, abort_flag);
+        tc_fence_after_sync();
+        if (y) {
+            uint32_t r[32];
+            const int t = 16 * sub + lane;
+            for (int part = 0; part < 2; ++part) {
+                const int v0 = 64 * half + 32 * part;
+                tmem_ld32(tmem + lane_base + kColY + v0, r);
+                tmem_wait_ld();
+                if (lane < 16 && t < n_valid) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(y + ((size_t)u * N + (size_t)c * kC + t) * kD + v0);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
+                        w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+                        w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+                        w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+                        dst[j] = w;
+                    }
+                }
+            }
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        if (tid == 0 && c + kFwdStages < NC) issue_loads(c + kFwdStages);
+    }
+
+    // S_N = Diag(E_last) S''
+    if (SN) {
+        tc_fence_after_sync();
+        uint32_t r[32];
+        for (int part = 0; part < 2; ++part) {
+            const int v0 = 64 * half + 32 * part;
+            tmem_ld32(tmem + lane_base + kColS + v0, r);
+            tmem_wait_ld();
+            float4 *dst = reinterpret_cast<float4 *>(SN + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * e_prev, __uint_as_float(r[4 * j + 1]) * e_prev,
+                                     __uint_as_float(r[4 * j + 2]) * e_prev, __uint_as_float(r[4 * j + 3]) * e_prev);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && *abort_flag) report_error(status, HGRN2_ERR_TIMEOUT, 1);
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [U][rows][128] bf16 tensor, tiles of [box_rows][64] with the 128-byte swizzle; rows beyond `rows`
+// read as zero.
+bool make_map(CUtensorMap *m, const void *base, uint64_t U, uint64_t rows, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {128, rows, U};
+    cuuint64_t strides[2] = {256, rows * 256};
+    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool tc_supported(const hgrn2_desc *d)
+{
+    static const bool enabled = getenv("HGRN2_TC") != nullptr;
+    return enabled && d->io == HGRN2_BF16 && d->dk == kD && d->dv == kD;
+}
+int  tc_default_chunk() { return kC; }
+bool tc_chunk_supported(int C) { return C == kC; }
+
+size_t tc_saved_bytes(const hgrn2_desc *d, int C)
+{
+    const size_t NC = ((size_t)d->N + C - 1) / C;
+    return (size_t)d->B * d->H * NC * kD * kD * sizeof(__nv_bfloat16);
+}
+
+cudaError_t launch_tc_fwd(const SeqArgs &a)
+{
+    const uint64_t U = (uint64_t)a.B * a.H;
+    CUtensorMap mo, mf, mi;
+    if (!make_map(&mo, a.o, U, a.N, kC) || !make_map(&mf, a.f, U, a.N, kC) || !make_map(&mi, a.i, U, a.N, kC))
+        return cudaErrorInvalidValue;
+    cudaError_t err = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmemBytes);
+    if (err != cudaSuccess) return err;
+    tc_fwd_kernel<<<(unsigned)U, kThreads, kFwdSmemBytes, a.stream>>>(
+        mo, mf, mi, a.S0, static_cast<__nv_bfloat16 *>(a.y), a.SN, reinterpret_cast<__nv_bfloat16 *>(a.states), a.N,
+        a.NC, a.status);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_tc_bwd(const SeqArgs &) { return cudaErrorNotSupported; }
+
 }  // namespace hgrn2
