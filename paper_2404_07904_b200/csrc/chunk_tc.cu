@@ -21,8 +21,6 @@
 //
 // Tensor-memory plan (512 columns): S' at columns [0,128) (lane = key dim, column = value dim),
 // Y at [128,256) and A at [256,320) in the M = 64 accumulator layout (row r -> lane 32*(r/16) + r%16).
-#include <cstdlib>
-
 #include "tc_common.cuh"
 
 namespace hgrn2 {
@@ -359,6 +357,414 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// ---- backward ---------------------------------------------------------------------------------------
+// Reverse sweep over the chunks with the state gradient resident in tensor memory.  In the mid frame
+// (file header), with dS'' = Diag(E) dS_out and S' the saved forward state of the chunk:
+//
+//   A  = tril(Qs Ks^T)          dA = tril(dY V^T)
+//   dQs^T       = Ks^T dA^T + S' dY^T            (accumulator [key dim][t]: lane = key dim)
+//   dKs_intra^T = Qs^T dA                        (accumulator [key dim][s])
+//   dKs_inter^T = dS'' V^T                       (accumulator [key dim][s])
+//   dV          = A^T dY + Ks dS''               (accumulator [s][value dim])
+//   dS'         = dS'' + Qs^T dY,   dS_in = Diag(Pm) dS'
+//   a = Qs*dQs - Ks*dKs_intra,  e = Ks*dKs_inter,  R_k = sum_v dS''[k,v] S'[k,v]
+//   dg_t = sum_{j>=t} a_j + sum_{s<t} e_s + R            (gradient w.r.t. log f_t; no cancellation
+//                                                         between the inter-chunk terms)
+//   d_o = dQs * exp(b_t - b_m),  dk = (dKs_intra + dKs_inter) * exp(b_m - b_s),  d_f = dg / f - dk
+//
+// The three key-dimension-major accumulators put one key dimension in each TMEM lane, so the thread
+// that owns the lane sees a whole column of the chunk and the scans along time stay in registers.
+// Tensor-memory plan: dS [0,128); A [128,192) and dA [192,256) first, then dQs^T and dKs_intra^T in
+// the same columns; dKs_inter^T [256,320); dV [320,448).
+constexpr int kBwdStages = 2;
+constexpr uint32_t kBwdStageBytes = 4 * kTile;                        // q, f, v, dy
+constexpr uint32_t kBwdOffS = kBwdStages * kBwdStageBytes;            // S' (bf16, from the forward)
+constexpr uint32_t kBwdOffDS = kBwdOffS + kStateTile;                 // bf16 copy of dS''
+constexpr uint32_t kBwdOffP = kBwdOffDS + kStateTile;                 // bf16 tril(A)
+constexpr uint32_t kBwdOffDP = kBwdOffP + kSlab;                      // bf16 tril(dA)
+constexpr uint32_t kBwdOffTot = kBwdOffDP + kSlab;                    // float tot[4][128]
+constexpr uint32_t kBwdOffPm = kBwdOffTot + 4 * 128 * 4;
+constexpr uint32_t kBwdOffE = kBwdOffPm + 128 * 4;
+constexpr uint32_t kBwdOffR = kBwdOffE + 128 * 4;                     // float rpart[2][128]
+constexpr uint32_t kBwdOffX = kBwdOffR + 2 * 128 * 4;                 // float xa[128], xe[128]
+constexpr uint32_t kBwdOffBar = kBwdOffX + 2 * 128 * 4;
+constexpr uint32_t kBwdSmemBytes = kBwdOffBar + 128 + 1024;
+
+constexpr uint32_t kColDS = 0, kColA2 = 128, kColDA = 192, kColDQ = 128, kColDKi = 192, kColDKx = 256, kColDV = 320;
+
+struct BwdCtl {
+    uint64_t full[kBwdStages];
+    uint64_t sfull, bar1, bar2;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
+              const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
+              const __grid_constant__ CUtensorMap map_saved, const __nv_bfloat16 *__restrict__ f_gmem,
+              const float *__restrict__ dSN, __nv_bfloat16 *__restrict__ d_o, __nv_bfloat16 *__restrict__ d_f,
+              __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N, int NC, StatusBlock *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *sbuf = smem + kBwdOffS;
+    uint8_t *dsbuf = smem + kBwdOffDS;
+    uint8_t *pbuf = smem + kBwdOffP;
+    uint8_t *dpbuf = smem + kBwdOffDP;
+    float *tot = reinterpret_cast<float *>(smem + kBwdOffTot);
+    float *pm = reinterpret_cast<float *>(smem + kBwdOffPm);
+    float *ee = reinterpret_cast<float *>(smem + kBwdOffE);
+    float *rpart = reinterpret_cast<float *>(smem + kBwdOffR);
+    float *xa = reinterpret_cast<float *>(smem + kBwdOffX);
+    float *xe = xa + 128;
+    BwdCtl *ctl = reinterpret_cast<BwdCtl *>(smem + kBwdOffBar);
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int u = blockIdx.x;
+    const int sub = warp & 3, half = warp >> 2;
+    const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
+
+    if (tid == 0) {
+        for (int s = 0; s < kBwdStages; ++s) mbar_init(&ctl->full[s], 1);
+        mbar_init(&ctl->sfull, 1);
+        mbar_init(&ctl->bar1, 1);
+        mbar_init(&ctl->bar2, 1);
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&map_o);
+        tma_prefetch_desc(&map_f);
+        tma_prefetch_desc(&map_i);
+        tma_prefetch_desc(&map_dy);
+        tma_prefetch_desc(&map_saved);
+    }
+    if (warp == 0) tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+
+    // it = 0, 1, ... counts processed chunks; chunk index c = NC - 1 - it
+    auto issue_loads = [&](int it) {
+        const int s = it % kBwdStages, c = NC - 1 - it;
+        uint8_t *st = smem + s * kBwdStageBytes;
+        mbar_arrive_expect_tx(&ctl->full[s], kBwdStageBytes);
+        for (int b = 0; b < 2; ++b) {
+            tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
+            tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
+            tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
+            tma_load_3d(st + 3 * kTile + b * kSlab, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
+        }
+    };
+    auto issue_state_load = [&](int it) {
+        const int c = NC - 1 - it;
+        mbar_arrive_expect_tx(&ctl->sfull, kStateTile);
+        for (int b = 0; b < 2; ++b) tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, u * NC + c);
+    };
+    if (tid == 0) {
+        for (int it = 0; it < kBwdStages && it < NC; ++it) issue_loads(it);
+        issue_state_load(0);
+    }
+
+    const int krow = 32 * sub + lane;
+    {
+        uint32_t r[32];
+        for (int part = 0; part < 2; ++part) {
+            const int v0 = 64 * half + 32 * part;
+            if (dSN) {
+                const float4 *src = reinterpret_cast<const float4 *>(dSN + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 x = __ldg(src + j);
+                    r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
+                    r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
+            }
+            tmem_st32(tmem + lane_base + kColDS + v0, r);
+        }
+        tmem_wait_st();
+    }
+    float pm_prev = 1.f;
+
+    constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T
+    constexpr uint32_t idKX = idesc_bf16(128, 64, 0, 0);      // dS'' (K-major) x V (K-major); S' x dY
+    constexpr uint32_t idDV2 = idesc_bf16(64, 128, 0, 1);     // Ks (K-major) x dS'' (MN-major)
+    constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
+    constexpr uint32_t idDQ1 = idesc_bf16(128, 64, 1, 0);     // Ks^T (MN-major) x dA^T (dP K-major)
+    constexpr uint32_t idDKi = idesc_bf16(128, 64, 1, 1);     // Qs^T (MN-major) x dA (dP MN-major)
+    constexpr uint32_t idDV1 = idesc_bf16(64, 128, 1, 1);     // P^T (MN-major) x dY (MN-major)
+
+    for (int it = 0; it < NC; ++it) {
+        const int c = NC - 1 - it;
+        const int s = it % kBwdStages;
+        uint8_t *qbuf = smem + s * kBwdStageBytes;
+        uint8_t *fbuf = qbuf + kTile;
+        uint8_t *vbuf = qbuf + 2 * kTile;
+        uint8_t *gbuf = qbuf + 3 * kTile;
+        const int n_valid = min(kC, N - c * kC);
+        mbar_wait(&ctl->full[s], (it / kBwdStages) & 1, abort_flag);
+
+        transform_chunk(qbuf, fbuf, tot, pm, ee, n_valid, tid);
+        fence_proxy_async_smem();
+        __syncthreads();
+
+        // dS'' = (Pm_prev * E) dS' (previous chunk's accumulator), bf16 copy, R partial sums
+        mbar_wait(&ctl->sfull, it & 1, abort_flag);
+        {
+            const float factor = pm_prev * ee[krow];
+            pm_prev = pm[krow];
+            float racc = 0.f;
+            uint32_t r[32];
+            for (int part = 0; part < 2; ++part) {
+                const int v0 = 64 * half + 32 * part;
+                tmem_ld32(tmem + lane_base + kColDS + v0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
+                tmem_st32(tmem + lane_base + kColDS + v0, r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int jch = 4 * part + j;
+                    const uint32_t off = half * kStateSlab + slab_chunk_off(krow, jch);
+                    const uint4 sw = *reinterpret_cast<const uint4 *>(sbuf + off);
+                    racc = fmaf(__uint_as_float(r[8 * j + 0]), bf16_lo(sw.x), racc);
+                    racc = fmaf(__uint_as_float(r[8 * j + 1]), bf16_hi(sw.x), racc);
+                    racc = fmaf(__uint_as_float(r[8 * j + 2]), bf16_lo(sw.y), racc);
+                    racc = fmaf(__uint_as_float(r[8 * j + 3]), bf16_hi(sw.y), racc);
+                    racc = fmaf(__uint_as_float(r[8 * j + 4]), bf16_lo(sw.z), racc);
+                    racc = fmaf(__uint_as_float(r[8 * j + 5]), bf16_hi(sw.z), racc);
+                    racc = fmaf(__uint_as_float(r[8 * j + 6]), bf16_lo(sw.w), racc);
+                    racc = fmaf(__uint_as_float(r[8 * j + 7]), bf16_hi(sw.w), racc);
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
+                    w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+                    w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+                    w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+                    *reinterpret_cast<uint4 *>(dsbuf + off) = w;
+                }
+            }
+            rpart[half * 128 + krow] = racc;
+            tmem_wait_st();
+        }
+        tc_fence_before_sync();
+        fence_proxy_async_smem();
+        __syncthreads();
+
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const uint32_t qa = smem_u32(qbuf), fa = smem_u32(fbuf), va = smem_u32(vbuf), ga = smem_u32(gbuf);
+            const uint32_t dsa = smem_u32(dsbuf);
+            for (int kk = 0; kk < 8; ++kk) {            // A = Qs Ks^T
+                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                mma_bf16_ss(tmem + kColA2, smem_desc_sw128(qa + koff, 16, 1024), smem_desc_sw128(fa + koff, 16, 1024),
+                            idA, kk > 0);
+            }
+            for (int kk = 0; kk < 8; ++kk) {            // dA = dY V^T
+                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                mma_bf16_ss(tmem + kColDA, smem_desc_sw128(ga + koff, 16, 1024), smem_desc_sw128(va + koff, 16, 1024),
+                            idA, kk > 0);
+            }
+            mma_commit(&ctl->bar1);
+            for (int kk = 0; kk < 8; ++kk) {            // dKs_inter^T = dS'' V^T
+                const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
+                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                mma_bf16_ss(tmem + kColDKx, smem_desc_sw128(dsa + ko_s, 16, 1024), smem_desc_sw128(va + koff, 16, 1024),
+                            idKX, kk > 0);
+            }
+            for (int kk = 0; kk < 8; ++kk) {            // dV = Ks dS''
+                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                mma_bf16_ss(tmem + kColDV, smem_desc_sw128(fa + koff, 16, 1024),
+                            smem_desc_sw128(dsa + kk * 2048, kStateSlab, 1024), idDV2, kk > 0);
+            }
+            for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
+                mma_bf16_ss(tmem + kColDS, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
+                            smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDS, 1);
+        }
+
+        // A and dA epilogue: causal mask, bf16 tiles P and dP
+        mbar_wait(&ctl->bar1, it & 1, abort_flag);
+        tc_fence_after_sync();
+        {
+            uint32_t r[32];
+            for (int which = 0; which < 2; ++which) {
+                tmem_ld32(tmem + lane_base + (which ? kColDA : kColA2) + 32 * half, r);
+                tmem_wait_ld();
+                if (lane < 16) {
+                    const int t = 16 * sub + lane;
+                    uint8_t *dstbuf = which ? dpbuf : pbuf;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int s0 = 32 * half + 8 * j;
+                        float x[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? __uint_as_float(r[8 * j + q]) : 0.f;
+                        uint4 w;
+                        w.x = pack_bf16(x[0], x[1]); w.y = pack_bf16(x[2], x[3]);
+                        w.z = pack_bf16(x[4], x[5]); w.w = pack_bf16(x[6], x[7]);
+                        *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = w;
+                    }
+                }
+            }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const uint32_t qa = smem_u32(qbuf), fa = smem_u32(fbuf), ga = smem_u32(gbuf);
+            const uint32_t sa = smem_u32(sbuf), pa = smem_u32(pbuf), dpa = smem_u32(dpbuf);
+            for (int kk = 0; kk < 4; ++kk)              // dQs^T = Ks^T dA^T
+                mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
+                            smem_desc_sw128(dpa + kk * 32, 16, 1024), idDQ1, kk > 0);
+            for (int kk = 0; kk < 8; ++kk) {            //        + S' dY^T
+                const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
+                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(sa + ko_s, 16, 1024), smem_desc_sw128(ga + koff, 16, 1024),
+                            idKX, 1);
+            }
+            for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
+                mma_bf16_ss(tmem + kColDKi, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
+                            smem_desc_sw128(dpa + kk * 2048, kSlab, 1024), idDKi, kk > 0);
+            for (int kk = 0; kk < 4; ++kk)              // dV += P^T dY
+                mma_bf16_ss(tmem + kColDV, smem_desc_sw128(pa + kk * 2048, kSlab, 1024),
+                            smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDV1, 1);
+            mma_commit(&ctl->bar2);
+        }
+
+        mbar_wait(&ctl->bar2, it & 1, abort_flag);
+        tc_fence_after_sync();
+        if (tid == 0 && it + 1 < NC) issue_state_load(it + 1);     // S' buffer is free again
+
+        // d_i = dV
+        {
+            uint32_t r[32];
+            const int t = 16 * sub + lane;
+            for (int part = 0; part < 2; ++part) {
+                const int v0 = 64 * half + 32 * part;
+                tmem_ld32(tmem + lane_base + kColDV + v0, r);
+                tmem_wait_ld();
+                if (lane < 16 && t < n_valid) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(d_i + ((size_t)u * N + (size_t)c * kC + t) * kD + v0);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
+                        w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+                        w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+                        w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+                        dst[j] = w;
+                    }
+                }
+            }
+        }
+
+        // d_o and d_f: thread (krow, half) owns key dimension krow and local times 32*half .. 32*half+31
+        {
+            const int tb = 32 * half;
+            const size_t gbase = ((size_t)u * N + (size_t)c * kC + tb) * kD + krow;
+            const uint32_t kslab = (krow >> 6) * kSlab;
+            const int kch = (krow & 63) >> 3;
+            const uint32_t kbic = (krow & 7) * 2;
+            float fv[32], m[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                fv[j] = (tb + j < n_valid) ? __bfloat162float(f_gmem[gbase + (size_t)j * kD]) : 1.f;
+            if (half == 0) {
+                float acc = 1.f;
+#pragma unroll
+                for (int j = 31; j >= 0; --j) { m[j] = fmaxf(acc, kProdFloor); acc *= fv[j]; }
+            } else {
+                float acc = 1.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) { acc *= fv[j]; m[j] = fmaxf(acc, kProdFloor); }
+            }
+            float a[32], dks[32], ev[32];
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + kColDQ + tb, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const uint32_t off = kslab + slab_chunk_off(tb + j, kch) + kbic;
+                const float qs = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(qbuf + off));
+                const float x = __uint_as_float(r[j]);
+                a[j] = qs * x;
+                const float sq = half == 0 ? __frcp_rn(m[j]) : m[j];
+                if (tb + j < n_valid) d_o[gbase + (size_t)j * kD] = __float2bfloat16_rn(x * sq);
+            }
+            tmem_ld32(tmem + lane_base + kColDKi + tb, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const uint32_t off = kslab + slab_chunk_off(tb + j, kch) + kbic;
+                const float ks = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(fbuf + off));
+                const float x = __uint_as_float(r[j]);
+                a[j] = fmaf(-ks, x, a[j]);
+                dks[j] = x;
+                ev[j] = ks;
+            }
+            tmem_ld32(tmem + lane_base + kColDKx + tb, r);
+            tmem_wait_ld();
+            float asum = 0.f, esum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float x = __uint_as_float(r[j]);
+                dks[j] += x;
+                ev[j] *= x;
+                asum += a[j];
+                esum += ev[j];
+            }
+            if (half == 1) xa[krow] = asum;       // each written by exactly one of the two threads of a key dim
+            if (half == 0) xe[krow] = esum;
+            __syncthreads();
+            const float R = rpart[krow] + rpart[128 + krow];
+            float pre = (half == 1) ? xe[krow] : 0.f;
+            float suf = (half == 0) ? xa[krow] : 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {        // exclusive prefix sums of e
+                const float e = ev[j];
+                ev[j] = pre;
+                pre += e;
+            }
+#pragma unroll
+            for (int j = 31; j >= 0; --j) {
+                suf += a[j];
+                const float dg = R + suf + ev[j];
+                const float sk = half == 0 ? m[j] : __frcp_rn(m[j]);
+                if (tb + j < n_valid)
+                    d_f[gbase + (size_t)j * kD] = __float2bfloat16_rn(dg / fmaxf(fv[j], kProdFloor) - dks[j] * sk);
+            }
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        if (tid == 0 && it + kBwdStages < NC) issue_loads(it + kBwdStages);
+    }
+
+    // dS_0 = Diag(Pm of chunk 0) dS'
+    if (dS0) {
+        tc_fence_after_sync();
+        uint32_t r[32];
+        for (int part = 0; part < 2; ++part) {
+            const int v0 = 64 * half + 32 * part;
+            tmem_ld32(tmem + lane_base + kColDS + v0, r);
+            tmem_wait_ld();
+            float4 *dst = reinterpret_cast<float4 *>(dS0 + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * pm_prev, __uint_as_float(r[4 * j + 1]) * pm_prev,
+                                     __uint_as_float(r[4 * j + 2]) * pm_prev, __uint_as_float(r[4 * j + 3]) * pm_prev);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && *abort_flag) report_error(status, HGRN2_ERR_TIMEOUT, 2);
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
 // ---- host side ------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -396,8 +802,7 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t U, uint64_t rows, uint3
 
 bool tc_supported(const hgrn2_desc *d)
 {
-    static const bool enabled = getenv("HGRN2_TC") != nullptr;
-    return enabled && d->io == HGRN2_BF16 && d->dk == kD && d->dv == kD;
+    return d->io == HGRN2_BF16 && d->dk == kD && d->dv == kD;
 }
 int  tc_default_chunk() { return kC; }
 bool tc_chunk_supported(int C) { return C == kC; }
@@ -422,6 +827,19 @@ cudaError_t launch_tc_fwd(const SeqArgs &a)
     return cudaGetLastError();
 }
 
-cudaError_t launch_tc_bwd(const SeqArgs &) { return cudaErrorNotSupported; }
+cudaError_t launch_tc_bwd(const SeqArgs &a)
+{
+    const uint64_t U = (uint64_t)a.B * a.H;
+    CUtensorMap mo, mf, mi, mg, ms;
+    if (!make_map(&mo, a.o, U, a.N, kC) || !make_map(&mf, a.f, U, a.N, kC) || !make_map(&mi, a.i, U, a.N, kC) ||
+        !make_map(&mg, a.dy, U, a.N, kC) || !make_map(&ms, a.states, U * a.NC, kD, kD))
+        return cudaErrorInvalidValue;
+    cudaError_t err = cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemBytes);
+    if (err != cudaSuccess) return err;
+    tc_bwd_kernel<<<(unsigned)U, kThreads, kBwdSmemBytes, a.stream>>>(
+        mo, mf, mi, mg, ms, static_cast<const __nv_bfloat16 *>(a.f), a.dSN, static_cast<__nv_bfloat16 *>(a.d_o),
+        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), a.dS0, a.N, a.NC, a.status);
+    return cudaGetLastError();
+}
 
 }  // namespace hgrn2

@@ -103,3 +103,75 @@ def test_chunk_form_matches_oracle(N, C, with_state):
     want = ref.hgrn2_bwd(o, f, i, S0, dy, dSN)
     for g, w in zip(got, want):
         np.testing.assert_allclose(g, w, rtol=1e-9, atol=1e-10)
+
+
+# --------------------------------------------------------------------------------------------------
+# The mid-chunk reference frame of the tensor-core kernels.  Only two rescaled operands exist,
+#   Qs_t = q_t exp(b_t - b_m),  Ks_s = k_s exp(b_m - b_s)      (m = middle of the chunk),
+# the state is carried as S' = Pm * S_in (Pm = exp(b_m)) and leaves as S_out = E * (S' + Ks^T V)
+# (E = exp(b_C - b_m)).  The decay gradient is formed from products in the same frame:
+#   a = Qs*dQs - Ks*dKs_intra,  e = Ks*dKs_inter,  R_k = sum_v dS''[k,v] S'[k,v],  dS'' = E * dS_out
+#   dg_t = sum_{j>=t} a_j + sum_{s<t} e_s + R
+# --------------------------------------------------------------------------------------------------
+def midframe_fwd_bwd(o, f, i, S0, dy, dSN, C):
+    B, H, N, dk = o.shape
+    dv = i.shape[-1]
+    assert N % C == 0
+    T = lambda x: np.swapaxes(x, -1, -2)
+    y = np.zeros((B, H, N, dv))
+    S = np.zeros((B, H, dk, dv)) if S0 is None else S0.copy()
+    saved = []
+    for c0 in range(0, N, C):
+        sl = slice(c0, c0 + C)
+        b = np.cumsum(np.log(f[:, :, sl]), axis=2)
+        bm = b[:, :, C // 2 - 1:C // 2]
+        Qs = o[:, :, sl] * np.exp(b - bm)
+        Ks = (1 - f[:, :, sl]) * np.exp(bm - b)
+        Pm, E = np.exp(bm[:, :, 0]), np.exp(b[:, :, -1] - bm[:, :, 0])
+        Sp = Pm[..., None] * S
+        saved.append(Sp)
+        y[:, :, sl] = np.tril(Qs @ T(Ks)) @ i[:, :, sl] + Qs @ Sp
+        S = E[..., None] * (Sp + T(Ks) @ i[:, :, sl])
+    SN = S
+    d_o, d_f, d_i = np.zeros_like(o), np.zeros_like(f), np.zeros_like(i)
+    dS_out = np.zeros((B, H, dk, dv)) if dSN is None else dSN.copy()
+    for ci in reversed(range(N // C)):
+        sl = slice(ci * C, ci * C + C)
+        fk, v, g = f[:, :, sl], i[:, :, sl], dy[:, :, sl]
+        b = np.cumsum(np.log(fk), axis=2)
+        bm = b[:, :, C // 2 - 1:C // 2]
+        sq, sk = np.exp(b - bm), np.exp(bm - b)
+        Qs, Ks = o[:, :, sl] * sq, (1 - fk) * sk
+        Pm, E = np.exp(bm[:, :, 0]), np.exp(b[:, :, -1] - bm[:, :, 0])
+        Sp = saved[ci]
+        dS2 = E[..., None] * dS_out
+        A = np.tril(Qs @ T(Ks))
+        dA = np.tril(g @ T(v))
+        dQs = dA @ Ks + g @ T(Sp)
+        dKs_intra = T(dA) @ Qs
+        dKs_inter = v @ T(dS2)
+        d_i[:, :, sl] = T(A) @ g + Ks @ dS2
+        a = Qs * dQs - Ks * dKs_intra
+        e = Ks * dKs_inter
+        R = (dS2 * Sp).sum(-1)
+        dg = np.flip(np.cumsum(np.flip(a, 2), 2), 2) + (np.cumsum(e, 2) - e) + R[:, :, None, :]
+        dkk = (dKs_intra + dKs_inter) * sk
+        d_o[:, :, sl] = dQs * sq
+        d_f[:, :, sl] = dg / fk - dkk
+        dS_out = Pm[..., None] * (dS2 + T(Qs) @ g)
+    return y, SN, d_o, d_f, d_i, dS_out
+
+
+@pytest.mark.parametrize("N,C", [(32, 8), (24, 4), (64, 64)])
+def test_mid_frame_form_matches_oracle(N, C):
+    r = np.random.default_rng(7 + N)
+    B, H, dk, dv = 1, 2, 6, 5
+    o = r.standard_normal((B, H, N, dk)); i = r.standard_normal((B, H, N, dv))
+    f = 0.3 + 0.7 / (1 + np.exp(-r.standard_normal((B, H, N, dk))))
+    dy = r.standard_normal(i.shape)
+    S0 = r.standard_normal((B, H, dk, dv)); dSN = r.standard_normal((B, H, dk, dv))
+    got = midframe_fwd_bwd(o, f, i, S0, dy, dSN, C)
+    y_ref, SN_ref = ref.hgrn2_fwd(o, f, i, S0)
+    want = (y_ref, SN_ref) + tuple(ref.hgrn2_bwd(o, f, i, S0, dy, dSN))
+    for g, w in zip(got, want):
+        np.testing.assert_allclose(g, w, rtol=1e-8, atol=1e-9)
