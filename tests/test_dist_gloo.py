@@ -1,0 +1,64 @@
+"""The N > 1 path on CPU: two gloo ranks shard the independent (batch, head) units, each runs its shard
+(the oracle stands in for the GPU kernels here), rank 0 gathers, and the result must equal the unsharded
+run bit for bit; the max-over-ranks timing reduction of bench.py is exercised the same way."""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+def _worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    os.environ["OMP_NUM_THREADS"] = "2"
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2404_07904_b200 import workloads as W
+    from oracle import ref
+    w = W.scaled(W.CONFIGS["tiny_f32"], B=3, H=2, N=40, dk=16, dv=16, has_S0=True)
+    inp = W.make_inputs(w)                      # same seed on every rank: the global problem
+    units = w.B * w.H
+    start, count = W.shard_units(units, world, rank)
+    flat = {k: (None if v is None else v.reshape(units, 1, *v.shape[2:])) for k, v in inp.items()}
+    sl = slice(start, start + count)
+    y, SN = ref.hgrn2_fwd(flat["o"][sl], flat["f"][sl], flat["i"][sl], flat["S0"][sl])
+    # gather shards on rank 0 (bench.py needs no data collective; this is only to check the sharding)
+    gathered = [None] * world
+    dist.gather_object((start, y), gathered if rank == 0 else None, dst=0)
+    # max-over-ranks timing, as bench.py does with its event times
+    t = torch.tensor([10.0 + rank], dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        full = np.concatenate([g[1] for g in sorted(gathered, key=lambda g: g[0])], axis=0)
+        np.save(os.path.join(out_dir, "y.npy"), full)
+        np.save(os.path.join(out_dir, "t.npy"), t.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_rank_unit_sharding_matches_single_process(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    from paper_2404_07904_b200 import workloads as W
+    from oracle import ref
+    w = W.scaled(W.CONFIGS["tiny_f32"], B=3, H=2, N=40, dk=16, dv=16, has_S0=True)
+    inp = W.make_inputs(w)
+    y, _ = ref.hgrn2_fwd(inp["o"], inp["f"], inp["i"], inp["S0"])
+    got = np.load(tmp_path / "y.npy").reshape(y.shape)
+    np.testing.assert_array_equal(got, y)
+    assert float(np.load(tmp_path / "t.npy")[0]) == 11.0
