@@ -109,6 +109,42 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
                        void *d_o, void *d_f, void *d_i, float *dS0, void *ws,
                        void *cuda_stream);
 
+/* Largest chunk-state scratch, in bytes, that hgrn2_bwd_static_scratch can serve. */
+#define HGRN2_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+
+/* Backward pass that allocates nothing and asks the caller for no scratch.  (The paper has no
+ * counterpart: this entry point exists for integration reasons only.)
+ *
+ * It is meant for callers that cannot obtain device memory at the point of the call: code that runs
+ * inside a serving process whose memory pool already owns all of the GPU's memory, plug-ins that
+ * are handed tensors but no allocator, and latency-critical loops where cudaMalloc / cudaFree are
+ * off limits because they may synchronise the whole device.  Such a caller has neither a `saved`
+ * buffer from the forward pass nor a workspace, so this variant of hgrn2_bwd re-creates the
+ * chunk-start states in a fixed array of HGRN2_STATIC_SCRATCH_BYTES (+ a 256-byte status block)
+ * that is compiled into the library; every GPU that loads the library holds that array until the
+ * process exits.  The call itself performs no cudaMalloc, cudaFree or other allocating call.
+ *
+ * Arguments are those of hgrn2_bwd without `saved` and `ws`; results are those of hgrn2_bwd.
+ *   status_out  device pointer to at least 8 bytes, 16-byte aligned, or NULL.  The device-side
+ *               status word of the call is copied there on the stream, for hgrn2_poll.
+ * Limits and caveats
+ *   - hgrn2_workspace_bytes(desc) - 256 must not exceed HGRN2_STATIC_SCRATCH_BYTES (bf16 d = 128:
+ *     B*H*ceil(N/64) <= 1024 chunk states); larger problems return HGRN2_ERR_WORKSPACE and nothing
+ *     is launched.  Use hgrn2_bwd with a caller-owned workspace for those.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in
+ *     it.  Each call clears the status block and overwrites every state it later reads, so stale
+ *     contents are never consumed; but two calls that can overlap on the GPU (different streams,
+ *     or different host threads without ordering) race on the array and must be serialised by
+ *     the caller.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress,
+ *     with that device current).  Make that first call outside any stream capture.
+ * Errors: as hgrn2_bwd, plus HGRN2_ERR_WORKSPACE as above and HGRN2_ERR_CUDA if the address
+ * lookup fails. */
+hgrn2_status hgrn2_bwd_static_scratch(const hgrn2_desc *desc, const void *o, const void *f,
+                                      const void *i, const float *S0, const void *dy,
+                                      const float *dSN, void *d_o, void *d_f, void *d_i,
+                                      float *dS0, void *status_out, void *cuda_stream);
+
 /* One decode step for every unit (Eq. 3 once; constant-size state, Section 1).
  *   o, f [B][H][dk], i [B][H][dv] in (desc->io); desc->N is ignored
  *   S    [B][H][dk][dv] float32, updated in place

@@ -26,8 +26,9 @@ STATUS_NAMES = {
 # Every symbol include/hgrn2.h declares.
 EXPORTS = (
     "hgrn2_saved_bytes", "hgrn2_workspace_bytes", "hgrn2_fwd", "hgrn2_bwd", "hgrn2_step",
-    "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path",
+    "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path", "hgrn2_bwd_static_scratch",
 )
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 
 class Hgrn2Error(RuntimeError):
@@ -72,6 +73,8 @@ def load() -> ctypes.CDLL:
     lib.hgrn2_fwd.argtypes = [dp] + [vp] * 9
     lib.hgrn2_bwd.restype = ctypes.c_int
     lib.hgrn2_bwd.argtypes = [dp] + [vp] * 13
+    lib.hgrn2_bwd_static_scratch.restype = ctypes.c_int
+    lib.hgrn2_bwd_static_scratch.argtypes = [dp] + [vp] * 12
     lib.hgrn2_step.restype = ctypes.c_int
     lib.hgrn2_step.argtypes = [dp] + [vp] * 6
     _lib = lib
@@ -181,6 +184,22 @@ def hgrn2_bwd(o, f, i, S0, dy, dSN=None, saved=None, *, d_o=None, d_f=None, d_i=
                             _ptr(saved), _ptr(d_o), _ptr(d_f), _ptr(d_i), _ptr(dS0), _ptr(ws), _stream(stream))
     _check(code, "hgrn2_bwd")
     return d_o, d_f, d_i, dS0, ws
+
+
+def hgrn2_bwd_static_scratch(o, f, i, S0, dy, dSN, d_o, d_f, d_i, dS0=None, status_out=None, *, chunk=0, flags=0,
+                             stream=None):
+    """Backward for callers that may not allocate: every buffer, outputs included, is passed in, and the
+    chunk-state scratch is the fixed array inside the library (problems whose states exceed
+    STATIC_SCRATCH_BYTES raise HGRN2_ERR_WORKSPACE).  This wrapper allocates nothing either.  Calls that
+    may overlap on the GPU share that array and must be serialised by the caller."""
+    B, H, N, dk = o.shape
+    dv = i.shape[-1]
+    desc = make_desc(B, H, N, dk, dv, _io_code(o), chunk, flags)
+    code = load().hgrn2_bwd_static_scratch(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S0), _ptr(dy),
+                                           _ptr(dSN), _ptr(d_o), _ptr(d_f), _ptr(d_i), _ptr(dS0), _ptr(status_out),
+                                           _stream(stream))
+    _check(code, "hgrn2_bwd_static_scratch")
+    return d_o, d_f, d_i, dS0
 
 
 def hgrn2_step(o, f, i, S, *, y=None, stream=None):
