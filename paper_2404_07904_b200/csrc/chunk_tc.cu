@@ -31,60 +31,74 @@ using namespace tc;
 
 constexpr int kC = 64;
 constexpr int kD = 128;
-constexpr int kThreads = 256;
+constexpr int kWorkers = 256;                   // warps 0..7: transforms, TMEM epilogues, outputs
+constexpr int kThreads = kWorkers + 32;         // warp 8: TMA loads and tcgen05.mma issue (one lane)
 constexpr uint32_t kSlab = kC * 128;            // bytes of one slab of a [64][128] tile
 constexpr uint32_t kTile = 2 * kSlab;           // one [64][128] bf16 tile
 constexpr uint32_t kStateSlab = kD * 128;       // bytes of one slab of the [128][128] state copy
 constexpr uint32_t kStateTile = 2 * kStateSlab;
 constexpr float kProdFloor = 7.888609052210118e-31f;   // 2^-100
-
-constexpr uint32_t kColS = 0, kColY = 128, kColA = 256;
 constexpr uint32_t kTmemCols = 512;
 
-// ---- shared-memory map of the forward kernel (offsets from a 1024-byte aligned base) -------------
-constexpr int kFwdStages = 2;
-constexpr uint32_t kFwdStageBytes = 3 * kTile;                        // q, f, v
-constexpr uint32_t kFwdOffS = kFwdStages * kFwdStageBytes;            // bf16 copy of S'
-constexpr uint32_t kFwdOffP = kFwdOffS + kStateTile;                  // bf16 tril(A), one slab
-constexpr uint32_t kFwdOffTot = kFwdOffP + kSlab;                     // float tot[4][128]
-constexpr uint32_t kFwdOffPm = kFwdOffTot + 4 * 128 * 4;              // float pm[128]
-constexpr uint32_t kFwdOffE = kFwdOffPm + 128 * 4;                    // float ee[128]
-constexpr uint32_t kFwdOffBar = kFwdOffE + 128 * 4;                   // mbarriers etc.
-constexpr uint32_t kFwdSmemBytes = kFwdOffBar + 128 + 1024;           // + alignment slack
+// Optional per-phase cycle counters of worker thread 0 of CTA 0 (development aid; compiled out unless
+// HGRN2_PHASE_TIMING is defined).  Totals land in the padding words of the status block.
+#ifdef HGRN2_PHASE_TIMING
+#define PT_DECL long long pt_t0 = clock64(); long long pt_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+#define PT_MARK(i) { const long long pt_t = clock64(); pt_acc[i] += pt_t - pt_t0; pt_t0 = pt_t; }
+#define PT_DUMP(st) if (tid == 0 && blockIdx.x == 0 && (st) != nullptr) { for (int pt_i = 0; pt_i < 12; ++pt_i) (st)->pad[pt_i] = (int)pt_acc[pt_i]; }
+#else
+#define PT_DECL
+#define PT_MARK(i)
+#define PT_DUMP(st)
+#endif
 
-struct FwdCtl {
-    uint64_t full[kFwdStages];
-    uint64_t barA, barY;
-    uint32_t tmem_base;
-    int abort_flag;
-};
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+__device__ __forceinline__ uint4 pack8(const uint32_t *r)
+{
+    uint4 w;
+    w.x = pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1]));
+    w.y = pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3]));
+    w.z = pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5]));
+    w.w = pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7]));
+    return w;
+}
 
 // In-place rescaling of the raw o and f tiles of one chunk into Qs and Ks (see the file header).
-// Thread layout: 64 column pairs x 4 row quarters; quarter q owns rows 16q..16q+15.
+// Thread layout: 64 column pairs x 4 row quarters; quarter q owns rows 16q..16q+15.  Quarter totals
+// go through `tot`; Pm and E of the chunk are left in `pm` and `ee`.  Called by all 256 workers.
 __device__ __forceinline__ void transform_chunk(uint8_t *qbuf, uint8_t *fbuf, float *tot, float *pm, float *ee,
                                                 int n_valid, int tid)
 {
     const int quarter = tid >> 6, p = tid & 63;
     const int col = 2 * p;
-    const uint32_t slab_off = (col >> 6) * kSlab;
     const int jch = (col & 63) >> 3;
-    const uint32_t bic = (col & 7) * 2;
+    const uint32_t base = (col >> 6) * kSlab + quarter * 16 * 128 + (col & 7) * 2;
+    uint32_t xo[8];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) xo[jj] = base + ((jch ^ jj) << 4);   // row 16q + j has (row & 7) == (j & 7)
     uint32_t qw[16];
     float f0[16], f1[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        const int r = quarter * 16 + j;
-        const uint32_t off = slab_off + slab_chunk_off(r, jch) + bic;
+        const uint32_t off = xo[j & 7] + j * 128;
         uint32_t fw = *reinterpret_cast<const uint32_t *>(fbuf + off);
         qw[j] = *reinterpret_cast<const uint32_t *>(qbuf + off);
-        if (r >= n_valid) {               // neutral padding token: f = 1, o = 0
+        if (quarter * 16 + j >= n_valid) {       // neutral padding token: f = 1, o = 0
             fw = 0x3F803F80u;
             qw[j] = 0u;
         }
         f0[j] = bf16_lo(fw);
         f1[j] = bf16_hi(fw);
     }
-    // m0[j], m1[j]: product of f over the rows strictly between row j and the middle of the chunk
+    // m0[j], m1[j]: product of f over the rows between row j and the middle of the chunk
     // (quarters 0, 1: rows j+1 .. 31; quarters 2, 3: rows 32 .. j), restricted to this quarter.
     float m0[16], m1[16];
     float t0, t1;
@@ -105,20 +119,20 @@ __device__ __forceinline__ void transform_chunk(uint8_t *qbuf, uint8_t *fbuf, fl
         }
         t0 = a0; t1 = a1;
     }
-    tot[quarter * 128 + col] = t0;
-    tot[quarter * 128 + col + 1] = t1;
-    __syncthreads();
+    *reinterpret_cast<float2 *>(tot + quarter * 128 + col) = make_float2(t0, t1);
+    worker_sync();
     float o0 = 1.f, o1 = 1.f;
-    if (quarter == 0) { o0 = tot[128 + col]; o1 = tot[128 + col + 1]; }
-    if (quarter == 3) { o0 = tot[256 + col]; o1 = tot[256 + col + 1]; }
-    if (quarter == 0) { pm[col] = fmaxf(t0 * o0, kProdFloor); pm[col + 1] = fmaxf(t1 * o1, kProdFloor); }
-    if (quarter == 3) { ee[col] = fmaxf(t0 * o0, kProdFloor); ee[col + 1] = fmaxf(t1 * o1, kProdFloor); }
+    if (quarter == 0) { const float2 x = *reinterpret_cast<const float2 *>(tot + 128 + col); o0 = x.x; o1 = x.y; }
+    if (quarter == 3) { const float2 x = *reinterpret_cast<const float2 *>(tot + 256 + col); o0 = x.x; o1 = x.y; }
+    if (quarter == 0)
+        *reinterpret_cast<float2 *>(pm + col) = make_float2(fmaxf(t0 * o0, kProdFloor), fmaxf(t1 * o1, kProdFloor));
+    if (quarter == 3)
+        *reinterpret_cast<float2 *>(ee + col) = make_float2(fmaxf(t0 * o0, kProdFloor), fmaxf(t1 * o1, kProdFloor));
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        const int r = quarter * 16 + j;
-        const uint32_t off = slab_off + slab_chunk_off(r, jch) + bic;
+        const uint32_t off = xo[j & 7] + j * 128;
         const float mm0 = fmaxf(m0[j] * o0, kProdFloor), mm1 = fmaxf(m1[j] * o1, kProdFloor);
-        const float i0 = __frcp_rn(mm0), i1 = __frcp_rn(mm1);
+        const float i0 = rcp_fast(mm0), i1 = rcp_fast(mm1);
         const float sq0 = quarter < 2 ? i0 : mm0, sq1 = quarter < 2 ? i1 : mm1;
         const float sk0 = quarter < 2 ? mm0 : i0, sk1 = quarter < 2 ? mm1 : i1;
         const float q0 = bf16_lo(qw[j]), q1 = bf16_hi(qw[j]);
@@ -126,6 +140,69 @@ __device__ __forceinline__ void transform_chunk(uint8_t *qbuf, uint8_t *fbuf, fl
         *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0[j]) * sk0, (1.f - f1[j]) * sk1);
     }
 }
+
+// Causal mask + bf16 of one 64 x 64 fp32 accumulator (M = 64 layout) into a K-major slab.
+__device__ __forceinline__ void tril_to_slab(uint32_t taddr, uint8_t *dstbuf, int sub, int half, int lane)
+{
+    uint32_t r[32];
+    tmem_ld32(taddr, r);
+    tmem_wait_ld();
+    if (lane < 16) {
+        const int t = 16 * sub + lane;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int s0 = 32 * half + 8 * j;
+            uint32_t x[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? r[8 * j + q] : 0u;
+            *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = pack8(x);
+        }
+    }
+}
+
+// One 64 x 128 fp32 accumulator (M = 64 layout) to a bf16 [token][128] global tensor.
+__device__ __forceinline__ void rows_to_global(uint32_t taddr_half, __nv_bfloat16 *dst_row0, int sub, int half,
+                                               int lane, int n_valid)
+{
+    uint32_t r[32];
+    const int t = 16 * sub + lane;
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+        tmem_ld32(taddr_half + 32 * part, r);
+        tmem_wait_ld();
+        if (lane < 16 && t < n_valid) {
+            uint4 *dst = reinterpret_cast<uint4 *>(dst_row0 + (size_t)t * kD + 64 * half + 32 * part);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j] = pack8(r + 8 * j);
+        }
+    }
+}
+
+// ---- forward ----------------------------------------------------------------------------------------
+// Skewed software pipeline.  The issuer lane keeps the tensor cores and TMA busy; the 256 workers run
+//   transform(c+1) | A epilogue(c) | state maintenance(c+1) | Y epilogue(c)
+// per iteration, so the MMAs of chunk c overlap the transform of chunk c+1, and the second product
+// Y += P V overlaps the maintenance.  Y is double-buffered in TMEM.
+constexpr int kFwdStages = 3;
+constexpr uint32_t kFwdStageBytes = 3 * kTile;                        // q, f, v
+constexpr uint32_t kFwdOffS = kFwdStages * kFwdStageBytes;            // bf16 copy of S'
+constexpr uint32_t kFwdOffP = kFwdOffS + kStateTile;                  // bf16 tril(A), one slab
+constexpr uint32_t kFwdOffTot = kFwdOffP + kSlab;                     // float tot[4][128]
+constexpr uint32_t kFwdOffPm = kFwdOffTot + 4 * 128 * 4;              // float pm[128]
+constexpr uint32_t kFwdOffE = kFwdOffPm + 128 * 4;                    // float ee[128]
+constexpr uint32_t kFwdOffBar = kFwdOffE + 128 * 4;                   // mbarriers etc.
+constexpr uint32_t kFwdSmemBytes = kFwdOffBar + 256 + 1024;           // + alignment slack
+
+constexpr uint32_t kColS = 0, kColY = 128 /* two buffers of 128 */, kColA = 384;
+
+struct FwdCtl {
+    uint64_t full[kFwdStages];     // TMA -> workers
+    uint64_t xs_ready;             // workers -> issuer: Qs, Ks, S' (TMEM + bf16 copy) of a chunk are in place
+    uint64_t p_ready;              // workers -> issuer: tril(A) is in shared memory
+    uint64_t barA, barS, barY[2];  // tcgen05.commit -> workers
+    uint32_t tmem_base;
+    int abort_flag;
+};
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
@@ -145,13 +222,15 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int u = blockIdx.x;
-    const int sub = warp & 3, half = warp >> 2;          // TMEM sub-partition and column half of this warp
-    const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
 
     if (tid == 0) {
         for (int s = 0; s < kFwdStages; ++s) mbar_init(&ctl->full[s], 1);
+        mbar_init(&ctl->xs_ready, kWorkers);
+        mbar_init(&ctl->p_ready, kWorkers);
         mbar_init(&ctl->barA, 1);
-        mbar_init(&ctl->barY, 1);
+        mbar_init(&ctl->barS, 1);
+        mbar_init(&ctl->barY[0], 1);
+        mbar_init(&ctl->barY[1], 1);
         ctl->abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
@@ -164,191 +243,178 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     tc_fence_after_sync();
     const uint32_t tmem = ctl->tmem_base;
 
-    auto issue_loads = [&](int c) {
-        const int s = c % kFwdStages;
-        uint8_t *st = smem + s * kFwdStageBytes;
-        mbar_arrive_expect_tx(&ctl->full[s], kFwdStageBytes);
-        for (int b = 0; b < 2; ++b) {
-            tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
-            tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
-            tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
-        }
-    };
-    if (tid == 0) {
-        for (int c = 0; c < kFwdStages && c < NC; ++c) issue_loads(c);
-    }
-
-    // S'' <- S0 (the accumulator holds the state of the previous frame, to be rescaled per chunk)
-    const int krow = 32 * sub + lane;
-    {
-        uint32_t r[32];
-        for (int part = 0; part < 2; ++part) {
-            const int v0 = 64 * half + 32 * part;
-            if (S0) {
-                const float4 *src = reinterpret_cast<const float4 *>(S0 + ((size_t)u * kD + krow) * kD + v0);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 x = __ldg(src + j);
-                    r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
-                    r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
+    if (warp == 8) {
+        // ================= issuer: TMA loads and MMA issue =================
+        if (lane == 0) {
+            constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
+            constexpr uint32_t idescY = idesc_bf16(64, 128, 0, 1);     // Qs or P (K-major) x S' or V (MN-major)
+            constexpr uint32_t idescS = idesc_bf16(128, 128, 1, 1);    // Ks^T (MN-major) x V (MN-major)
+            auto issue_loads = [&](int c) {
+                const int s = c % kFwdStages;
+                uint8_t *st = smem + s * kFwdStageBytes;
+                mbar_arrive_expect_tx(&ctl->full[s], kFwdStageBytes);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
                 }
-            } else {
+            };
+            for (int c = 0; c < kFwdStages && c < NC; ++c) issue_loads(c);
+            const uint32_t sa = smem_u32(sbuf), pa = smem_u32(pbuf);
+            for (int c = 0; c < NC; ++c) {
+                const uint32_t qa = smem_u32(smem + (c % kFwdStages) * kFwdStageBytes);
+                const uint32_t fa = qa + kTile, va = qa + 2 * kTile;
+                const uint32_t ty = tmem + kColY + 128 * (c & 1);
+                mbar_wait(&ctl->xs_ready, c & 1, abort_flag);
+                tc_fence_after_sync();
+                if (y) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    for (int kk = 0; kk < 8; ++kk) {        // A = Qs Ks^T
+                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                        mma_bf16_ss(tmem + kColA, smem_desc_sw128(qa + koff, 16, 1024),
+                                    smem_desc_sw128(fa + koff, 16, 1024), idescA, kk > 0);
+                    }
+                    mma_commit(&ctl->barA);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {        // Y = Qs S'
+                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                        mma_bf16_ss(ty, smem_desc_sw128(qa + koff, 16, 1024),
+                                    smem_desc_sw128(sa + kk * 2048, kStateSlab, 1024), idescY, kk > 0);
+                    }
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // S' += Ks^T V
+                    mma_bf16_ss(tmem + kColS, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
+                                smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescS, 1);
+                mma_commit(&ctl->barS);
+                if (y) {
+                    mbar_wait(&ctl->p_ready, c & 1, abort_flag);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)          // Y += P V
+                        mma_bf16_ss(ty, smem_desc_sw128(pa + kk * 32, 16, 1024),
+                                    smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescY, 1);
+                }
+                mma_commit(&ctl->barY[c & 1]);
+                // the stage of chunk c-1 is free once its MMAs are complete: refill it with chunk c+2
+                if (c >= 1 && c + kFwdStages - 1 < NC) {
+                    mbar_wait(&ctl->barY[(c - 1) & 1], ((c - 1) >> 1) & 1, abort_flag);
+                    issue_loads(c + kFwdStages - 1);
+                }
             }
-            tmem_st32(tmem + lane_base + kColS + v0, r);
         }
-        tmem_wait_st();
-    }
-    float e_prev = 1.f;
+    } else {
+        // ================= workers =================
+        const int sub = warp & 3, half = warp >> 2;      // TMEM sub-partition and column half of this warp
+        const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
+        const int krow = 32 * sub + lane;
+        float e_prev = 1.f;
 
-    constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
-    constexpr uint32_t idescY1 = idesc_bf16(64, 128, 0, 1);    // Qs (K-major) x S' (MN-major)
-    constexpr uint32_t idescY2 = idesc_bf16(64, 128, 0, 1);    // P  (K-major) x V  (MN-major)
-    constexpr uint32_t idescS = idesc_bf16(128, 128, 1, 1);    // Ks^T (MN-major) x V (MN-major)
-
-    for (int c = 0; c < NC; ++c) {
-        const int s = c % kFwdStages;
-        uint8_t *qbuf = smem + s * kFwdStageBytes;
-        uint8_t *fbuf = qbuf + kTile;
-        uint8_t *vbuf = qbuf + 2 * kTile;
-        const int n_valid = min(kC, N - c * kC);
-        mbar_wait(&ctl->full[s], (c / kFwdStages) & 1, abort_flag);
-
-        transform_chunk(qbuf, fbuf, tot, pm, ee, n_valid, tid);
-        fence_proxy_async_smem();
-        __syncthreads();
-
-        // state maintenance: S' = (E_prev * Pm) S'', bf16 copy to shared memory (+ saved for backward)
-        {
+        // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk); bf16 copy for the MMAs
+        // and for the backward pass; then hand the chunk to the issuer.
+        auto maintain = [&](int c, bool first) {
             const float factor = e_prev * pm[krow];
             e_prev = ee[krow];
             uint32_t r[32];
+#pragma unroll
             for (int part = 0; part < 2; ++part) {
                 const int v0 = 64 * half + 32 * part;
-                tmem_ld32(tmem + lane_base + kColS + v0, r);
-                tmem_wait_ld();
+                if (first) {
+                    if (S0) {
+                        const float4 *src = reinterpret_cast<const float4 *>(S0 + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 x = __ldg(src + j);
+                            r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
+                            r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    }
+                } else {
+                    tmem_ld32(tmem + lane_base + kColS + v0, r);
+                    tmem_wait_ld();
+                }
 #pragma unroll
                 for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
                 tmem_st32(tmem + lane_base + kColS + v0, r);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
-                    w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                    w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                    w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                    const int jch = 4 * part + j;       // 16-byte chunk inside this half's slab row
-                    *reinterpret_cast<uint4 *>(sbuf + half * kStateSlab + slab_chunk_off(krow, jch)) = w;
+                    const uint4 w = pack8(r + 8 * j);
+                    *reinterpret_cast<uint4 *>(sbuf + half * kStateSlab + slab_chunk_off(krow, 4 * part + j)) = w;
                     if (saved)
                         *reinterpret_cast<uint4 *>(saved + (((size_t)u * NC + c) * kD + krow) * kD + v0 + 8 * j) = w;
                 }
             }
             tmem_wait_st();
-        }
-        tc_fence_before_sync();
-        fence_proxy_async_smem();
-        __syncthreads();
-
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const uint32_t qa = smem_u32(qbuf), fa = smem_u32(fbuf), va = smem_u32(vbuf), sa = smem_u32(sbuf);
-            if (y) {
-                for (int kk = 0; kk < 8; ++kk) {        // A = Qs Ks^T
-                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                    mma_bf16_ss(tmem + kColA, smem_desc_sw128(qa + koff, 16, 1024), smem_desc_sw128(fa + koff, 16, 1024),
-                                idescA, kk > 0);
-                }
-                mma_commit(&ctl->barA);
-                for (int kk = 0; kk < 8; ++kk) {        // Y = Qs S'
-                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                    mma_bf16_ss(tmem + kColY, smem_desc_sw128(qa + koff, 16, 1024),
-                                smem_desc_sw128(sa + kk * 2048, kStateSlab, 1024), idescY1, kk > 0);
-                }
-            }
-            for (int kk = 0; kk < 4; ++kk)              // S' += Ks^T V
-                mma_bf16_ss(tmem + kColS, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
-                            smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescS, 1);
-            if (!y) mma_commit(&ctl->barY);
-        }
-
-        if (y) {
-            // A epilogue: causal mask, bf16, K-major tile for the second product
-            mbar_wait(&ctl->barA, c & 1, abort_flag);
-            tc_fence_after_sync();
-            {
-                uint32_t r[32];
-                tmem_ld32(tmem + lane_base + kColA + 32 * half, r);
-                tmem_wait_ld();
-                if (lane < 16) {
-                    const int t = 16 * sub + lane;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int s0 = 32 * half + 8 * j;
-                        float x[8];
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? __uint_as_float(r[8 * j + q]) : 0.f;
-                        uint4 w;
-                        w.x = pack_bf16(x[0], x[1]); w.y = pack_bf16(x[2], x[3]);
-                        w.z = pack_bf16(x[4], x[5]); w.w = pack_bf16(x[6], x[7]);
-                        *reinterpret_cast<uint4 *>(pbuf + slab_chunk_off(t, 4 * half + j)) = w;
-                    }
-                }
-            }
-            fence_proxy_async_smem();
             tc_fence_before_sync();
-            __syncthreads();
-            if (tid == 0) {
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->xs_ready);
+        };
+
+        mbar_wait(&ctl->full[0], 0, abort_flag);
+        transform_chunk(smem, smem + kTile, tot, pm, ee, min(kC, N), tid);
+        worker_sync();
+        maintain(0, true);
+        PT_DECL
+
+        for (int c = 0; c < NC; ++c) {
+            const int n_valid = min(kC, N - c * kC);
+            if (c + 1 < NC) {
+                const int s1 = (c + 1) % kFwdStages;
+                uint8_t *qbuf = smem + s1 * kFwdStageBytes;
+                mbar_wait(&ctl->full[s1], ((c + 1) / kFwdStages) & 1, abort_flag);
+                PT_MARK(0)
+                transform_chunk(qbuf, qbuf + kTile, tot, pm, ee, min(kC, N - (c + 1) * kC), tid);
+                worker_sync();
+                PT_MARK(1)
+            }
+            if (y) {
+                mbar_wait(&ctl->barA, c & 1, abort_flag);
                 tc_fence_after_sync();
-                const uint32_t pa = smem_u32(pbuf), va = smem_u32(vbuf);
-                for (int kk = 0; kk < 4; ++kk)          // Y += P V
-                    mma_bf16_ss(tmem + kColY, smem_desc_sw128(pa + kk * 32, 16, 1024),
-                                smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescY2, 1);
-                mma_commit(&ctl->barY);
+                PT_MARK(2)
+                tril_to_slab(tmem + lane_base + kColA + 32 * half, pbuf, sub, half, lane);
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                mbar_arrive(&ctl->p_ready);
+                PT_MARK(3)
+            }
+            if (c + 1 < NC) {
+                mbar_wait(&ctl->barS, c & 1, abort_flag);
+                tc_fence_after_sync();
+                PT_MARK(4)
+                maintain(c + 1, false);
+                PT_MARK(5)
+            }
+            if (y) {
+                mbar_wait(&ctl->barY[c & 1], (c >> 1) & 1, abort_flag);
+                tc_fence_after_sync();
+                PT_MARK(6)
+                rows_to_global(tmem + lane_base + kColY + 128 * (c & 1) + 64 * half,
+                               y + ((size_t)u * N + (size_t)c * kC) * kD, sub, half, lane, n_valid);
+                tc_fence_before_sync();
+                PT_MARK(7)
             }
         }
+        PT_DUMP(status)
 
-        mbar_wait(&ctl->barY, c & 1, abort_flag);
+        // S_N = Diag(E_last) S''
+        mbar_wait(&ctl->barS, (NC - 1) & 1, abort_flag);
         tc_fence_after_sync();
-        if (y) {
+        if (SN) {
             uint32_t r[32];
-            const int t = 16 * sub + lane;
+#pragma unroll
             for (int part = 0; part < 2; ++part) {
                 const int v0 = 64 * half + 32 * part;
-                tmem_ld32(tmem + lane_base + kColY + v0, r);
+                tmem_ld32(tmem + lane_base + kColS + v0, r);
                 tmem_wait_ld();
-                if (lane < 16 && t < n_valid) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(y + ((size_t)u * N + (size_t)c * kC + t) * kD + v0);
+                float4 *dst = reinterpret_cast<float4 *>(SN + ((size_t)u * kD + krow) * kD + v0);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
-                        w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                        w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                        w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                        dst[j] = w;
-                    }
-                }
+                for (int j = 0; j < 8; ++j)
+                    dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * e_prev, __uint_as_float(r[4 * j + 1]) * e_prev,
+                                         __uint_as_float(r[4 * j + 2]) * e_prev, __uint_as_float(r[4 * j + 3]) * e_prev);
             }
-        }
-        tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0 && c + kFwdStages < NC) issue_loads(c + kFwdStages);
-    }
-
-    // S_N = Diag(E_last) S''
-    if (SN) {
-        tc_fence_after_sync();
-        uint32_t r[32];
-        for (int part = 0; part < 2; ++part) {
-            const int v0 = 64 * half + 32 * part;
-            tmem_ld32(tmem + lane_base + kColS + v0, r);
-            tmem_wait_ld();
-            float4 *dst = reinterpret_cast<float4 *>(SN + ((size_t)u * kD + krow) * kD + v0);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * e_prev, __uint_as_float(r[4 * j + 1]) * e_prev,
-                                     __uint_as_float(r[4 * j + 2]) * e_prev, __uint_as_float(r[4 * j + 3]) * e_prev);
         }
     }
     tc_fence_before_sync();
@@ -376,6 +442,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 // that owns the lane sees a whole column of the chunk and the scans along time stay in registers.
 // Tensor-memory plan: dS [0,128); A [128,192) and dA [192,256) first, then dQs^T and dKs_intra^T in
 // the same columns; dKs_inter^T [256,320); dV [320,448).
+//
+// Worker schedule per processed chunk `it` (chunk index c = NC-1-it):
+//   P/dP epilogue(it) | transform(it+1) | dV epilogue(it), d_o/d_f phase(it) | dS maintenance(it+1)
+// so the second group of MMAs overlaps the next transform.  The raw-tile stage is released to TMA as
+// soon as the d_o/d_f phase has read Qs and Ks from it.
 constexpr int kBwdStages = 2;
 constexpr uint32_t kBwdStageBytes = 4 * kTile;                        // q, f, v, dy
 constexpr uint32_t kBwdOffS = kBwdStages * kBwdStageBytes;            // S' (bf16, from the forward)
@@ -388,13 +459,17 @@ constexpr uint32_t kBwdOffE = kBwdOffPm + 128 * 4;
 constexpr uint32_t kBwdOffR = kBwdOffE + 128 * 4;                     // float rpart[2][128]
 constexpr uint32_t kBwdOffX = kBwdOffR + 2 * 128 * 4;                 // float xa[128], xe[128]
 constexpr uint32_t kBwdOffBar = kBwdOffX + 2 * 128 * 4;
-constexpr uint32_t kBwdSmemBytes = kBwdOffBar + 128 + 1024;
+constexpr uint32_t kBwdSmemBytes = kBwdOffBar + 256 + 1024;
 
 constexpr uint32_t kColDS = 0, kColA2 = 128, kColDA = 192, kColDQ = 128, kColDKi = 192, kColDKx = 256, kColDV = 320;
 
 struct BwdCtl {
-    uint64_t full[kBwdStages];
-    uint64_t sfull, bar1, bar2;
+    uint64_t full[kBwdStages];     // TMA (raw tiles) -> workers
+    uint64_t sfull;                // TMA (saved S') -> workers
+    uint64_t g1_ready;             // workers -> issuer: Qs, Ks, dS'' ready: first MMA group may go
+    uint64_t pd_ready;             // workers -> issuer: tril(A), tril(dA) in shared memory: second group may go
+    uint64_t f_done;               // workers -> issuer: the chunk's stage has been read for the last time
+    uint64_t bar1, bar2;           // tcgen05.commit -> workers
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -423,12 +498,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int u = blockIdx.x;
-    const int sub = warp & 3, half = warp >> 2;
-    const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
 
     if (tid == 0) {
         for (int s = 0; s < kBwdStages; ++s) mbar_init(&ctl->full[s], 1);
         mbar_init(&ctl->sfull, 1);
+        mbar_init(&ctl->g1_ready, kWorkers);
+        mbar_init(&ctl->pd_ready, kWorkers);
+        mbar_init(&ctl->f_done, kWorkers);
         mbar_init(&ctl->bar1, 1);
         mbar_init(&ctl->bar2, 1);
         ctl->abort_flag = 0;
@@ -445,91 +521,141 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     tc_fence_after_sync();
     const uint32_t tmem = ctl->tmem_base;
 
-    // it = 0, 1, ... counts processed chunks; chunk index c = NC - 1 - it
-    auto issue_loads = [&](int it) {
-        const int s = it % kBwdStages, c = NC - 1 - it;
-        uint8_t *st = smem + s * kBwdStageBytes;
-        mbar_arrive_expect_tx(&ctl->full[s], kBwdStageBytes);
-        for (int b = 0; b < 2; ++b) {
-            tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
-            tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
-            tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
-            tma_load_3d(st + 3 * kTile + b * kSlab, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
-        }
-    };
-    auto issue_state_load = [&](int it) {
-        const int c = NC - 1 - it;
-        mbar_arrive_expect_tx(&ctl->sfull, kStateTile);
-        for (int b = 0; b < 2; ++b) tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, u * NC + c);
-    };
-    if (tid == 0) {
-        for (int it = 0; it < kBwdStages && it < NC; ++it) issue_loads(it);
-        issue_state_load(0);
-    }
-
-    const int krow = 32 * sub + lane;
-    {
-        uint32_t r[32];
-        for (int part = 0; part < 2; ++part) {
-            const int v0 = 64 * half + 32 * part;
-            if (dSN) {
-                const float4 *src = reinterpret_cast<const float4 *>(dSN + ((size_t)u * kD + krow) * kD + v0);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 x = __ldg(src + j);
-                    r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
-                    r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
+    if (warp == 8) {
+        // ================= issuer =================
+        if (lane == 0) {
+            constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T
+            constexpr uint32_t idKX = idesc_bf16(128, 64, 0, 0);      // dS'' (K-major) x V (K-major); S' x dY
+            constexpr uint32_t idDV2 = idesc_bf16(64, 128, 0, 1);     // Ks (K-major) x dS'' (MN-major)
+            constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
+            constexpr uint32_t idDQ1 = idesc_bf16(128, 64, 1, 0);     // Ks^T (MN-major) x dA^T (dP K-major)
+            constexpr uint32_t idDKi = idesc_bf16(128, 64, 1, 1);     // Qs^T (MN-major) x dA (dP MN-major)
+            constexpr uint32_t idDV1 = idesc_bf16(64, 128, 1, 1);     // P^T (MN-major) x dY (MN-major)
+            // it = 0, 1, ... counts processed chunks; chunk index c = NC - 1 - it
+            auto issue_loads = [&](int it) {
+                const int s = it % kBwdStages, c = NC - 1 - it;
+                uint8_t *st = smem + s * kBwdStageBytes;
+                mbar_arrive_expect_tx(&ctl->full[s], kBwdStageBytes);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + 3 * kTile + b * kSlab, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
                 }
-            } else {
+            };
+            auto issue_state_load = [&](int it) {
+                const int c = NC - 1 - it;
+                mbar_arrive_expect_tx(&ctl->sfull, kStateTile);
+                for (int b = 0; b < 2; ++b)
+                    tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, u * NC + c);
+            };
+            for (int it = 0; it < kBwdStages && it < NC; ++it) issue_loads(it);
+            issue_state_load(0);
+            const uint32_t sa = smem_u32(sbuf), dsa = smem_u32(dsbuf), pa = smem_u32(pbuf), dpa = smem_u32(dpbuf);
+            for (int it = 0; it < NC; ++it) {
+                const uint32_t qa = smem_u32(smem + (it % kBwdStages) * kBwdStageBytes);
+                const uint32_t fa = qa + kTile, va = qa + 2 * kTile, ga = qa + 3 * kTile;
+                mbar_wait(&ctl->g1_ready, it & 1, abort_flag);
+                tc_fence_after_sync();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = 0u;
+                for (int kk = 0; kk < 8; ++kk) {            // A = Qs Ks^T
+                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                    mma_bf16_ss(tmem + kColA2, smem_desc_sw128(qa + koff, 16, 1024),
+                                smem_desc_sw128(fa + koff, 16, 1024), idA, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {            // dA = dY V^T
+                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                    mma_bf16_ss(tmem + kColDA, smem_desc_sw128(ga + koff, 16, 1024),
+                                smem_desc_sw128(va + koff, 16, 1024), idA, kk > 0);
+                }
+                mma_commit(&ctl->bar1);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {            // dKs_inter^T = dS'' V^T
+                    const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
+                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                    mma_bf16_ss(tmem + kColDKx, smem_desc_sw128(dsa + ko_s, 16, 1024),
+                                smem_desc_sw128(va + koff, 16, 1024), idKX, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {            // dV = Ks dS''
+                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                    mma_bf16_ss(tmem + kColDV, smem_desc_sw128(fa + koff, 16, 1024),
+                                smem_desc_sw128(dsa + kk * 2048, kStateSlab, 1024), idDV2, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
+                    mma_bf16_ss(tmem + kColDS, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
+                                smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDS, 1);
+                mbar_wait(&ctl->pd_ready, it & 1, abort_flag);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dQs^T = Ks^T dA^T
+                    mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
+                                smem_desc_sw128(dpa + kk * 32, 16, 1024), idDQ1, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {            //        + S' dY^T
+                    const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
+                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                    mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(sa + ko_s, 16, 1024),
+                                smem_desc_sw128(ga + koff, 16, 1024), idKX, 1);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
+                    mma_bf16_ss(tmem + kColDKi, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
+                                smem_desc_sw128(dpa + kk * 2048, kSlab, 1024), idDKi, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dV += P^T dY
+                    mma_bf16_ss(tmem + kColDV, smem_desc_sw128(pa + kk * 2048, kSlab, 1024),
+                                smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDV1, 1);
+                mma_commit(&ctl->bar2);
+                // S' of this chunk is dead once the second group is complete: fetch the next one
+                mbar_wait(&ctl->bar2, it & 1, abort_flag);
+                if (it + 1 < NC) issue_state_load(it + 1);
+                // the raw-tile stage is dead once the workers have read Qs and Ks for d_o / d_f
+                mbar_wait(&ctl->f_done, it & 1, abort_flag);
+                if (it + kBwdStages < NC) issue_loads(it + kBwdStages);
             }
-            tmem_st32(tmem + lane_base + kColDS + v0, r);
         }
-        tmem_wait_st();
-    }
-    float pm_prev = 1.f;
+    } else {
+        // ================= workers =================
+        const int sub = warp & 3, half = warp >> 2;
+        const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
+        const int krow = 32 * sub + lane;
+        float pm_prev = 1.f;
 
-    constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T
-    constexpr uint32_t idKX = idesc_bf16(128, 64, 0, 0);      // dS'' (K-major) x V (K-major); S' x dY
-    constexpr uint32_t idDV2 = idesc_bf16(64, 128, 0, 1);     // Ks (K-major) x dS'' (MN-major)
-    constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
-    constexpr uint32_t idDQ1 = idesc_bf16(128, 64, 1, 0);     // Ks^T (MN-major) x dA^T (dP K-major)
-    constexpr uint32_t idDKi = idesc_bf16(128, 64, 1, 1);     // Qs^T (MN-major) x dA (dP MN-major)
-    constexpr uint32_t idDV1 = idesc_bf16(64, 128, 1, 1);     // P^T (MN-major) x dY (MN-major)
-
-    for (int it = 0; it < NC; ++it) {
-        const int c = NC - 1 - it;
-        const int s = it % kBwdStages;
-        uint8_t *qbuf = smem + s * kBwdStageBytes;
-        uint8_t *fbuf = qbuf + kTile;
-        uint8_t *vbuf = qbuf + 2 * kTile;
-        uint8_t *gbuf = qbuf + 3 * kTile;
-        const int n_valid = min(kC, N - c * kC);
-        mbar_wait(&ctl->full[s], (it / kBwdStages) & 1, abort_flag);
-
-        transform_chunk(qbuf, fbuf, tot, pm, ee, n_valid, tid);
-        fence_proxy_async_smem();
-        __syncthreads();
-
-        // dS'' = (Pm_prev * E) dS' (previous chunk's accumulator), bf16 copy, R partial sums
-        mbar_wait(&ctl->sfull, it & 1, abort_flag);
-        {
+        // dS'' = (Pm_prev E) dS' (the accumulator, or dSN first), bf16 copy, partial sums of R
+        auto maintain = [&](bool first) {
             const float factor = pm_prev * ee[krow];
             pm_prev = pm[krow];
             float racc = 0.f;
             uint32_t r[32];
+#pragma unroll
             for (int part = 0; part < 2; ++part) {
                 const int v0 = 64 * half + 32 * part;
-                tmem_ld32(tmem + lane_base + kColDS + v0, r);
-                tmem_wait_ld();
+                if (first) {
+                    if (dSN) {
+                        const float4 *src = reinterpret_cast<const float4 *>(dSN + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 x = __ldg(src + j);
+                            r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
+                            r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    }
+                } else {
+                    tmem_ld32(tmem + lane_base + kColDS + v0, r);
+                    tmem_wait_ld();
+                }
 #pragma unroll
                 for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
                 tmem_st32(tmem + lane_base + kColDS + v0, r);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int jch = 4 * part + j;
-                    const uint32_t off = half * kStateSlab + slab_chunk_off(krow, jch);
+                    const uint32_t off = half * kStateSlab + slab_chunk_off(krow, 4 * part + j);
                     const uint4 sw = *reinterpret_cast<const uint4 *>(sbuf + off);
                     racc = fmaf(__uint_as_float(r[8 * j + 0]), bf16_lo(sw.x), racc);
                     racc = fmaf(__uint_as_float(r[8 * j + 1]), bf16_hi(sw.x), racc);
@@ -539,224 +665,168 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     racc = fmaf(__uint_as_float(r[8 * j + 5]), bf16_hi(sw.z), racc);
                     racc = fmaf(__uint_as_float(r[8 * j + 6]), bf16_lo(sw.w), racc);
                     racc = fmaf(__uint_as_float(r[8 * j + 7]), bf16_hi(sw.w), racc);
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
-                    w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                    w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                    w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                    *reinterpret_cast<uint4 *>(dsbuf + off) = w;
+                    *reinterpret_cast<uint4 *>(dsbuf + off) = pack8(r + 8 * j);
                 }
             }
             rpart[half * 128 + krow] = racc;
             tmem_wait_st();
-        }
-        tc_fence_before_sync();
-        fence_proxy_async_smem();
-        __syncthreads();
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->g1_ready);
+        };
 
-        if (tid == 0) {
+        mbar_wait(&ctl->full[0], 0, abort_flag);
+        transform_chunk(smem, smem + kTile, tot, pm, ee, min(kC, N - (NC - 1) * kC), tid);
+        worker_sync();
+        mbar_wait(&ctl->sfull, 0, abort_flag);
+        maintain(true);
+        PT_DECL
+
+        for (int it = 0; it < NC; ++it) {
+            const int c = NC - 1 - it;
+            uint8_t *qbuf = smem + (it % kBwdStages) * kBwdStageBytes;
+            uint8_t *fbuf = qbuf + kTile;
+            const int n_valid = min(kC, N - c * kC);
+
+            // tril(A), tril(dA) -> shared memory
+            mbar_wait(&ctl->bar1, it & 1, abort_flag);
             tc_fence_after_sync();
-            const uint32_t qa = smem_u32(qbuf), fa = smem_u32(fbuf), va = smem_u32(vbuf), ga = smem_u32(gbuf);
-            const uint32_t dsa = smem_u32(dsbuf);
-            for (int kk = 0; kk < 8; ++kk) {            // A = Qs Ks^T
-                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                mma_bf16_ss(tmem + kColA2, smem_desc_sw128(qa + koff, 16, 1024), smem_desc_sw128(fa + koff, 16, 1024),
-                            idA, kk > 0);
-            }
-            for (int kk = 0; kk < 8; ++kk) {            // dA = dY V^T
-                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                mma_bf16_ss(tmem + kColDA, smem_desc_sw128(ga + koff, 16, 1024), smem_desc_sw128(va + koff, 16, 1024),
-                            idA, kk > 0);
-            }
-            mma_commit(&ctl->bar1);
-            for (int kk = 0; kk < 8; ++kk) {            // dKs_inter^T = dS'' V^T
-                const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
-                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                mma_bf16_ss(tmem + kColDKx, smem_desc_sw128(dsa + ko_s, 16, 1024), smem_desc_sw128(va + koff, 16, 1024),
-                            idKX, kk > 0);
-            }
-            for (int kk = 0; kk < 8; ++kk) {            // dV = Ks dS''
-                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                mma_bf16_ss(tmem + kColDV, smem_desc_sw128(fa + koff, 16, 1024),
-                            smem_desc_sw128(dsa + kk * 2048, kStateSlab, 1024), idDV2, kk > 0);
-            }
-            for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
-                mma_bf16_ss(tmem + kColDS, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
-                            smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDS, 1);
-        }
+            PT_MARK(0)
+            tril_to_slab(tmem + lane_base + kColA2 + 32 * half, pbuf, sub, half, lane);
+            tril_to_slab(tmem + lane_base + kColDA + 32 * half, dpbuf, sub, half, lane);
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->pd_ready);
+            PT_MARK(1)
 
-        // A and dA epilogue: causal mask, bf16 tiles P and dP
-        mbar_wait(&ctl->bar1, it & 1, abort_flag);
-        tc_fence_after_sync();
-        {
-            uint32_t r[32];
-            for (int which = 0; which < 2; ++which) {
-                tmem_ld32(tmem + lane_base + (which ? kColDA : kColA2) + 32 * half, r);
+            // next chunk's operands while the second MMA group runs
+            if (it + 1 < NC) {
+                const int s1 = (it + 1) % kBwdStages;
+                uint8_t *qn = smem + s1 * kBwdStageBytes;
+                mbar_wait(&ctl->full[s1], ((it + 1) / kBwdStages) & 1, abort_flag);
+                PT_MARK(2)
+                transform_chunk(qn, qn + kTile, tot, pm, ee, min(kC, N - (c - 1) * kC), tid);
+                worker_sync();
+                PT_MARK(3)
+            }
+
+            mbar_wait(&ctl->bar2, it & 1, abort_flag);
+            tc_fence_after_sync();
+            PT_MARK(4)
+
+            // d_i = dV
+            rows_to_global(tmem + lane_base + kColDV + 64 * half, d_i + ((size_t)u * N + (size_t)c * kC) * kD, sub,
+                           half, lane, n_valid);
+            PT_MARK(5)
+
+            // d_o and d_f: thread (krow, half) owns key dimension krow and local times 32*half .. 32*half+31
+            {
+                const int tb = 32 * half;
+                const size_t gbase = ((size_t)u * N + (size_t)c * kC + tb) * kD + krow;
+                const int kch = (krow & 63) >> 3;
+                const uint32_t kbase = (krow >> 6) * kSlab + tb * 128 + (krow & 7) * 2;
+                uint32_t xo[8];
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj) xo[jj] = kbase + ((kch ^ jj) << 4);    // (tb + j) & 7 == j & 7
+                float fv[32], m[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    fv[j] = (tb + j < n_valid) ? __bfloat162float(f_gmem[gbase + (size_t)j * kD]) : 1.f;
+                if (half == 0) {
+                    float acc = 1.f;
+#pragma unroll
+                    for (int j = 31; j >= 0; --j) { m[j] = fmaxf(acc, kProdFloor); acc *= fv[j]; }
+                } else {
+                    float acc = 1.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) { acc *= fv[j]; m[j] = fmaxf(acc, kProdFloor); }
+                }
+                float a[32], dks[32], ev[32];
+                uint32_t r[32];
+                tmem_ld32(tmem + lane_base + kColDQ + tb, r);
                 tmem_wait_ld();
-                if (lane < 16) {
-                    const int t = 16 * sub + lane;
-                    uint8_t *dstbuf = which ? dpbuf : pbuf;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int s0 = 32 * half + 8 * j;
-                        float x[8];
+                for (int j = 0; j < 32; ++j) {
+                    const float qs = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(qbuf + xo[j & 7] + j * 128));
+                    const float x = __uint_as_float(r[j]);
+                    a[j] = qs * x;
+                    const float mi = rcp_fast(m[j]);
+                    const float sq = half == 0 ? mi : m[j];
+                    m[j] = half == 0 ? m[j] : mi;            // from here on m holds exp(b_m - b_s)
+                    if (tb + j < n_valid) d_o[gbase + (size_t)j * kD] = __float2bfloat16_rn(x * sq);
+                }
+                tmem_ld32(tmem + lane_base + kColDKi + tb, r);
+                tmem_wait_ld();
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? __uint_as_float(r[8 * j + q]) : 0.f;
-                        uint4 w;
-                        w.x = pack_bf16(x[0], x[1]); w.y = pack_bf16(x[2], x[3]);
-                        w.z = pack_bf16(x[4], x[5]); w.w = pack_bf16(x[6], x[7]);
-                        *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = w;
-                    }
+                for (int j = 0; j < 32; ++j) {
+                    const float ks = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(fbuf + xo[j & 7] + j * 128));
+                    const float x = __uint_as_float(r[j]);
+                    a[j] = fmaf(-ks, x, a[j]);
+                    dks[j] = x;
+                    ev[j] = ks;
+                }
+                mbar_arrive(&ctl->f_done);          // last read of this chunk's stage
+                tmem_ld32(tmem + lane_base + kColDKx + tb, r);
+                tmem_wait_ld();
+                float asum = 0.f, esum = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float x = __uint_as_float(r[j]);
+                    dks[j] = (dks[j] + x) * m[j];
+                    ev[j] *= x;
+                    asum += a[j];
+                    esum += ev[j];
+                }
+                if (half == 1) xa[krow] = asum;       // each written by exactly one of the two threads of a key dim
+                if (half == 0) xe[krow] = esum;
+                const float R = rpart[krow] + rpart[128 + krow];
+                PT_MARK(6)
+                worker_sync();
+                PT_MARK(7)
+                float pre = (half == 1) ? xe[krow] : 0.f;
+                float suf = (half == 0) ? xa[krow] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {        // exclusive prefix sums of e
+                    const float e = ev[j];
+                    ev[j] = pre;
+                    pre += e;
+                }
+#pragma unroll
+                for (int j = 31; j >= 0; --j) {
+                    suf += a[j];
+                    const float dg = R + suf + ev[j];
+                    if (tb + j < n_valid)
+                        d_f[gbase + (size_t)j * kD] =
+                            __float2bfloat16_rn(fmaf(dg, rcp_fast(fmaxf(fv[j], kProdFloor)), -dks[j]));
                 }
             }
-        }
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();
+            tc_fence_before_sync();
+            PT_MARK(8)
 
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const uint32_t qa = smem_u32(qbuf), fa = smem_u32(fbuf), ga = smem_u32(gbuf);
-            const uint32_t sa = smem_u32(sbuf), pa = smem_u32(pbuf), dpa = smem_u32(dpbuf);
-            for (int kk = 0; kk < 4; ++kk)              // dQs^T = Ks^T dA^T
-                mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
-                            smem_desc_sw128(dpa + kk * 32, 16, 1024), idDQ1, kk > 0);
-            for (int kk = 0; kk < 8; ++kk) {            //        + S' dY^T
-                const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
-                const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(sa + ko_s, 16, 1024), smem_desc_sw128(ga + koff, 16, 1024),
-                            idKX, 1);
+            if (it + 1 < NC) {
+                mbar_wait(&ctl->sfull, (it + 1) & 1, abort_flag);
+                PT_MARK(9)
+                maintain(false);
+                PT_MARK(10)
             }
-            for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
-                mma_bf16_ss(tmem + kColDKi, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
-                            smem_desc_sw128(dpa + kk * 2048, kSlab, 1024), idDKi, kk > 0);
-            for (int kk = 0; kk < 4; ++kk)              // dV += P^T dY
-                mma_bf16_ss(tmem + kColDV, smem_desc_sw128(pa + kk * 2048, kSlab, 1024),
-                            smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDV1, 1);
-            mma_commit(&ctl->bar2);
         }
+        PT_DUMP(status)
 
-        mbar_wait(&ctl->bar2, it & 1, abort_flag);
-        tc_fence_after_sync();
-        if (tid == 0 && it + 1 < NC) issue_state_load(it + 1);     // S' buffer is free again
-
-        // d_i = dV
-        {
+        // dS_0 = Diag(Pm of chunk 0) dS'
+        if (dS0) {
+            tc_fence_after_sync();
             uint32_t r[32];
-            const int t = 16 * sub + lane;
+#pragma unroll
             for (int part = 0; part < 2; ++part) {
                 const int v0 = 64 * half + 32 * part;
-                tmem_ld32(tmem + lane_base + kColDV + v0, r);
+                tmem_ld32(tmem + lane_base + kColDS + v0, r);
                 tmem_wait_ld();
-                if (lane < 16 && t < n_valid) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(d_i + ((size_t)u * N + (size_t)c * kC + t) * kD + v0);
+                float4 *dst = reinterpret_cast<float4 *>(dS0 + ((size_t)u * kD + krow) * kD + v0);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
-                        w.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                        w.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                        w.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                        dst[j] = w;
-                    }
-                }
+                for (int j = 0; j < 8; ++j)
+                    dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * pm_prev, __uint_as_float(r[4 * j + 1]) * pm_prev,
+                                         __uint_as_float(r[4 * j + 2]) * pm_prev, __uint_as_float(r[4 * j + 3]) * pm_prev);
             }
-        }
-
-        // d_o and d_f: thread (krow, half) owns key dimension krow and local times 32*half .. 32*half+31
-        {
-            const int tb = 32 * half;
-            const size_t gbase = ((size_t)u * N + (size_t)c * kC + tb) * kD + krow;
-            const uint32_t kslab = (krow >> 6) * kSlab;
-            const int kch = (krow & 63) >> 3;
-            const uint32_t kbic = (krow & 7) * 2;
-            float fv[32], m[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                fv[j] = (tb + j < n_valid) ? __bfloat162float(f_gmem[gbase + (size_t)j * kD]) : 1.f;
-            if (half == 0) {
-                float acc = 1.f;
-#pragma unroll
-                for (int j = 31; j >= 0; --j) { m[j] = fmaxf(acc, kProdFloor); acc *= fv[j]; }
-            } else {
-                float acc = 1.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) { acc *= fv[j]; m[j] = fmaxf(acc, kProdFloor); }
-            }
-            float a[32], dks[32], ev[32];
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + kColDQ + tb, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const uint32_t off = kslab + slab_chunk_off(tb + j, kch) + kbic;
-                const float qs = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(qbuf + off));
-                const float x = __uint_as_float(r[j]);
-                a[j] = qs * x;
-                const float sq = half == 0 ? __frcp_rn(m[j]) : m[j];
-                if (tb + j < n_valid) d_o[gbase + (size_t)j * kD] = __float2bfloat16_rn(x * sq);
-            }
-            tmem_ld32(tmem + lane_base + kColDKi + tb, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const uint32_t off = kslab + slab_chunk_off(tb + j, kch) + kbic;
-                const float ks = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(fbuf + off));
-                const float x = __uint_as_float(r[j]);
-                a[j] = fmaf(-ks, x, a[j]);
-                dks[j] = x;
-                ev[j] = ks;
-            }
-            tmem_ld32(tmem + lane_base + kColDKx + tb, r);
-            tmem_wait_ld();
-            float asum = 0.f, esum = 0.f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float x = __uint_as_float(r[j]);
-                dks[j] += x;
-                ev[j] *= x;
-                asum += a[j];
-                esum += ev[j];
-            }
-            if (half == 1) xa[krow] = asum;       // each written by exactly one of the two threads of a key dim
-            if (half == 0) xe[krow] = esum;
-            __syncthreads();
-            const float R = rpart[krow] + rpart[128 + krow];
-            float pre = (half == 1) ? xe[krow] : 0.f;
-            float suf = (half == 0) ? xa[krow] : 0.f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {        // exclusive prefix sums of e
-                const float e = ev[j];
-                ev[j] = pre;
-                pre += e;
-            }
-#pragma unroll
-            for (int j = 31; j >= 0; --j) {
-                suf += a[j];
-                const float dg = R + suf + ev[j];
-                const float sk = half == 0 ? m[j] : __frcp_rn(m[j]);
-                if (tb + j < n_valid)
-                    d_f[gbase + (size_t)j * kD] = __float2bfloat16_rn(dg / fmaxf(fv[j], kProdFloor) - dks[j] * sk);
-            }
-        }
-        tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0 && it + kBwdStages < NC) issue_loads(it + kBwdStages);
-    }
-
-    // dS_0 = Diag(Pm of chunk 0) dS'
-    if (dS0) {
-        tc_fence_after_sync();
-        uint32_t r[32];
-        for (int part = 0; part < 2; ++part) {
-            const int v0 = 64 * half + 32 * part;
-            tmem_ld32(tmem + lane_base + kColDS + v0, r);
-            tmem_wait_ld();
-            float4 *dst = reinterpret_cast<float4 *>(dS0 + ((size_t)u * kD + krow) * kD + v0);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * pm_prev, __uint_as_float(r[4 * j + 1]) * pm_prev,
-                                     __uint_as_float(r[4 * j + 2]) * pm_prev, __uint_as_float(r[4 * j + 3]) * pm_prev);
         }
     }
     tc_fence_before_sync();
