@@ -7,7 +7,7 @@
 using namespace hgrn2;
 
 namespace hgrn2 {
-// tensor-core family (chunk_tc.cu)
+// tensor-core family (chunk_tc_fwd.cu, chunk_tc_bwd.cu)
 bool        tc_supported(const hgrn2_desc *d);
 int         tc_default_chunk();
 bool        tc_chunk_supported(int C);

@@ -1,27 +1,6 @@
-// Chunkwise HGRN2 forward / backward on the Blackwell tensor cores (tcgen05 + TMEM + TMA),
-// bf16 I/O, fp32 state, d_k = d_v = 128, chunk length C = 64.  One CTA per (batch, head) unit walks
-// the chunks in order with the running state resident in tensor memory.
-//
-// Mid-chunk reference frame.  Within a chunk let b_j = sum_{r<=j} log f_r (per key dimension) and
-// let m be the middle of the chunk (after local row 31).  Only two rescaled operands are formed:
-//
-//     Qs_t = q_t * exp(b_t - b_m)          Ks_s = k_s * exp(b_m - b_s)          (q = o, k = 1 - f)
-//
-// so that Qs_t . Ks_s = q_t k_s exp(b_t - b_s) for every pair, and with Pm = exp(b_m),
-// E = exp(b_C - b_m) (per key dimension):
-//
-//     A  = tril(Qs Ks^T)                       S' = Diag(Pm) S_in      (state in the mid frame)
-//     Y  = A V + Qs S'                         S_out = Diag(E) (S' + Ks^T V)
-//
-// The factors exp(b_t - b_m) are in-chunk cumulative PRODUCTS of f taken outward from the middle
-// (the linear-space image of the log-space cumulative sum): rows after m multiply by prod f, rows
-// before m divide by it.  Products are floored at 2^-100, so extreme decay inside half a chunk
-// (more than 2^100 across 32 steps) loses accuracy but never produces Inf or NaN.
-// Per chunk the state accumulator in TMEM is rescaled once, by E(previous chunk) * Pm(this chunk).
-//
-// Tensor-memory plan (512 columns): S' at columns [0,128) (lane = key dim, column = value dim),
-// Y at [128,256) and A at [256,320) in the M = 64 accumulator layout (row r -> lane 32*(r/16) + r%16).
-#include "tc_common.cuh"
+// Chunkwise HGRN2 backward on the Blackwell tensor cores (tcgen05 + TMEM + TMA), bf16 I/O, fp32
+// state gradient, d_k = d_v = 128, chunk length C = 64 (frame and formulas: tc_chunk.cuh).
+#include "tc_chunk.cuh"
 
 namespace hgrn2 {
 
@@ -29,16 +8,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kC = 64;
-constexpr int kD = 128;
 constexpr int kWorkers = 256;                   // warps 0..7: transforms, TMEM epilogues, outputs
 constexpr int kThreads = kWorkers + 32;         // warp 8: TMA loads and tcgen05.mma issue (one lane)
-constexpr uint32_t kSlab = kC * 128;            // bytes of one slab of a [64][128] tile
-constexpr uint32_t kTile = 2 * kSlab;           // one [64][128] bf16 tile
-constexpr uint32_t kStateSlab = kD * 128;       // bytes of one slab of the [128][128] state copy
-constexpr uint32_t kStateTile = 2 * kStateSlab;
-constexpr float kProdFloor = 7.888609052210118e-31f;   // 2^-100
-constexpr uint32_t kTmemCols = 512;
 
 // Optional per-phase cycle counters of worker thread 0 of CTA 0 (development aid; compiled out unless
 // HGRN2_PHASE_TIMING is defined).  Totals land in the padding words of the status block.
@@ -53,23 +24,6 @@ constexpr uint32_t kTmemCols = 512;
 #endif
 
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
-__device__ __forceinline__ float rcp_fast(float x)
-{
-    float r;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
-
-__device__ __forceinline__ uint4 pack8(const uint32_t *r)
-{
-    uint4 w;
-    w.x = pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1]));
-    w.y = pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3]));
-    w.z = pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5]));
-    w.w = pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7]));
-    return w;
-}
 
 // In-place rescaling of the raw o and f tiles of one chunk into Qs and Ks (see the file header).
 // Thread layout: 64 column pairs x 4 row quarters; quarter q owns rows 16q..16q+15.  Quarter totals
@@ -141,25 +95,6 @@ __device__ __forceinline__ void transform_chunk(uint8_t *qbuf, uint8_t *fbuf, fl
     }
 }
 
-// Causal mask + bf16 of one 64 x 64 fp32 accumulator (M = 64 layout) into a K-major slab.
-__device__ __forceinline__ void tril_to_slab(uint32_t taddr, uint8_t *dstbuf, int sub, int half, int lane)
-{
-    uint32_t r[32];
-    tmem_ld32(taddr, r);
-    tmem_wait_ld();
-    if (lane < 16) {
-        const int t = 16 * sub + lane;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int s0 = 32 * half + 8 * j;
-            uint32_t x[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? r[8 * j + q] : 0u;
-            *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = pack8(x);
-        }
-    }
-}
-
 // One 64 x 128 fp32 accumulator (M = 64 layout) to a bf16 [token][128] global tensor.
 __device__ __forceinline__ void rows_to_global(uint32_t taddr_half, __nv_bfloat16 *dst_row0, int sub, int half,
                                                int lane, int n_valid)
@@ -176,251 +111,6 @@ __device__ __forceinline__ void rows_to_global(uint32_t taddr_half, __nv_bfloat1
             for (int j = 0; j < 4; ++j) dst[j] = pack8(r + 8 * j);
         }
     }
-}
-
-// ---- forward ----------------------------------------------------------------------------------------
-// Skewed software pipeline.  The issuer lane keeps the tensor cores and TMA busy; the 256 workers run
-//   transform(c+1) | A epilogue(c) | state maintenance(c+1) | Y epilogue(c)
-// per iteration, so the MMAs of chunk c overlap the transform of chunk c+1, and the second product
-// Y += P V overlaps the maintenance.  Y is double-buffered in TMEM.
-constexpr int kFwdStages = 3;
-constexpr uint32_t kFwdStageBytes = 3 * kTile;                        // q, f, v
-constexpr uint32_t kFwdOffS = kFwdStages * kFwdStageBytes;            // bf16 copy of S'
-constexpr uint32_t kFwdOffP = kFwdOffS + kStateTile;                  // bf16 tril(A), one slab
-constexpr uint32_t kFwdOffTot = kFwdOffP + kSlab;                     // float tot[4][128]
-constexpr uint32_t kFwdOffPm = kFwdOffTot + 4 * 128 * 4;              // float pm[128]
-constexpr uint32_t kFwdOffE = kFwdOffPm + 128 * 4;                    // float ee[128]
-constexpr uint32_t kFwdOffBar = kFwdOffE + 128 * 4;                   // mbarriers etc.
-constexpr uint32_t kFwdSmemBytes = kFwdOffBar + 256 + 1024;           // + alignment slack
-
-constexpr uint32_t kColS = 0, kColY = 128 /* two buffers of 128 */, kColA = 384;
-
-struct FwdCtl {
-    uint64_t full[kFwdStages];     // TMA -> workers
-    uint64_t xs_ready;             // workers -> issuer: Qs, Ks, S' (TMEM + bf16 copy) of a chunk are in place
-    uint64_t p_ready;              // workers -> issuer: tril(A) is in shared memory
-    uint64_t barA, barS, barY[2];  // tcgen05.commit -> workers
-    uint32_t tmem_base;
-    int abort_flag;
-};
-
-__global__ void __launch_bounds__(kThreads, 1)
-tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
-              const __grid_constant__ CUtensorMap map_i, const float *__restrict__ S0,
-              __nv_bfloat16 *__restrict__ y, float *__restrict__ SN, __nv_bfloat16 *__restrict__ saved, int N,
-              int NC, StatusBlock *status)
-{
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *sbuf = smem + kFwdOffS;
-    uint8_t *pbuf = smem + kFwdOffP;
-    float *tot = reinterpret_cast<float *>(smem + kFwdOffTot);
-    float *pm = reinterpret_cast<float *>(smem + kFwdOffPm);
-    float *ee = reinterpret_cast<float *>(smem + kFwdOffE);
-    FwdCtl *ctl = reinterpret_cast<FwdCtl *>(smem + kFwdOffBar);
-    volatile int *abort_flag = &ctl->abort_flag;
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int u = blockIdx.x;
-
-    if (tid == 0) {
-        for (int s = 0; s < kFwdStages; ++s) mbar_init(&ctl->full[s], 1);
-        mbar_init(&ctl->xs_ready, kWorkers);
-        mbar_init(&ctl->p_ready, kWorkers);
-        mbar_init(&ctl->barA, 1);
-        mbar_init(&ctl->barS, 1);
-        mbar_init(&ctl->barY[0], 1);
-        mbar_init(&ctl->barY[1], 1);
-        ctl->abort_flag = 0;
-        fence_barrier_init();
-        tma_prefetch_desc(&map_o);
-        tma_prefetch_desc(&map_f);
-        tma_prefetch_desc(&map_i);
-    }
-    if (warp == 0) tmem_alloc(&ctl->tmem_base, kTmemCols);
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem = ctl->tmem_base;
-
-    if (warp == 8) {
-        // ================= issuer: TMA loads and MMA issue =================
-        if (lane == 0) {
-            constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
-            constexpr uint32_t idescY = idesc_bf16(64, 128, 0, 1);     // Qs or P (K-major) x S' or V (MN-major)
-            constexpr uint32_t idescS = idesc_bf16(128, 128, 1, 1);    // Ks^T (MN-major) x V (MN-major)
-            auto issue_loads = [&](int c) {
-                const int s = c % kFwdStages;
-                uint8_t *st = smem + s * kFwdStageBytes;
-                mbar_arrive_expect_tx(&ctl->full[s], kFwdStageBytes);
-                for (int b = 0; b < 2; ++b) {
-                    tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
-                }
-            };
-            for (int c = 0; c < kFwdStages && c < NC; ++c) issue_loads(c);
-            const uint32_t sa = smem_u32(sbuf), pa = smem_u32(pbuf);
-            for (int c = 0; c < NC; ++c) {
-                const uint32_t qa = smem_u32(smem + (c % kFwdStages) * kFwdStageBytes);
-                const uint32_t fa = qa + kTile, va = qa + 2 * kTile;
-                const uint32_t ty = tmem + kColY + 128 * (c & 1);
-                mbar_wait(&ctl->xs_ready, c & 1, abort_flag);
-                tc_fence_after_sync();
-                if (y) {
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {        // A = Qs Ks^T
-                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                        mma_bf16_ss(tmem + kColA, smem_desc_sw128(qa + koff, 16, 1024),
-                                    smem_desc_sw128(fa + koff, 16, 1024), idescA, kk > 0);
-                    }
-                    mma_commit(&ctl->barA);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {        // Y = Qs S'
-                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                        mma_bf16_ss(ty, smem_desc_sw128(qa + koff, 16, 1024),
-                                    smem_desc_sw128(sa + kk * 2048, kStateSlab, 1024), idescY, kk > 0);
-                    }
-                }
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)              // S' += Ks^T V
-                    mma_bf16_ss(tmem + kColS, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
-                                smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescS, 1);
-                mma_commit(&ctl->barS);
-                if (y) {
-                    mbar_wait(&ctl->p_ready, c & 1, abort_flag);
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)          // Y += P V
-                        mma_bf16_ss(ty, smem_desc_sw128(pa + kk * 32, 16, 1024),
-                                    smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescY, 1);
-                }
-                mma_commit(&ctl->barY[c & 1]);
-                // the stage of chunk c-1 is free once its MMAs are complete: refill it with chunk c+2
-                if (c >= 1 && c + kFwdStages - 1 < NC) {
-                    mbar_wait(&ctl->barY[(c - 1) & 1], ((c - 1) >> 1) & 1, abort_flag);
-                    issue_loads(c + kFwdStages - 1);
-                }
-            }
-        }
-    } else {
-        // ================= workers =================
-        const int sub = warp & 3, half = warp >> 2;      // TMEM sub-partition and column half of this warp
-        const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
-        const int krow = 32 * sub + lane;
-        float e_prev = 1.f;
-
-        // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk); bf16 copy for the MMAs
-        // and for the backward pass; then hand the chunk to the issuer.
-        auto maintain = [&](int c, bool first) {
-            const float factor = e_prev * pm[krow];
-            e_prev = ee[krow];
-            uint32_t r[32];
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                const int v0 = 64 * half + 32 * part;
-                if (first) {
-                    if (S0) {
-                        const float4 *src = reinterpret_cast<const float4 *>(S0 + ((size_t)u * kD + krow) * kD + v0);
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 x = __ldg(src + j);
-                            r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
-                            r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) r[j] = 0u;
-                    }
-                } else {
-                    tmem_ld32(tmem + lane_base + kColS + v0, r);
-                    tmem_wait_ld();
-                }
-#pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
-                tmem_st32(tmem + lane_base + kColS + v0, r);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 w = pack8(r + 8 * j);
-                    *reinterpret_cast<uint4 *>(sbuf + half * kStateSlab + slab_chunk_off(krow, 4 * part + j)) = w;
-                    if (saved)
-                        *reinterpret_cast<uint4 *>(saved + (((size_t)u * NC + c) * kD + krow) * kD + v0 + 8 * j) = w;
-                }
-            }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            fence_proxy_async_smem();
-            mbar_arrive(&ctl->xs_ready);
-        };
-
-        mbar_wait(&ctl->full[0], 0, abort_flag);
-        transform_chunk(smem, smem + kTile, tot, pm, ee, min(kC, N), tid);
-        worker_sync();
-        maintain(0, true);
-        PT_DECL
-
-        for (int c = 0; c < NC; ++c) {
-            const int n_valid = min(kC, N - c * kC);
-            if (c + 1 < NC) {
-                const int s1 = (c + 1) % kFwdStages;
-                uint8_t *qbuf = smem + s1 * kFwdStageBytes;
-                mbar_wait(&ctl->full[s1], ((c + 1) / kFwdStages) & 1, abort_flag);
-                PT_MARK(0)
-                transform_chunk(qbuf, qbuf + kTile, tot, pm, ee, min(kC, N - (c + 1) * kC), tid);
-                worker_sync();
-                PT_MARK(1)
-            }
-            if (y) {
-                mbar_wait(&ctl->barA, c & 1, abort_flag);
-                tc_fence_after_sync();
-                PT_MARK(2)
-                tril_to_slab(tmem + lane_base + kColA + 32 * half, pbuf, sub, half, lane);
-                fence_proxy_async_smem();
-                tc_fence_before_sync();
-                mbar_arrive(&ctl->p_ready);
-                PT_MARK(3)
-            }
-            if (c + 1 < NC) {
-                mbar_wait(&ctl->barS, c & 1, abort_flag);
-                tc_fence_after_sync();
-                PT_MARK(4)
-                maintain(c + 1, false);
-                PT_MARK(5)
-            }
-            if (y) {
-                mbar_wait(&ctl->barY[c & 1], (c >> 1) & 1, abort_flag);
-                tc_fence_after_sync();
-                PT_MARK(6)
-                rows_to_global(tmem + lane_base + kColY + 128 * (c & 1) + 64 * half,
-                               y + ((size_t)u * N + (size_t)c * kC) * kD, sub, half, lane, n_valid);
-                tc_fence_before_sync();
-                PT_MARK(7)
-            }
-        }
-        PT_DUMP(status)
-
-        // S_N = Diag(E_last) S''
-        mbar_wait(&ctl->barS, (NC - 1) & 1, abort_flag);
-        tc_fence_after_sync();
-        if (SN) {
-            uint32_t r[32];
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                const int v0 = 64 * half + 32 * part;
-                tmem_ld32(tmem + lane_base + kColS + v0, r);
-                tmem_wait_ld();
-                float4 *dst = reinterpret_cast<float4 *>(SN + ((size_t)u * kD + krow) * kD + v0);
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * e_prev, __uint_as_float(r[4 * j + 1]) * e_prev,
-                                         __uint_as_float(r[4 * j + 2]) * e_prev, __uint_as_float(r[4 * j + 3]) * e_prev);
-            }
-        }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (tid == 0 && *abort_flag) report_error(status, HGRN2_ERR_TIMEOUT, 1);
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ---- backward ---------------------------------------------------------------------------------------
@@ -835,67 +525,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
-// ---- host side ------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// [U][rows][128] bf16 tensor, tiles of [box_rows][64] with the 128-byte swizzle; rows beyond `rows`
-// read as zero.
-bool make_map(CUtensorMap *m, const void *base, uint64_t U, uint64_t rows, uint32_t box_rows)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {128, rows, U};
-    cuuint64_t strides[2] = {256, rows * 256};
-    cuuint32_t box[3] = {64, box_rows, 1};
-    cuuint32_t es[3] = {1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
-
-bool tc_supported(const hgrn2_desc *d)
-{
-    return d->io == HGRN2_BF16 && d->dk == kD && d->dv == kD;
-}
-int  tc_default_chunk() { return kC; }
-bool tc_chunk_supported(int C) { return C == kC; }
-
-size_t tc_saved_bytes(const hgrn2_desc *d, int C)
-{
-    const size_t NC = ((size_t)d->N + C - 1) / C;
-    return (size_t)d->B * d->H * NC * kD * kD * sizeof(__nv_bfloat16);
-}
-
-cudaError_t launch_tc_fwd(const SeqArgs &a)
-{
-    const uint64_t U = (uint64_t)a.B * a.H;
-    CUtensorMap mo, mf, mi;
-    if (!make_map(&mo, a.o, U, a.N, kC) || !make_map(&mf, a.f, U, a.N, kC) || !make_map(&mi, a.i, U, a.N, kC))
-        return cudaErrorInvalidValue;
-    cudaError_t err = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmemBytes);
-    if (err != cudaSuccess) return err;
-    tc_fwd_kernel<<<(unsigned)U, kThreads, kFwdSmemBytes, a.stream>>>(
-        mo, mf, mi, a.S0, static_cast<__nv_bfloat16 *>(a.y), a.SN, reinterpret_cast<__nv_bfloat16 *>(a.states), a.N,
-        a.NC, a.status);
-    return cudaGetLastError();
-}
 
 cudaError_t launch_tc_bwd(const SeqArgs &a)
 {

@@ -1,0 +1,363 @@
+// Chunkwise HGRN2 forward on the Blackwell tensor cores (tcgen05 + TMEM + TMA), bf16 I/O, fp32
+// state, d_k = d_v = 128, chunk length C = 64.  One CTA per (batch, head) unit walks the chunks in
+// order with the running state resident in tensor memory (frame and formulas: tc_chunk.cuh).
+//
+// Warp roles (15 warps, none of them ever waits on a CTA-wide barrier inside the chunk loop):
+//   warps 0..3   transform: raw o, f tiles -> Qs, Ks in place, running ahead of the rest by up to
+//                two chunks (three TMA stages);
+//   warps 4..11  epilogues: rescale the state accumulator once per chunk and publish its bf16 copy
+//                S' (the critical chain), causal mask of A into an operand slab, Y into a staging tile;
+//   warp 12      TMA loads of o, f, i;
+//   warp 13      tcgen05.mma issue, and the TMA store of S' (the saved chunk state) straight from
+//                the operand copy;
+//   warp 14      TMA stores of the Y tiles.
+// Hand-offs are mbarriers; every wait is bounded (tc_common.cuh).
+//
+// Tensor-memory plan (512 columns): S' at [0,128) (lane = key dim, column = value dim); Y, double
+// buffered, at [128,384) and A, double buffered, at [384,512) in the M = 64 accumulator layout
+// (row r -> lane 32 * (r / 16) + r % 16).
+#include "tc_chunk.cuh"
+
+namespace hgrn2 {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kTWarps = 4, kEWarps = 8;
+constexpr int kEThreads = kEWarps * 32;
+constexpr int kWarpLoad = kTWarps + kEWarps, kWarpMma = kWarpLoad + 1, kWarpStore = kWarpLoad + 2;
+constexpr int kThreads = (kWarpStore + 1) * 32;
+
+constexpr int kStages = 3;
+constexpr uint32_t kStageBytes = 3 * kTile;                       // q, f, v
+constexpr uint32_t kOffS = kStages * kStageBytes;                 // bf16 copy of S'
+constexpr uint32_t kOffP = kOffS + kStateTile;                    // bf16 tril(A): two slabs (double buffer)
+constexpr uint32_t kOffY = kOffP + 2 * kSlab;                     // Y staging tile for the TMA store
+constexpr uint32_t kOffPm = kOffY + kTile;                        // float pm[4][128]
+constexpr uint32_t kOffE = kOffPm + 4 * 128 * 4;                  // float ee[4][128]
+constexpr uint32_t kOffCtl = kOffE + 4 * 128 * 4;
+constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024;             // + alignment slack
+
+constexpr uint32_t kColS = 0, kColY = 128, kColA = 384;
+
+struct Ctl {
+    uint64_t full[kStages];      // TMA -> transform warps, MMA warp
+    uint64_t empty[kStages];     // tcgen05.commit -> TMA warp: every MMA reading the stage has completed
+    uint64_t t_done[kStages];    // transform warps -> MMA warp, epilogue warps (Pm, E of the chunk)
+    uint64_t m_done;             // epilogue warps -> MMA warp: S' of the chunk is in TMEM and shared memory
+    uint64_t barA[2];            // tcgen05.commit -> epilogue warps: A is complete
+    uint64_t p_ready[2];         // epilogue warps -> MMA warp: tril(A) is in shared memory
+    uint64_t barS;               // tcgen05.commit -> epilogue warps: state update complete, S' copy reusable
+    uint64_t barY[2];            // tcgen05.commit -> epilogue warps: Y is complete
+    uint64_t y_tfree[2];         // epilogue warps -> MMA warp: the Y accumulator has been read out
+    uint64_t y_staged;           // epilogue warps -> store warp
+    uint64_t y_sfree;            // store warp -> epilogue warps: the staging tile may be overwritten
+    uint32_t tmem_base;
+    int abort_flag;
+};
+static_assert(sizeof(Ctl) <= 256, "control block");
+static_assert(kSmemBytes <= 232448, "shared memory budget");
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
+              const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
+              const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
+              int want_y, int want_saved, int N, int NC, StatusBlock *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *sbuf = smem + kOffS;
+    uint8_t *pbuf = smem + kOffP;
+    uint8_t *ybuf = smem + kOffY;
+    float *pm = reinterpret_cast<float *>(smem + kOffPm);
+    float *ee = reinterpret_cast<float *>(smem + kOffE);
+    Ctl *ctl = reinterpret_cast<Ctl *>(smem + kOffCtl);
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int u = blockIdx.x;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], 1);
+            mbar_init(&ctl->t_done[s], kTransformThreads);
+        }
+        mbar_init(&ctl->m_done, kEThreads);
+        mbar_init(&ctl->barS, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&ctl->barA[b], 1);
+            mbar_init(&ctl->p_ready[b], kEThreads);
+            mbar_init(&ctl->barY[b], 1);
+            mbar_init(&ctl->y_tfree[b], kEThreads);
+        }
+        mbar_init(&ctl->y_staged, kEThreads);
+        mbar_init(&ctl->y_sfree, 1);
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&map_o);
+        tma_prefetch_desc(&map_f);
+        tma_prefetch_desc(&map_i);
+        tma_prefetch_desc(&map_y);
+        tma_prefetch_desc(&map_saved);
+    }
+    if (warp == 0) tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp < kTWarps) {
+        // ================= transform warps =================
+        for (int c = 0; c < NC; ++c) {
+            const int s = c % kStages;
+            uint8_t *qbuf = smem + s * kStageBytes;
+            mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
+            const int n_valid = N - c * kC;
+            if (n_valid >= kC)
+                transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, kC, tid);
+            else
+                transform_stream<false>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, n_valid, tid);
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->t_done[s]);
+        }
+    } else if (warp < kWarpLoad) {
+        // ================= epilogue warps =================
+        const int sub = warp & 3, half = (warp - kTWarps) >> 2;   // TMEM lane quarter, column half
+        const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
+        const int krow = 32 * sub + lane;
+        float e_prev = 1.f;
+
+        // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk) back into TMEM, and
+        // its bf16 copy for the MMAs and for the saved-state store; then hand the chunk to the MMA warp.
+        auto maintain = [&](int c) {
+            mbar_wait(&ctl->t_done[c % kStages], (c / kStages) & 1, abort_flag);
+            const float factor = e_prev * pm[(c & 3) * 128 + krow];
+            e_prev = ee[(c & 3) * 128 + krow];
+            const int v0 = 64 * half;
+            uint32_t r[64];
+            if (c == 0) {
+                if (S0) {
+                    const float4 *src = reinterpret_cast<const float4 *>(S0 + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float4 x = __ldg(src + j);
+                        r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
+                        r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) r[j] = 0u;
+                }
+            } else {
+                mbar_wait(&ctl->barS, (c - 1) & 1, abort_flag);
+                tc_fence_after_sync();
+                tmem_ld32(tmem + lane_base + kColS + v0, *reinterpret_cast<uint32_t(*)[32]>(r));
+                tmem_ld32(tmem + lane_base + kColS + v0 + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
+                tmem_wait_ld();
+            }
+#pragma unroll
+            for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
+            tmem_st32(tmem + lane_base + kColS + v0, *reinterpret_cast<uint32_t(*)[32]>(r));
+            tmem_st32(tmem + lane_base + kColS + v0 + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4 *>(sbuf + half * kStateSlab + slab_chunk_off(krow, j)) = pack8(r + 8 * j);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->m_done);
+        };
+
+        // Y of chunk c: accumulator -> bf16 staging tile -> (store warp) TMA store.
+        auto y_out = [&](int c) {
+            const int b = c & 1;
+            uint32_t r[64];
+            mbar_wait(&ctl->barY[b], (c >> 1) & 1, abort_flag);
+            tc_fence_after_sync();
+            const uint32_t ta = tmem + lane_base + kColY + 128 * b + 64 * half;
+            tmem_ld32(ta, *reinterpret_cast<uint32_t(*)[32]>(r));
+            tmem_ld32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->y_tfree[b]);
+            if (c >= 1) mbar_wait(&ctl->y_sfree, (c - 1) & 1, abort_flag);
+            if (lane < 16) {
+                const int t = 16 * sub + lane;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    *reinterpret_cast<uint4 *>(ybuf + half * kSlab + slab_chunk_off(t, j)) = pack8(r + 8 * j);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->y_staged);
+        };
+
+        for (int c = 0; c <= NC; ++c) {
+            if (c < NC) maintain(c);
+            if (want_y && c >= 1) y_out(c - 1);
+            if (want_y && c < NC) {
+                mbar_wait(&ctl->barA[c & 1], (c >> 1) & 1, abort_flag);
+                tc_fence_after_sync();
+                tril_to_slab(tmem + lane_base + kColA + 64 * (c & 1) + 32 * half, pbuf + (c & 1) * kSlab, sub, half, lane);
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                mbar_arrive(&ctl->p_ready[c & 1]);
+            }
+        }
+
+        // S_N = Diag(E_last) S''
+        mbar_wait(&ctl->barS, (NC - 1) & 1, abort_flag);
+        tc_fence_after_sync();
+        if (SN) {
+            uint32_t r[32];
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                const int v0 = 64 * half + 32 * part;
+                tmem_ld32(tmem + lane_base + kColS + v0, r);
+                tmem_wait_ld();
+                float4 *dst = reinterpret_cast<float4 *>(SN + ((size_t)u * kD + krow) * kD + v0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * e_prev, __uint_as_float(r[4 * j + 1]) * e_prev,
+                                         __uint_as_float(r[4 * j + 2]) * e_prev, __uint_as_float(r[4 * j + 3]) * e_prev);
+            }
+        }
+    } else if (warp == kWarpLoad) {
+        // ================= TMA loads =================
+        if (lane == 0) {
+            for (int c = 0; c < NC; ++c) {
+                const int s = c % kStages;
+                if (c >= kStages) mbar_wait(&ctl->empty[s], ((c / kStages) - 1) & 1, abort_flag);
+                uint8_t *st = smem + s * kStageBytes;
+                mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
+                }
+            }
+        }
+    } else if (warp == kWarpMma) {
+        // ================= MMA issue (+ saved-state stores) =================
+        if (lane == 0) {
+            constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
+            constexpr uint32_t idescY = idesc_bf16(64, 128, 0, 1);     // Qs or P (K-major) x S' or V (MN-major)
+            constexpr uint32_t idescS = idesc_bf16(128, 128, 1, 1);    // Ks^T (MN-major) x V (MN-major)
+            const uint32_t sa = smem_u32(sbuf);
+            for (int c = 0; c < NC; ++c) {
+                const int s = c % kStages, b = c & 1;
+                const uint32_t qa = smem_u32(smem + s * kStageBytes);
+                const uint32_t fa = qa + kTile, va = qa + 2 * kTile;
+                const uint32_t pa = smem_u32(pbuf + b * kSlab);
+                const uint32_t ty = tmem + kColY + 128 * b, ta = tmem + kColA + 64 * b;
+                mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
+                mbar_wait(&ctl->t_done[s], (c / kStages) & 1, abort_flag);
+                mbar_wait(&ctl->m_done, c & 1, abort_flag);
+                tc_fence_after_sync();
+                if (want_saved) {
+                    tma_store_3d(&map_saved, sbuf, 0, 0, u * NC + c);
+                    tma_store_3d(&map_saved, sbuf + kStateSlab, 64, 0, u * NC + c);
+                    tma_store_commit();
+                }
+                if (want_y) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {        // A = Qs Ks^T
+                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                        mma_bf16_ss(ta, smem_desc_sw128(qa + koff, 16, 1024), smem_desc_sw128(fa + koff, 16, 1024),
+                                    idescA, kk > 0);
+                    }
+                    mma_commit(&ctl->barA[b]);
+                    if (c >= 2) {
+                        mbar_wait(&ctl->y_tfree[b], ((c - 2) >> 1) & 1, abort_flag);
+                        tc_fence_after_sync();
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {        // Y = Qs S'
+                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
+                        mma_bf16_ss(ty, smem_desc_sw128(qa + koff, 16, 1024),
+                                    smem_desc_sw128(sa + kk * 2048, kStateSlab, 1024), idescY, kk > 0);
+                    }
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // S' += Ks^T V
+                    mma_bf16_ss(tmem + kColS, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
+                                smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescS, 1);
+                if (want_saved) tma_store_wait_read();      // the S' copy is rewritten once barS fires
+                mma_commit(&ctl->barS);
+                if (want_y) {
+                    mbar_wait(&ctl->p_ready[b], (c >> 1) & 1, abort_flag);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)          // Y += P V
+                        mma_bf16_ss(ty, smem_desc_sw128(pa + kk * 32, 16, 1024),
+                                    smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescY, 1);
+                    mma_commit(&ctl->barY[b]);
+                }
+                mma_commit(&ctl->empty[s]);
+            }
+            if (want_saved) tma_store_wait_all();
+        }
+    } else {
+        // ================= Y stores =================
+        if (lane == 0 && want_y) {
+            for (int c = 0; c < NC; ++c) {
+                mbar_wait(&ctl->y_staged, c & 1, abort_flag);
+                tma_store_3d(&map_y, ybuf, 0, c * kC, u);
+                tma_store_3d(&map_y, ybuf + kSlab, 64, c * kC, u);
+                tma_store_commit();
+                tma_store_wait_read();
+                mbar_arrive(&ctl->y_sfree);
+            }
+            tma_store_wait_all();
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && *abort_flag) {
+        report_error(status, HGRN2_ERR_TIMEOUT, 1);
+        // a load may still be in flight towards this CTA's shared memory: give it time to land
+        for (int s = 0; s < kStages; ++s) {
+            const int last = ((NC - 1 - s) / kStages) * kStages + s;     // last chunk that used stage s
+            if (last >= 0 && s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
+        }
+    }
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace
+
+bool tc_supported(const hgrn2_desc *d)
+{
+    return d->io == HGRN2_BF16 && d->dk == kD && d->dv == kD;
+}
+int  tc_default_chunk() { return kC; }
+bool tc_chunk_supported(int C) { return C == kC; }
+
+size_t tc_saved_bytes(const hgrn2_desc *d, int C)
+{
+    const size_t NC = ((size_t)d->N + C - 1) / C;
+    return (size_t)d->B * d->H * NC * kD * kD * sizeof(__nv_bfloat16);
+}
+
+cudaError_t launch_tc_fwd(const SeqArgs &a)
+{
+    const uint64_t U = (uint64_t)a.B * a.H;
+    CUtensorMap mo, mf, mi, my, ms;
+    // tensor maps need a valid base even for outputs that are not wanted: point those at an input
+    const void *ybase = a.y ? a.y : a.i;
+    const void *sbase = a.states ? static_cast<const void *>(a.states) : a.i;
+    const uint64_t srows = a.states ? (uint64_t)kD : (uint64_t)a.N;
+    const uint64_t sunits = a.states ? U * a.NC : U;
+    if (!make_map(&mo, a.o, U, a.N, kC) || !make_map(&mf, a.f, U, a.N, kC) || !make_map(&mi, a.i, U, a.N, kC) ||
+        !make_map(&my, ybase, U, a.N, kC) || !make_map(&ms, sbase, sunits, srows, a.states ? kD : kC))
+        return cudaErrorInvalidValue;
+    cudaError_t err = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (err != cudaSuccess) return err;
+    tc_fwd_kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, a.S0, a.SN, a.y != nullptr,
+                                                                   a.states != nullptr, a.N, a.NC, a.status);
+    return cudaGetLastError();
+}
+
+}  // namespace hgrn2

@@ -1,0 +1,159 @@
+// Pieces shared by the tensor-core forward and backward kernels: tile geometry, the in-place
+// operand transform of one chunk, accumulator-to-operand conversions and the TMA tensor maps.
+//
+// Mid-chunk reference frame.  Within a chunk of C = 64 steps let b_j = sum_{r<=j} log f_r (per key
+// dimension) and let m be the middle of the chunk (after local row 31).  Only two rescaled operands
+// are formed:
+//
+//     Qs_t = q_t * exp(b_t - b_m)          Ks_s = k_s * exp(b_m - b_s)          (q = o, k = 1 - f)
+//
+// so that Qs_t . Ks_s = q_t k_s exp(b_t - b_s) for every pair, and with Pm = exp(b_m),
+// E = exp(b_C - b_m) (per key dimension):
+//
+//     A  = tril(Qs Ks^T)                       S' = Diag(Pm) S_in      (state in the mid frame)
+//     Y  = A V + Qs S'                         S_out = Diag(E) (S' + Ks^T V)
+//
+// The factors exp(b_t - b_m) are in-chunk cumulative PRODUCTS of f taken outward from the middle
+// (the linear-space image of the log-space cumulative sum): rows after m multiply by prod f, rows
+// before m divide by it.  Products are floored at 2^-100, so extreme decay inside half a chunk
+// (more than 2^100 across 32 steps) loses accuracy but never produces Inf or NaN.
+#pragma once
+
+#include "tc_common.cuh"
+
+namespace hgrn2 {
+namespace tc {
+
+constexpr int kC = 64;                          // chunk length
+constexpr int kD = 128;                         // d_k = d_v
+constexpr uint32_t kSlab = kC * 128;            // bytes of one slab of a [64][128] bf16 tile
+constexpr uint32_t kTile = 2 * kSlab;           // one [64][128] bf16 tile
+constexpr uint32_t kStateSlab = kD * 128;       // bytes of one slab of a [128][128] bf16 state copy
+constexpr uint32_t kStateTile = 2 * kStateSlab;
+constexpr float kProdFloor = 7.888609052210118e-31f;   // 2^-100
+constexpr uint32_t kTmemCols = 512;
+constexpr int kTransformThreads = 128;          // threads that run transform_stream together
+
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+__device__ __forceinline__ uint4 pack8(const uint32_t *r)
+{
+    uint4 w;
+    w.x = pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1]));
+    w.y = pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3]));
+    w.z = pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5]));
+    w.w = pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7]));
+    return w;
+}
+
+// In-place rescaling of the raw o and f tiles of one chunk into Qs and Ks (see the file header).
+// Run by 128 threads with no synchronisation among them: thread = one column pair x one half of the
+// chunk.  The half before the middle walks its rows downwards from row 31, the half after it walks
+// upwards from row 32, each carrying the running product of f, so nothing but the current row is
+// live.  Pm (product over rows 0..31) and E (product over rows 32..63) of the chunk are left in
+// pm[128] and ee[128].  Rows at or beyond n_valid are the neutral token f = 1, o = 0.
+template <bool kFull>
+__device__ __forceinline__ void transform_stream(uint8_t *qbuf, uint8_t *fbuf, float *pm, float *ee, int n_valid,
+                                                 int tid)
+{
+    const int h = tid >> 6, p = tid & 63;
+    const int col = 2 * p;
+    const int jch = (col & 63) >> 3;
+    const uint32_t base = (col >> 6) * kSlab + (col & 7) * 2;
+    uint32_t xo[8];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) xo[jj] = base + ((jch ^ jj) << 4);
+    float a0 = 1.f, a1 = 1.f;
+    if (h == 1) {
+#pragma unroll
+        for (int r = 32; r < 64; ++r) {
+            const uint32_t off = xo[r & 7] + r * 128;
+            uint32_t fw = *reinterpret_cast<const uint32_t *>(fbuf + off);
+            uint32_t qw = *reinterpret_cast<const uint32_t *>(qbuf + off);
+            if (!kFull && r >= n_valid) { fw = 0x3F803F80u; qw = 0u; }
+            const float f0 = bf16_lo(fw), f1 = bf16_hi(fw);
+            a0 *= f0; a1 *= f1;
+            const float m0 = fmaxf(a0, kProdFloor), m1 = fmaxf(a1, kProdFloor);
+            const float i0 = rcp_fast(m0), i1 = rcp_fast(m1);
+            *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(bf16_lo(qw) * m0, bf16_hi(qw) * m1);
+            *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0) * i0, (1.f - f1) * i1);
+        }
+        *reinterpret_cast<float2 *>(ee + col) = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
+    } else {
+#pragma unroll
+        for (int r = 31; r >= 0; --r) {
+            const uint32_t off = xo[r & 7] + r * 128;
+            uint32_t fw = *reinterpret_cast<const uint32_t *>(fbuf + off);
+            uint32_t qw = *reinterpret_cast<const uint32_t *>(qbuf + off);
+            if (!kFull && r >= n_valid) { fw = 0x3F803F80u; qw = 0u; }
+            const float f0 = bf16_lo(fw), f1 = bf16_hi(fw);
+            const float m0 = fmaxf(a0, kProdFloor), m1 = fmaxf(a1, kProdFloor);
+            const float i0 = rcp_fast(m0), i1 = rcp_fast(m1);
+            *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(bf16_lo(qw) * i0, bf16_hi(qw) * i1);
+            *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0) * m0, (1.f - f1) * m1);
+            a0 *= f0; a1 *= f1;
+        }
+        *reinterpret_cast<float2 *>(pm + col) = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
+    }
+}
+
+// Causal mask + bf16 of 32 columns (32 * half ...) of one 64 x 64 fp32 accumulator in the M = 64
+// layout (row r -> lane 32 * (r / 16) + r % 16) into a K-major slab.  `sub` = TMEM lane quarter.
+__device__ __forceinline__ void tril_to_slab(uint32_t taddr, uint8_t *dstbuf, int sub, int half, int lane)
+{
+    uint32_t r[32];
+    tmem_ld32(taddr, r);
+    tmem_wait_ld();
+    if (lane < 16) {
+        const int t = 16 * sub + lane;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int s0 = 32 * half + 8 * j;
+            uint32_t x[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? r[8 * j + q] : 0u;
+            *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = pack8(x);
+        }
+    }
+}
+
+// ---- host side: tensor maps ---------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [U][rows][128] bf16 tensor, tiles of [box_rows][64] with the 128-byte swizzle; rows beyond `rows`
+// read as zero and are dropped on stores.
+inline bool make_map(CUtensorMap *m, const void *base, uint64_t U, uint64_t rows, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {128, rows, U};
+    cuuint64_t strides[2] = {256, rows * 256};
+    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace tc
+}  // namespace hgrn2
