@@ -11,18 +11,6 @@ using namespace tc;
 constexpr int kWorkers = 256;                   // warps 0..7: transforms, TMEM epilogues, outputs
 constexpr int kThreads = kWorkers + 32;         // warp 8: TMA loads and tcgen05.mma issue (one lane)
 
-// Optional per-phase cycle counters of worker thread 0 of CTA 0 (development aid; compiled out unless
-// HGRN2_PHASE_TIMING is defined).  Totals land in the padding words of the status block.
-#ifdef HGRN2_PHASE_TIMING
-#define PT_DECL long long pt_t0 = clock64(); long long pt_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-#define PT_MARK(i) { const long long pt_t = clock64(); pt_acc[i] += pt_t - pt_t0; pt_t0 = pt_t; }
-#define PT_DUMP(st) if (tid == 0 && blockIdx.x == 0 && (st) != nullptr) { for (int pt_i = 0; pt_i < 12; ++pt_i) (st)->pad[pt_i] = (int)pt_acc[pt_i]; }
-#else
-#define PT_DECL
-#define PT_MARK(i)
-#define PT_DUMP(st)
-#endif
-
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // In-place rescaling of the raw o and f tiles of one chunk into Qs and Ks (see the file header).
@@ -500,7 +488,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 PT_MARK(10)
             }
         }
-        PT_DUMP(status)
+        PT_DUMP(status, 0, 12, tid == 0)
 
         // dS_0 = Diag(Pm of chunk 0) dS'
         if (dS0) {

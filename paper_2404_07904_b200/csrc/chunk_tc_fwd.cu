@@ -2,15 +2,19 @@
 // state, d_k = d_v = 128, chunk length C = 64.  One CTA per (batch, head) unit walks the chunks in
 // order with the running state resident in tensor memory (frame and formulas: tc_chunk.cuh).
 //
-// Warp roles (15 warps, none of them ever waits on a CTA-wide barrier inside the chunk loop):
-//   warps 0..3   transform: raw o, f tiles -> Qs, Ks in place, running ahead of the rest by up to
-//                two chunks (three TMA stages);
-//   warps 4..11  epilogues: rescale the state accumulator once per chunk and publish its bf16 copy
-//                S' (the critical chain), causal mask of A into an operand slab, Y into a staging tile;
-//   warp 12      TMA loads of o, f, i;
-//   warp 13      tcgen05.mma issue, and the TMA store of S' (the saved chunk state) straight from
-//                the operand copy;
-//   warp 14      TMA stores of the Y tiles.
+// Warp roles (none of them ever waits on a CTA-wide barrier inside the chunk loop; every stretch of
+// work between two hand-offs is latency-bound, so the roles are many and narrow rather than few and
+// wide, and their loops stay rolled to keep the instruction footprint small):
+//   T   transform warps (4 per group): raw o, f tiles -> Qs, Ks in place, running ahead of the rest
+//       by up to two chunks (three TMA stages);
+//   E1  8 state warps: rescale the accumulator once per chunk (the critical chain) and publish its
+//       bf16 copy S' for Y = Qs S' and for the saved-state store;
+//   E2  4 output warps: causal mask of A into an operand slab, Y into a staging tile;
+//   L   1 warp: TMA loads of o, f, i;
+//   MS  1 warp: tcgen05.mma issue of the state update S' += Ks^T V;
+//   MY  1 warp: tcgen05.mma issue of A = Qs Ks^T, Y = Qs S', Y += tril(A) V, and the TMA store of S'
+//       (the saved chunk state) straight from the operand copy;
+//   ST  1 warp: TMA stores of the Y tiles.
 // Hand-offs are mbarriers; every wait is bounded (tc_common.cuh).
 //
 // Tensor-memory plan (512 columns): S' at [0,128) (lane = key dim, column = value dim); Y, double
@@ -24,10 +28,14 @@ namespace {
 
 using namespace tc;
 
-constexpr int kTWarps = 4, kEWarps = 8;
-constexpr int kEThreads = kEWarps * 32;
-constexpr int kWarpLoad = kTWarps + kEWarps, kWarpMma = kWarpLoad + 1, kWarpStore = kWarpLoad + 2;
+constexpr int kTGroups = 1, kTWarps = 4 * kTGroups;
+constexpr int kE1Warps = 8, kE2Warps = 4;
+constexpr int kE1Threads = kE1Warps * 32, kE2Threads = kE2Warps * 32;
+constexpr int kWarpE1 = kTWarps, kWarpE2 = kWarpE1 + kE1Warps;
+constexpr int kWarpLoad = kWarpE2 + kE2Warps, kWarpMmaS = kWarpLoad + 1, kWarpMmaY = kWarpLoad + 2,
+              kWarpStore = kWarpLoad + 3;
 constexpr int kThreads = (kWarpStore + 1) * 32;
+static_assert(kWarpE1 % 4 == 0 && kWarpE2 % 4 == 0, "epilogue warps must start on a TMEM lane-quarter boundary");
 
 constexpr int kStages = 3;
 constexpr uint32_t kStageBytes = 3 * kTile;                       // q, f, v
@@ -42,17 +50,19 @@ constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024;             // + alignment
 constexpr uint32_t kColS = 0, kColY = 128, kColA = 384;
 
 struct Ctl {
-    uint64_t full[kStages];      // TMA -> transform warps, MMA warp
-    uint64_t empty[kStages];     // tcgen05.commit -> TMA warp: every MMA reading the stage has completed
-    uint64_t t_done[kStages];    // transform warps -> MMA warp, epilogue warps (Pm, E of the chunk)
-    uint64_t m_done;             // epilogue warps -> MMA warp: S' of the chunk is in TMEM and shared memory
-    uint64_t barA[2];            // tcgen05.commit -> epilogue warps: A is complete
-    uint64_t p_ready[2];         // epilogue warps -> MMA warp: tril(A) is in shared memory
-    uint64_t barS;               // tcgen05.commit -> epilogue warps: state update complete, S' copy reusable
-    uint64_t barY[2];            // tcgen05.commit -> epilogue warps: Y is complete
-    uint64_t y_tfree[2];         // epilogue warps -> MMA warp: the Y accumulator has been read out
-    uint64_t y_staged;           // epilogue warps -> store warp
-    uint64_t y_sfree;            // store warp -> epilogue warps: the staging tile may be overwritten
+    uint64_t full[kStages];      // TMA -> T, MS, MY
+    uint64_t empty[kStages];     // tcgen05.commit (MS and MY) -> L: every MMA reading the stage has completed
+    uint64_t t_done[kStages];    // T -> MS, MY, E1 (Pm, E of the chunk)
+    uint64_t m_tmem;             // E1 -> MS: the accumulator holds S' of the chunk
+    uint64_t m_done;             // E1 -> MY: the bf16 copy of S' is in shared memory
+    uint64_t barS;               // tcgen05.commit -> E1: state update complete
+    uint64_t barS2;              // tcgen05.commit -> E1: Y = Qs S' complete and stored, S' copy reusable
+    uint64_t barA[2];            // tcgen05.commit -> E2: A is complete
+    uint64_t p_ready[2];         // E2 -> MY: tril(A) is in shared memory
+    uint64_t barY[2];            // tcgen05.commit -> E2: Y is complete
+    uint64_t y_tfree[2];         // E2 -> MY: the Y accumulator has been read out
+    uint64_t y_staged;           // E2 -> ST
+    uint64_t y_sfree;            // ST -> E2: the staging tile may be overwritten
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -81,18 +91,20 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->empty[s], 1);
+            mbar_init(&ctl->empty[s], 2);
             mbar_init(&ctl->t_done[s], kTransformThreads);
         }
-        mbar_init(&ctl->m_done, kEThreads);
+        mbar_init(&ctl->m_tmem, kE1Threads);
+        mbar_init(&ctl->m_done, kE1Threads);
         mbar_init(&ctl->barS, 1);
+        mbar_init(&ctl->barS2, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&ctl->barA[b], 1);
-            mbar_init(&ctl->p_ready[b], kEThreads);
+            mbar_init(&ctl->p_ready[b], kE2Threads);
             mbar_init(&ctl->barY[b], 1);
-            mbar_init(&ctl->y_tfree[b], kEThreads);
+            mbar_init(&ctl->y_tfree[b], kE2Threads);
         }
-        mbar_init(&ctl->y_staged, kEThreads);
+        mbar_init(&ctl->y_staged, kE2Threads);
         mbar_init(&ctl->y_sfree, 1);
         ctl->abort_flag = 0;
         fence_barrier_init();
@@ -107,35 +119,42 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = ctl->tmem_base;
+    const int sub = warp & 3;                                        // TMEM lane quarter of this warp
+    const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
 
     if (warp < kTWarps) {
-        // ================= transform warps =================
-        for (int c = 0; c < NC; ++c) {
+        // ================= T: transform =================
+        PT_DECL
+        const int tt = tid & (kTransformThreads - 1);
+        for (int c = warp >> 2; c < NC; c += kTGroups) {
             const int s = c % kStages;
             uint8_t *qbuf = smem + s * kStageBytes;
             mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
+            PT_MARK(0)
             const int n_valid = N - c * kC;
-            if (n_valid >= kC)
-                transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, kC, tid);
-            else
-                transform_stream<false>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, n_valid, tid);
+            if (n_valid >= kC) {
+                transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, kC, tt);
+            } else {
+                transform_stream<false>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, n_valid, tt);
+            }
             fence_proxy_async_smem();
             mbar_arrive(&ctl->t_done[s]);
+            PT_MARK(1)
         }
-    } else if (warp < kWarpLoad) {
-        // ================= epilogue warps =================
-        const int sub = warp & 3, half = (warp - kTWarps) >> 2;   // TMEM lane quarter, column half
-        const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
+        PT_DUMP(status, 0, 2, tid == 0)
+    } else if (warp < kWarpE2) {
+        // ================= E1: state warps =================
+        const int half = (warp - kWarpE1) >> 2;                      // column half [64 * half, 64 * half + 64)
         const int krow = 32 * sub + lane;
+        const int v0 = 64 * half;
         float e_prev = 1.f;
-
-        // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk) back into TMEM, and
-        // its bf16 copy for the MMAs and for the saved-state store; then hand the chunk to the MMA warp.
-        auto maintain = [&](int c) {
+        PT_DECL
+        for (int c = 0; c < NC; ++c) {
+            // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk) back into TMEM
             mbar_wait(&ctl->t_done[c % kStages], (c / kStages) & 1, abort_flag);
+            PT_MARK(0)
             const float factor = e_prev * pm[(c & 3) * 128 + krow];
             e_prev = ee[(c & 3) * 128 + krow];
-            const int v0 = 64 * half;
             uint32_t r[64];
             if (c == 0) {
                 if (S0) {
@@ -152,6 +171,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 }
             } else {
                 mbar_wait(&ctl->barS, (c - 1) & 1, abort_flag);
+                PT_MARK(1)
                 tc_fence_after_sync();
                 tmem_ld32(tmem + lane_base + kColS + v0, *reinterpret_cast<uint32_t(*)[32]>(r));
                 tmem_ld32(tmem + lane_base + kColS + v0 + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
@@ -161,50 +181,24 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
             tmem_st32(tmem + lane_base + kColS + v0, *reinterpret_cast<uint32_t(*)[32]>(r));
             tmem_st32(tmem + lane_base + kColS + v0 + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
+            uint4 sw[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<uint4 *>(sbuf + half * kStateSlab + slab_chunk_off(krow, j)) = pack8(r + 8 * j);
+            for (int j = 0; j < 8; ++j) sw[j] = pack8(r + 8 * j);
             tmem_wait_st();
             tc_fence_before_sync();
+            mbar_arrive(&ctl->m_tmem);
+            PT_MARK(2)
+            // its bf16 copy, once Y = Qs S' of the previous chunk no longer reads the old one
+            if (c >= 1) mbar_wait(&ctl->barS2, (c - 1) & 1, abort_flag);
+            PT_MARK(3)
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4 *>(sbuf + half * kStateSlab + slab_chunk_off(krow, j)) = sw[j];
             fence_proxy_async_smem();
             mbar_arrive(&ctl->m_done);
-        };
-
-        // Y of chunk c: accumulator -> bf16 staging tile -> (store warp) TMA store.
-        auto y_out = [&](int c) {
-            const int b = c & 1;
-            uint32_t r[64];
-            mbar_wait(&ctl->barY[b], (c >> 1) & 1, abort_flag);
-            tc_fence_after_sync();
-            const uint32_t ta = tmem + lane_base + kColY + 128 * b + 64 * half;
-            tmem_ld32(ta, *reinterpret_cast<uint32_t(*)[32]>(r));
-            tmem_ld32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
-            tmem_wait_ld();
-            tc_fence_before_sync();
-            mbar_arrive(&ctl->y_tfree[b]);
-            if (c >= 1) mbar_wait(&ctl->y_sfree, (c - 1) & 1, abort_flag);
-            if (lane < 16) {
-                const int t = 16 * sub + lane;
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    *reinterpret_cast<uint4 *>(ybuf + half * kSlab + slab_chunk_off(t, j)) = pack8(r + 8 * j);
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(&ctl->y_staged);
-        };
-
-        for (int c = 0; c <= NC; ++c) {
-            if (c < NC) maintain(c);
-            if (want_y && c >= 1) y_out(c - 1);
-            if (want_y && c < NC) {
-                mbar_wait(&ctl->barA[c & 1], (c >> 1) & 1, abort_flag);
-                tc_fence_after_sync();
-                tril_to_slab(tmem + lane_base + kColA + 64 * (c & 1) + 32 * half, pbuf + (c & 1) * kSlab, sub, half, lane);
-                fence_proxy_async_smem();
-                tc_fence_before_sync();
-                mbar_arrive(&ctl->p_ready[c & 1]);
-            }
+            PT_MARK(4)
         }
+        PT_DUMP(status, 2, 5, tid == kWarpE1 * 32)
 
         // S_N = Diag(E_last) S''
         mbar_wait(&ctl->barS, (NC - 1) & 1, abort_flag);
@@ -213,18 +207,65 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             uint32_t r[32];
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
-                const int v0 = 64 * half + 32 * part;
-                tmem_ld32(tmem + lane_base + kColS + v0, r);
+                tmem_ld32(tmem + lane_base + kColS + v0 + 32 * part, r);
                 tmem_wait_ld();
-                float4 *dst = reinterpret_cast<float4 *>(SN + ((size_t)u * kD + krow) * kD + v0);
+                float4 *dst = reinterpret_cast<float4 *>(SN + ((size_t)u * kD + krow) * kD + v0 + 32 * part);
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * e_prev, __uint_as_float(r[4 * j + 1]) * e_prev,
                                          __uint_as_float(r[4 * j + 2]) * e_prev, __uint_as_float(r[4 * j + 3]) * e_prev);
             }
         }
+    } else if (warp < kWarpLoad) {
+        // ================= E2: output warps =================
+        if (want_y) {
+            const int t = 16 * sub + lane;                           // accumulator row of lanes 0..15
+            PT_DECL
+            // iteration c: tril(A(c)) -> operand slab | Y(c-1) -> staging tile
+            for (int c = 0; c <= NC; ++c) {
+                if (c < NC) {
+                    const int b = c & 1;
+                    mbar_wait(&ctl->barA[b], (c >> 1) & 1, abort_flag);
+                    PT_MARK(0)
+                    tc_fence_after_sync();
+                    tril_to_slab(tmem + lane_base + kColA + 64 * b, pbuf + b * kSlab, sub, 0, lane);
+                    tril_to_slab(tmem + lane_base + kColA + 64 * b + 32, pbuf + b * kSlab, sub, 1, lane);
+                    fence_proxy_async_smem();
+                    tc_fence_before_sync();
+                    mbar_arrive(&ctl->p_ready[b]);
+                    PT_MARK(1)
+                }
+                if (c >= 1) {
+                    const int b = (c - 1) & 1;
+                    mbar_wait(&ctl->barY[b], ((c - 1) >> 1) & 1, abort_flag);
+                    PT_MARK(2)
+                    tc_fence_after_sync();
+                    if (c >= 2) mbar_wait(&ctl->y_sfree, (c - 2) & 1, abort_flag);
+                    PT_MARK(3)
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t r[64];
+                        const uint32_t ta = tmem + lane_base + kColY + 128 * b + 64 * h;
+                        tmem_ld32(ta, *reinterpret_cast<uint32_t(*)[32]>(r));
+                        tmem_ld32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
+                        tmem_wait_ld();
+                        if (lane < 16) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<uint4 *>(ybuf + h * kSlab + slab_chunk_off(t, j)) = pack8(r + 8 * j);
+                        }
+                    }
+                    tc_fence_before_sync();
+                    mbar_arrive(&ctl->y_tfree[b]);
+                    fence_proxy_async_smem();
+                    mbar_arrive(&ctl->y_staged);
+                    PT_MARK(4)
+                }
+            }
+            PT_DUMP(status, 7, 5, tid == kWarpE2 * 32)
+        }
     } else if (warp == kWarpLoad) {
-        // ================= TMA loads =================
+        // ================= L: TMA loads =================
         if (lane == 0) {
             for (int c = 0; c < NC; ++c) {
                 const int s = c % kStages;
@@ -238,68 +279,97 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 }
             }
         }
-    } else if (warp == kWarpMma) {
-        // ================= MMA issue (+ saved-state stores) =================
+    } else if (warp == kWarpMmaS) {
+        // ================= MS: state update =================
+        if (lane == 0) {
+            constexpr uint32_t idescS = idesc_bf16(128, 128, 1, 1);    // Ks^T (MN-major) x V (MN-major)
+            // Descriptors are formed once; a K step or a stage change only adds to the 14-bit
+            // start-address field (addresses are in 16-byte units and stay below 2^14).
+            const uint64_t dfm0 = smem_desc_sw128(smem_u32(smem) + kTile, kSlab, 1024);      // Ks, MN-major
+            const uint64_t dvm0 = smem_desc_sw128(smem_u32(smem) + 2 * kTile, kSlab, 1024);  // V, MN-major
+            PT_DECL
+            for (int c = 0; c < NC; ++c) {
+                const int s = c % kStages;
+                const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
+                mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
+                mbar_wait(&ctl->t_done[s], (c / kStages) & 1, abort_flag);
+                PT_MARK(0)
+                mbar_wait(&ctl->m_tmem, c & 1, abort_flag);
+                PT_MARK(1)
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // S' += Ks^T V
+                    mma_bf16_ss(tmem + kColS, dfm0 + so + (uint64_t)(kk * 128), dvm0 + so + (uint64_t)(kk * 128),
+                                idescS, 1);
+                mma_commit(&ctl->barS);
+                mma_commit(&ctl->empty[s]);
+                PT_MARK(2)
+            }
+            PT_DUMP(status, 12, 3, true)
+        }
+    } else if (warp == kWarpMmaY) {
+        // ================= MY: outputs (+ saved-state stores) =================
         if (lane == 0) {
             constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
             constexpr uint32_t idescY = idesc_bf16(64, 128, 0, 1);     // Qs or P (K-major) x S' or V (MN-major)
-            constexpr uint32_t idescS = idesc_bf16(128, 128, 1, 1);    // Ks^T (MN-major) x V (MN-major)
-            const uint32_t sa = smem_u32(sbuf);
+            const uint64_t dq0 = smem_desc_sw128(smem_u32(smem), 16, 1024);                  // Qs, K-major
+            const uint64_t dfk0 = smem_desc_sw128(smem_u32(smem) + kTile, 16, 1024);         // Ks, K-major
+            const uint64_t dvm0 = smem_desc_sw128(smem_u32(smem) + 2 * kTile, kSlab, 1024);  // V, MN-major
+            const uint64_t dsm = smem_desc_sw128(smem_u32(sbuf), kStateSlab, 1024);          // S', MN-major
+            const uint64_t dp0 = smem_desc_sw128(smem_u32(pbuf), 16, 1024);                  // tril(A), K-major
+            auto kmaj = [](int kk) { return (uint64_t)(((kk >> 2) * kSlab + (kk & 3) * 32) >> 4); };
+            PT_DECL
             for (int c = 0; c < NC; ++c) {
                 const int s = c % kStages, b = c & 1;
-                const uint32_t qa = smem_u32(smem + s * kStageBytes);
-                const uint32_t fa = qa + kTile, va = qa + 2 * kTile;
-                const uint32_t pa = smem_u32(pbuf + b * kSlab);
+                const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
+                const uint64_t dq = dq0 + so, dfk = dfk0 + so, dvm = dvm0 + so;
+                const uint64_t dp = dp0 + (uint64_t)b * (kSlab >> 4);
                 const uint32_t ty = tmem + kColY + 128 * b, ta = tmem + kColA + 64 * b;
                 mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (c / kStages) & 1, abort_flag);
+                PT_MARK(0)
+                if (want_y) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)          // A = Qs Ks^T
+                        mma_bf16_ss(ta, dq + kmaj(kk), dfk + kmaj(kk), idescA, kk > 0);
+                    mma_commit(&ctl->barA[b]);
+                }
                 mbar_wait(&ctl->m_done, c & 1, abort_flag);
-                tc_fence_after_sync();
+                PT_MARK(1)
                 if (want_saved) {
                     tma_store_3d(&map_saved, sbuf, 0, 0, u * NC + c);
                     tma_store_3d(&map_saved, sbuf + kStateSlab, 64, 0, u * NC + c);
                     tma_store_commit();
                 }
                 if (want_y) {
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {        // A = Qs Ks^T
-                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                        mma_bf16_ss(ta, smem_desc_sw128(qa + koff, 16, 1024), smem_desc_sw128(fa + koff, 16, 1024),
-                                    idescA, kk > 0);
-                    }
-                    mma_commit(&ctl->barA[b]);
                     if (c >= 2) {
                         mbar_wait(&ctl->y_tfree[b], ((c - 2) >> 1) & 1, abort_flag);
                         tc_fence_after_sync();
                     }
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {        // Y = Qs S'
-                        const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                        mma_bf16_ss(ty, smem_desc_sw128(qa + koff, 16, 1024),
-                                    smem_desc_sw128(sa + kk * 2048, kStateSlab, 1024), idescY, kk > 0);
-                    }
+                    for (int kk = 0; kk < 8; ++kk)          // Y = Qs S'
+                        mma_bf16_ss(ty, dq + kmaj(kk), dsm + (uint64_t)(kk * 128), idescY, kk > 0);
                 }
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)              // S' += Ks^T V
-                    mma_bf16_ss(tmem + kColS, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
-                                smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescS, 1);
-                if (want_saved) tma_store_wait_read();      // the S' copy is rewritten once barS fires
-                mma_commit(&ctl->barS);
+                PT_MARK(2)
+                if (want_saved) tma_store_wait_read();      // the S' copy is rewritten once barS2 fires
+                mma_commit(&ctl->barS2);
                 if (want_y) {
                     mbar_wait(&ctl->p_ready[b], (c >> 1) & 1, abort_flag);
+                    PT_MARK(3)
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)          // Y += P V
-                        mma_bf16_ss(ty, smem_desc_sw128(pa + kk * 32, 16, 1024),
-                                    smem_desc_sw128(va + kk * 2048, kSlab, 1024), idescY, 1);
+                        mma_bf16_ss(ty, dp + (uint64_t)(kk * 2), dvm + (uint64_t)(kk * 128), idescY, 1);
                     mma_commit(&ctl->barY[b]);
                 }
                 mma_commit(&ctl->empty[s]);
+                PT_MARK(4)
             }
+            PT_DUMP(status, 15, 5, true)
             if (want_saved) tma_store_wait_all();
         }
     } else {
-        // ================= Y stores =================
+        // ================= ST: Y stores =================
         if (lane == 0 && want_y) {
             for (int c = 0; c < NC; ++c) {
                 mbar_wait(&ctl->y_staged, c & 1, abort_flag);
@@ -319,7 +389,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         // a load may still be in flight towards this CTA's shared memory: give it time to land
         for (int s = 0; s < kStages; ++s) {
             const int last = ((NC - 1 - s) / kStages) * kStages + s;     // last chunk that used stage s
-            if (last >= 0 && s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
+            if (s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
         }
     }
     __syncthreads();

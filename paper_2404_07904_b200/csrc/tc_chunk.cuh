@@ -34,6 +34,18 @@ constexpr float kProdFloor = 7.888609052210118e-31f;   // 2^-100
 constexpr uint32_t kTmemCols = 512;
 constexpr int kTransformThreads = 128;          // threads that run transform_stream together
 
+// Optional per-role cycle counters of CTA 0 (development aid; compiled out unless HGRN2_PHASE_TIMING
+// is defined).  Totals land in the padding words of the status block.
+#ifdef HGRN2_PHASE_TIMING
+#define PT_DECL long long pt_t0 = clock64(); long long pt_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+#define PT_MARK(i) { const long long pt_t = clock64(); pt_acc[i] += pt_t - pt_t0; pt_t0 = pt_t; }
+#define PT_DUMP(st, base, n, cond) if ((cond) && blockIdx.x == 0 && (st) != nullptr) { for (int pt_i = 0; pt_i < (n); ++pt_i) (st)->pad[(base) + pt_i] = (int)(pt_acc[pt_i] >> 4); }
+#else
+#define PT_DECL
+#define PT_MARK(i)
+#define PT_DUMP(st, base, n, cond)
+#endif
+
 __device__ __forceinline__ float rcp_fast(float x)
 {
     float r;
@@ -54,52 +66,69 @@ __device__ __forceinline__ uint4 pack8(const uint32_t *r)
 // In-place rescaling of the raw o and f tiles of one chunk into Qs and Ks (see the file header).
 // Run by 128 threads with no synchronisation among them: thread = one column pair x one half of the
 // chunk.  The half before the middle walks its rows downwards from row 31, the half after it walks
-// upwards from row 32, each carrying the running product of f, so nothing but the current row is
-// live.  Pm (product over rows 0..31) and E (product over rows 32..63) of the chunk are left in
-// pm[128] and ee[128].  Rows at or beyond n_valid are the neutral token f = 1, o = 0.
-template <bool kFull>
-__device__ __forceinline__ void transform_stream(uint8_t *qbuf, uint8_t *fbuf, float *pm, float *ee, int n_valid,
-                                                 int tid)
+// upwards from row 32, each carrying the running product of f, so only a few rows are live.  Rows are
+// handled in batches of eight, and the loads of the next batch are issued before the stores of the
+// current one (the tiles are rewritten in place, so the compiler would otherwise serialise every
+// load behind the previous row's stores).  Pm (product over rows 0..31) and E (product over rows
+// 32..63) of the chunk are left in pm[128] and ee[128].  Rows at or beyond n_valid are the neutral
+// token f = 1, o = 0.
+template <bool kFull, bool kUp>
+__device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, float *tot, int n_valid, int p)
 {
-    const int h = tid >> 6, p = tid & 63;
     const int col = 2 * p;
     const int jch = (col & 63) >> 3;
     const uint32_t base = (col >> 6) * kSlab + (col & 7) * 2;
     uint32_t xo[8];
 #pragma unroll
     for (int jj = 0; jj < 8; ++jj) xo[jj] = base + ((jch ^ jj) << 4);
-    float a0 = 1.f, a1 = 1.f;
-    if (h == 1) {
+    auto row_of = [](int i) { return kUp ? 32 + i : 31 - i; };     // i-th row visited
+    uint32_t fw[8], qw[8], fn[8], qn[8];
 #pragma unroll
-        for (int r = 32; r < 64; ++r) {
-            const uint32_t off = xo[r & 7] + r * 128;
-            uint32_t fw = *reinterpret_cast<const uint32_t *>(fbuf + off);
-            uint32_t qw = *reinterpret_cast<const uint32_t *>(qbuf + off);
-            if (!kFull && r >= n_valid) { fw = 0x3F803F80u; qw = 0u; }
-            const float f0 = bf16_lo(fw), f1 = bf16_hi(fw);
-            a0 *= f0; a1 *= f1;
-            const float m0 = fmaxf(a0, kProdFloor), m1 = fmaxf(a1, kProdFloor);
-            const float i0 = rcp_fast(m0), i1 = rcp_fast(m1);
-            *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(bf16_lo(qw) * m0, bf16_hi(qw) * m1);
-            *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0) * i0, (1.f - f1) * i1);
-        }
-        *reinterpret_cast<float2 *>(ee + col) = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
-    } else {
-#pragma unroll
-        for (int r = 31; r >= 0; --r) {
-            const uint32_t off = xo[r & 7] + r * 128;
-            uint32_t fw = *reinterpret_cast<const uint32_t *>(fbuf + off);
-            uint32_t qw = *reinterpret_cast<const uint32_t *>(qbuf + off);
-            if (!kFull && r >= n_valid) { fw = 0x3F803F80u; qw = 0u; }
-            const float f0 = bf16_lo(fw), f1 = bf16_hi(fw);
-            const float m0 = fmaxf(a0, kProdFloor), m1 = fmaxf(a1, kProdFloor);
-            const float i0 = rcp_fast(m0), i1 = rcp_fast(m1);
-            *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(bf16_lo(qw) * i0, bf16_hi(qw) * i1);
-            *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0) * m0, (1.f - f1) * m1);
-            a0 *= f0; a1 *= f1;
-        }
-        *reinterpret_cast<float2 *>(pm + col) = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
+    for (int j = 0; j < 8; ++j) {
+        const int r = row_of(j);
+        const uint32_t off = xo[r & 7] + r * 128;
+        fn[j] = *reinterpret_cast<const uint32_t *>(fbuf + off);
+        qn[j] = *reinterpret_cast<const uint32_t *>(qbuf + off);
     }
+    float a0 = 1.f, a1 = 1.f;
+#pragma unroll 1
+    for (int b = 0; b < 4; ++b) {      // kept rolled: the body is long and every transform warp streams through it
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { fw[j] = fn[j]; qw[j] = qn[j]; }
+        if (b < 3) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int r = row_of(8 * (b + 1) + j);
+                const uint32_t off = xo[r & 7] + r * 128;
+                fn[j] = *reinterpret_cast<const uint32_t *>(fbuf + off);
+                qn[j] = *reinterpret_cast<const uint32_t *>(qbuf + off);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int r = row_of(8 * b + j);
+            const uint32_t off = xo[r & 7] + r * 128;
+            if (!kFull && r >= n_valid) { fw[j] = 0x3F803F80u; qw[j] = 0u; }
+            const float f0 = bf16_lo(fw[j]), f1 = bf16_hi(fw[j]);
+            if (kUp) { a0 *= f0; a1 *= f1; }
+            const float m0 = fmaxf(a0, kProdFloor), m1 = fmaxf(a1, kProdFloor);
+            const float i0 = rcp_fast(m0), i1 = rcp_fast(m1);
+            if (!kUp) { a0 *= f0; a1 *= f1; }
+            const float sq0 = kUp ? m0 : i0, sq1 = kUp ? m1 : i1;
+            const float sk0 = kUp ? i0 : m0, sk1 = kUp ? i1 : m1;
+            *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(bf16_lo(qw[j]) * sq0, bf16_hi(qw[j]) * sq1);
+            *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0) * sk0, (1.f - f1) * sk1);
+        }
+    }
+    *reinterpret_cast<float2 *>(tot + col) = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
+}
+
+template <bool kFull>
+__device__ __forceinline__ void transform_stream(uint8_t *qbuf, uint8_t *fbuf, float *pm, float *ee, int n_valid,
+                                                 int tid)
+{
+    if (tid >> 6) transform_half<kFull, true>(qbuf, fbuf, ee, n_valid, tid & 63);
+    else          transform_half<kFull, false>(qbuf, fbuf, pm, n_valid, tid & 63);
 }
 
 // Causal mask + bf16 of 32 columns (32 * half ...) of one 64 x 64 fp32 accumulator in the M = 64
