@@ -1,5 +1,41 @@
 // Chunkwise HGRN2 backward on the Blackwell tensor cores (tcgen05 + TMEM + TMA), bf16 I/O, fp32
-// state gradient, d_k = d_v = 128, chunk length C = 64 (frame and formulas: tc_chunk.cuh).
+// state gradient, d_k = d_v = 128, chunk length C = 64 (frame and notation: tc_chunk.cuh).
+//
+// Reverse sweep over the chunks with the state gradient resident in tensor memory.  In the mid frame,
+// with dS'' = Diag(E) dS_out and S' the saved forward state of the chunk:
+//
+//   A  = tril(Qs Ks^T)          dA = tril(dY V^T)
+//   dQs^T       = Ks^T dA^T + S' dY^T            (accumulator [key dim][t])
+//   dKs_intra^T = Qs^T dA                        (accumulator [key dim][s])
+//   dKs_inter^T = dS'' V^T                       (accumulator [key dim][s])
+//   dV^T        = dY^T A + dS''^T Ks^T           (accumulator [value dim][s])
+//   dS'         = dS'' + Qs^T dY,   dS_in = Diag(Pm) dS'
+//   a = Qs*dQs - Ks*dKs_intra,  e = Ks*dKs_inter,  R_k = sum_v dS''[k,v] S'[k,v]
+//   dg_t = sum_{j>=t} a_j + sum_{s<t} e_s + R            (gradient w.r.t. log f_t)
+//   d_o = dQs * exp(b_t - b_m),  dk = (dKs_intra + dKs_inter) * exp(b_m - b_s),  d_f = dg / f - dk
+//
+// Every accumulator that feeds an output puts one key (or value) dimension in each TMEM lane, so the
+// thread that owns the lane sees a whole column of the chunk: the scans along time stay in registers
+// and each output store of a warp covers 64 contiguous bytes of one token row.
+//
+// Warp roles (hand-offs are mbarriers, every wait is bounded; loops stay rolled to keep the
+// instruction footprint of the concurrently running roles small):
+//   T   4 warps: raw o, f tiles -> Qs, Ks in place, one chunk ahead (two TMA stages);
+//   E1  4 warps: rescale the dS accumulator and publish its bf16 copy dS'' (the chain between
+//       chunks), causal masks of A and dA into operand slabs, R;
+//   E3  8 warps: outputs.  d_i from dV^T; d_o and d_f from dQs^T, dKs_intra^T, dKs_inter^T.  A
+//       thread owns (key dim, half of the chunk) and walks its 32 steps outwards from the middle,
+//       carrying the decay product and the running sums; what is still missing then is one constant
+//       per key dimension (R plus the other half's sums), so the almost finished d_f and 1/f are
+//       parked in the TMEM columns just read and completed after the two halves have exchanged sums;
+//   L   1 warp: TMA loads (raw tiles, saved S');   M  1 warp: tcgen05.mma issue.
+// Per chunk the tensor pipe runs
+//   X : dS' += Qs^T dY | A | dA            (overlaps the outputs of the previous chunk)
+//   Y1: dKs_inter^T | dV^T = dS''^T Ks^T   (needs the previous chunk's dKs_inter^T, dV^T read out)
+//   Y2: dQs^T | dKs_intra^T | dV^T += dY^T A   (needs tril(A), tril(dA), S', and the parked values consumed)
+//
+// Tensor-memory plan (512 columns, no spare): dS [0,128); A [128,192), dA [192,256) in the M = 64
+// layout; dQs^T [256,320); dKs_intra^T [320,384); dKs_inter^T [384,448); dV^T [448,512).
 #include "tc_chunk.cuh"
 
 namespace hgrn2 {
@@ -8,149 +44,109 @@ namespace {
 
 using namespace tc;
 
-constexpr int kWorkers = 256;                   // warps 0..7: transforms, TMEM epilogues, outputs
-constexpr int kThreads = kWorkers + 32;         // warp 8: TMA loads and tcgen05.mma issue (one lane)
+constexpr int kTWarps = 4, kE1Warps = 4, kE3Warps = 8;
+constexpr int kE1Threads = kE1Warps * 32, kE3Threads = kE3Warps * 32;
+constexpr int kWarpE1 = kTWarps, kWarpE3 = kWarpE1 + kE1Warps;
+constexpr int kWarpLoad = kWarpE3 + kE3Warps, kWarpMma = kWarpLoad + 1;
+constexpr int kThreads = (kWarpMma + 1) * 32;
 
-__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+constexpr int kStages = 2;
+constexpr uint32_t kStageBytes = 4 * kTile;                       // q, f, v, dy
+constexpr uint32_t kOffS = kStages * kStageBytes;                 // S' (bf16, from the forward)
+constexpr uint32_t kOffDS = kOffS + kStateTile;                   // bf16 copy of dS''
+constexpr uint32_t kOffP = kOffDS + kStateTile;                   // bf16 tril(A)
+constexpr uint32_t kOffDP = kOffP + kSlab;                        // bf16 tril(dA)
+constexpr uint32_t kOffPm = kOffDP + kSlab;                       // float pm[4][128]
+constexpr uint32_t kOffE = kOffPm + 4 * 128 * 4;                  // float ee[4][128]
+constexpr uint32_t kOffR = kOffE + 4 * 128 * 4;                   // float rr[2][128]
+constexpr uint32_t kOffX = kOffR + 2 * 128 * 4;                   // float xa[128], xe[128]
+constexpr uint32_t kOffCtl = kOffX + 2 * 128 * 4;
+constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024;
 
-// In-place rescaling of the raw o and f tiles of one chunk into Qs and Ks (see the file header).
-// Thread layout: 64 column pairs x 4 row quarters; quarter q owns rows 16q..16q+15.  Quarter totals
-// go through `tot`; Pm and E of the chunk are left in `pm` and `ee`.  Called by all 256 workers.
-__device__ __forceinline__ void transform_chunk(uint8_t *qbuf, uint8_t *fbuf, float *tot, float *pm, float *ee,
-                                                int n_valid, int tid)
-{
-    const int quarter = tid >> 6, p = tid & 63;
-    const int col = 2 * p;
-    const int jch = (col & 63) >> 3;
-    const uint32_t base = (col >> 6) * kSlab + quarter * 16 * 128 + (col & 7) * 2;
-    uint32_t xo[8];
-#pragma unroll
-    for (int jj = 0; jj < 8; ++jj) xo[jj] = base + ((jch ^ jj) << 4);   // row 16q + j has (row & 7) == (j & 7)
-    uint32_t qw[16];
-    float f0[16], f1[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const uint32_t off = xo[j & 7] + j * 128;
-        uint32_t fw = *reinterpret_cast<const uint32_t *>(fbuf + off);
-        qw[j] = *reinterpret_cast<const uint32_t *>(qbuf + off);
-        if (quarter * 16 + j >= n_valid) {       // neutral padding token: f = 1, o = 0
-            fw = 0x3F803F80u;
-            qw[j] = 0u;
-        }
-        f0[j] = bf16_lo(fw);
-        f1[j] = bf16_hi(fw);
-    }
-    // m0[j], m1[j]: product of f over the rows between row j and the middle of the chunk
-    // (quarters 0, 1: rows j+1 .. 31; quarters 2, 3: rows 32 .. j), restricted to this quarter.
-    float m0[16], m1[16];
-    float t0, t1;
-    if (quarter < 2) {
-        float a0 = 1.f, a1 = 1.f;
-#pragma unroll
-        for (int j = 15; j >= 0; --j) {
-            m0[j] = a0; m1[j] = a1;
-            a0 *= f0[j]; a1 *= f1[j];
-        }
-        t0 = a0; t1 = a1;
-    } else {
-        float a0 = 1.f, a1 = 1.f;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            a0 *= f0[j]; a1 *= f1[j];
-            m0[j] = a0; m1[j] = a1;
-        }
-        t0 = a0; t1 = a1;
-    }
-    *reinterpret_cast<float2 *>(tot + quarter * 128 + col) = make_float2(t0, t1);
-    worker_sync();
-    float o0 = 1.f, o1 = 1.f;
-    if (quarter == 0) { const float2 x = *reinterpret_cast<const float2 *>(tot + 128 + col); o0 = x.x; o1 = x.y; }
-    if (quarter == 3) { const float2 x = *reinterpret_cast<const float2 *>(tot + 256 + col); o0 = x.x; o1 = x.y; }
-    if (quarter == 0)
-        *reinterpret_cast<float2 *>(pm + col) = make_float2(fmaxf(t0 * o0, kProdFloor), fmaxf(t1 * o1, kProdFloor));
-    if (quarter == 3)
-        *reinterpret_cast<float2 *>(ee + col) = make_float2(fmaxf(t0 * o0, kProdFloor), fmaxf(t1 * o1, kProdFloor));
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const uint32_t off = xo[j & 7] + j * 128;
-        const float mm0 = fmaxf(m0[j] * o0, kProdFloor), mm1 = fmaxf(m1[j] * o1, kProdFloor);
-        const float i0 = rcp_fast(mm0), i1 = rcp_fast(mm1);
-        const float sq0 = quarter < 2 ? i0 : mm0, sq1 = quarter < 2 ? i1 : mm1;
-        const float sk0 = quarter < 2 ? mm0 : i0, sk1 = quarter < 2 ? mm1 : i1;
-        const float q0 = bf16_lo(qw[j]), q1 = bf16_hi(qw[j]);
-        *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(q0 * sq0, q1 * sq1);
-        *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0[j]) * sk0, (1.f - f1[j]) * sk1);
-    }
-}
+constexpr uint32_t kColDS = 0, kColA = 128, kColDA = 192, kColDQ = 256, kColDKi = 320, kColDKx = 384, kColDV = 448;
 
-// One 64 x 128 fp32 accumulator (M = 64 layout) to a bf16 [token][128] global tensor.
-__device__ __forceinline__ void rows_to_global(uint32_t taddr_half, __nv_bfloat16 *dst_row0, int sub, int half,
-                                               int lane, int n_valid)
-{
-    uint32_t r[32];
-    const int t = 16 * sub + lane;
-#pragma unroll
-    for (int part = 0; part < 2; ++part) {
-        tmem_ld32(taddr_half + 32 * part, r);
-        tmem_wait_ld();
-        if (lane < 16 && t < n_valid) {
-            uint4 *dst = reinterpret_cast<uint4 *>(dst_row0 + (size_t)t * kD + 64 * half + 32 * part);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) dst[j] = pack8(r + 8 * j);
-        }
-    }
-}
-
-// ---- backward ---------------------------------------------------------------------------------------
-// Reverse sweep over the chunks with the state gradient resident in tensor memory.  In the mid frame
-// (file header), with dS'' = Diag(E) dS_out and S' the saved forward state of the chunk:
-//
-//   A  = tril(Qs Ks^T)          dA = tril(dY V^T)
-//   dQs^T       = Ks^T dA^T + S' dY^T            (accumulator [key dim][t]: lane = key dim)
-//   dKs_intra^T = Qs^T dA                        (accumulator [key dim][s])
-//   dKs_inter^T = dS'' V^T                       (accumulator [key dim][s])
-//   dV          = A^T dY + Ks dS''               (accumulator [s][value dim])
-//   dS'         = dS'' + Qs^T dY,   dS_in = Diag(Pm) dS'
-//   a = Qs*dQs - Ks*dKs_intra,  e = Ks*dKs_inter,  R_k = sum_v dS''[k,v] S'[k,v]
-//   dg_t = sum_{j>=t} a_j + sum_{s<t} e_s + R            (gradient w.r.t. log f_t; no cancellation
-//                                                         between the inter-chunk terms)
-//   d_o = dQs * exp(b_t - b_m),  dk = (dKs_intra + dKs_inter) * exp(b_m - b_s),  d_f = dg / f - dk
-//
-// The three key-dimension-major accumulators put one key dimension in each TMEM lane, so the thread
-// that owns the lane sees a whole column of the chunk and the scans along time stay in registers.
-// Tensor-memory plan: dS [0,128); A [128,192) and dA [192,256) first, then dQs^T and dKs_intra^T in
-// the same columns; dKs_inter^T [256,320); dV [320,448).
-//
-// Worker schedule per processed chunk `it` (chunk index c = NC-1-it):
-//   P/dP epilogue(it) | transform(it+1) | dV epilogue(it), d_o/d_f phase(it) | dS maintenance(it+1)
-// so the second group of MMAs overlaps the next transform.  The raw-tile stage is released to TMA as
-// soon as the d_o/d_f phase has read Qs and Ks from it.
-constexpr int kBwdStages = 2;
-constexpr uint32_t kBwdStageBytes = 4 * kTile;                        // q, f, v, dy
-constexpr uint32_t kBwdOffS = kBwdStages * kBwdStageBytes;            // S' (bf16, from the forward)
-constexpr uint32_t kBwdOffDS = kBwdOffS + kStateTile;                 // bf16 copy of dS''
-constexpr uint32_t kBwdOffP = kBwdOffDS + kStateTile;                 // bf16 tril(A)
-constexpr uint32_t kBwdOffDP = kBwdOffP + kSlab;                      // bf16 tril(dA)
-constexpr uint32_t kBwdOffTot = kBwdOffDP + kSlab;                    // float tot[4][128]
-constexpr uint32_t kBwdOffPm = kBwdOffTot + 4 * 128 * 4;
-constexpr uint32_t kBwdOffE = kBwdOffPm + 128 * 4;
-constexpr uint32_t kBwdOffR = kBwdOffE + 128 * 4;                     // float rpart[2][128]
-constexpr uint32_t kBwdOffX = kBwdOffR + 2 * 128 * 4;                 // float xa[128], xe[128]
-constexpr uint32_t kBwdOffBar = kBwdOffX + 2 * 128 * 4;
-constexpr uint32_t kBwdSmemBytes = kBwdOffBar + 256 + 1024;
-
-constexpr uint32_t kColDS = 0, kColA2 = 128, kColDA = 192, kColDQ = 128, kColDKi = 192, kColDKx = 256, kColDV = 320;
-
-struct BwdCtl {
-    uint64_t full[kBwdStages];     // TMA (raw tiles) -> workers
-    uint64_t sfull;                // TMA (saved S') -> workers
-    uint64_t g1_ready;             // workers -> issuer: Qs, Ks, dS'' ready: first MMA group may go
-    uint64_t pd_ready;             // workers -> issuer: tril(A), tril(dA) in shared memory: second group may go
-    uint64_t f_done;               // workers -> issuer: the chunk's stage has been read for the last time
-    uint64_t bar1, bar2;           // tcgen05.commit -> workers
+struct Ctl {
+    uint64_t full[kStages];       // TMA (raw tiles) -> T, M
+    uint64_t stage_read[kStages]; // E3 -> L: Qs, Ks of the stage have been read for the last time
+    uint64_t t_done[kStages];     // T -> M, E1
+    uint64_t sfull;               // TMA (saved S') -> E1, M
+    uint64_t m_done;              // E1 -> M: dS'' is in TMEM and in shared memory
+    uint64_t barX;                // tcgen05.commit -> E1: dS' update, A, dA complete
+    uint64_t pd_ready;            // E1 -> M: tril(A), tril(dA) are in shared memory
+    uint64_t barY1;               // tcgen05.commit -> E1: dS'' copy no longer read
+    uint64_t barY2;               // tcgen05.commit -> E3, L: every product of the chunk complete
+    uint64_t r_ready[2];          // E1 -> E3, L: R of the chunk is in shared memory, S' no longer read by threads
+                                  // (two barriers: the slower of the two waiters must not be lapped)
+    uint64_t acc_free1;           // E3 -> M: dKs_inter^T and dV^T have been read out
+    uint64_t acc_free2;           // E3 -> M: dQs^T and dKs_intra^T columns are free again
     uint32_t tmem_base;
     int abort_flag;
 };
+static_assert(sizeof(Ctl) <= 256, "control block");
+static_assert(kSmemBytes <= 232448, "shared memory budget");
+
+__device__ __forceinline__ void e3_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// d_o and the nearly finished d_f of one thread: key dimension k, local times [32 * kUp, 32 * kUp + 32),
+// walked outwards from the middle of the chunk in blocks of eight.  Returns this half's sums of a and e.
+// f_g / do_g point at element (row 0 of the chunk, column k) of f and d_o in global memory.
+template <bool kUp>
+__device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qtile, const uint8_t *ktile, int k,
+                                           const __nv_bfloat16 *f_g, __nv_bfloat16 *do_g, int n_valid, float &asum,
+                                           float &esum)
+{
+    const int kch = (k & 63) >> 3;
+    const uint32_t kbase = (k >> 6) * kSlab + (k & 7) * 2;
+    float cp = 1.f;                 // running product of f between the middle and the current row
+    float G = 0.f, H = 0.f;         // running sums of a and e over the rows visited so far
+#pragma unroll 1
+    for (int b = 0; b < 4; ++b) {
+        const int t0 = kUp ? 32 + 8 * b : 24 - 8 * b;          // lowest row of the block (a multiple of 8)
+        uint32_t x[8], y[8], z[8];
+        tmem_ld8(tmem_lane + kColDQ + t0, x);
+        tmem_ld8(tmem_lane + kColDKi + t0, y);
+        tmem_ld8(tmem_lane + kColDKx + t0, z);
+        float fv[8], qs[8], ks[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int t = t0 + j;
+            const uint32_t off = kbase + t * 128 + ((kch ^ j) << 4);
+            fv[j] = (t < n_valid) ? __bfloat162float(f_g[(size_t)t * kD]) : 1.f;
+            qs[j] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(qtile + off));
+            ks[j] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(ktile + off));
+        }
+        tmem_wait_ld();
+        float u[8], rf[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int j = kUp ? i : 7 - i;                      // visiting order: away from the middle
+            const int t = t0 + j;
+            if (kUp) cp *= fv[j];
+            const float m = fmaxf(cp, kProdFloor);
+            const float mi = rcp_fast(m);
+            if (!kUp) cp *= fv[j];
+            const float sq = kUp ? m : mi, sk = kUp ? mi : m;
+            const float xx = __uint_as_float(x[j]), yy = __uint_as_float(y[j]), zz = __uint_as_float(z[j]);
+            if (t < n_valid) do_g[(size_t)t * kD] = __float2bfloat16_rn(xx * sq);
+            const float a = fmaf(qs[j], xx, -ks[j] * yy);
+            const float e = ks[j] * zz;
+            const float dk = (yy + zz) * sk;
+            rf[j] = rcp_fast(fmaxf(fv[j], kProdFloor));
+            if (kUp) {              // rows after the middle: sums over the rows strictly before t
+                u[j] = fmaf(H - G, rf[j], -dk);
+                G += a; H += e;
+            } else {                // rows before the middle: sums over the rows from t on
+                G += a; H += e;
+                u[j] = fmaf(G - H, rf[j], -dk);
+            }
+        }
+        // park u and 1/f in the columns just read
+        tmem_st8(tmem_lane + kColDQ + t0, u);
+        tmem_st8(tmem_lane + kColDKi + t0, rf);
+    }
+    asum = G;
+    esum = H;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
@@ -161,30 +157,37 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *sbuf = smem + kBwdOffS;
-    uint8_t *dsbuf = smem + kBwdOffDS;
-    uint8_t *pbuf = smem + kBwdOffP;
-    uint8_t *dpbuf = smem + kBwdOffDP;
-    float *tot = reinterpret_cast<float *>(smem + kBwdOffTot);
-    float *pm = reinterpret_cast<float *>(smem + kBwdOffPm);
-    float *ee = reinterpret_cast<float *>(smem + kBwdOffE);
-    float *rpart = reinterpret_cast<float *>(smem + kBwdOffR);
-    float *xa = reinterpret_cast<float *>(smem + kBwdOffX);
+    uint8_t *sbuf = smem + kOffS;
+    uint8_t *dsbuf = smem + kOffDS;
+    uint8_t *pbuf = smem + kOffP;
+    uint8_t *dpbuf = smem + kOffDP;
+    float *pm = reinterpret_cast<float *>(smem + kOffPm);
+    float *ee = reinterpret_cast<float *>(smem + kOffE);
+    float *rr = reinterpret_cast<float *>(smem + kOffR);
+    float *xa = reinterpret_cast<float *>(smem + kOffX);
     float *xe = xa + 128;
-    BwdCtl *ctl = reinterpret_cast<BwdCtl *>(smem + kBwdOffBar);
+    Ctl *ctl = reinterpret_cast<Ctl *>(smem + kOffCtl);
     volatile int *abort_flag = &ctl->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int u = blockIdx.x;
 
     if (tid == 0) {
-        for (int s = 0; s < kBwdStages; ++s) mbar_init(&ctl->full[s], 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->stage_read[s], kE3Threads);
+            mbar_init(&ctl->t_done[s], kTransformThreads);
+        }
         mbar_init(&ctl->sfull, 1);
-        mbar_init(&ctl->g1_ready, kWorkers);
-        mbar_init(&ctl->pd_ready, kWorkers);
-        mbar_init(&ctl->f_done, kWorkers);
-        mbar_init(&ctl->bar1, 1);
-        mbar_init(&ctl->bar2, 1);
+        mbar_init(&ctl->m_done, kE1Threads);
+        mbar_init(&ctl->barX, 1);
+        mbar_init(&ctl->pd_ready, kE1Threads);
+        mbar_init(&ctl->barY1, 1);
+        mbar_init(&ctl->barY2, 1);
+        mbar_init(&ctl->r_ready[0], kE1Threads);
+        mbar_init(&ctl->r_ready[1], kE1Threads);
+        mbar_init(&ctl->acc_free1, kE3Threads);
+        mbar_init(&ctl->acc_free2, kE3Threads);
         ctl->abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
@@ -198,22 +201,202 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = ctl->tmem_base;
+    const int sub = warp & 3;                                        // TMEM lane quarter of this warp
+    const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
+    const int krow = 32 * sub + lane;                                // TMEM lane of this thread
 
-    if (warp == 8) {
-        // ================= issuer =================
+    // it = 0, 1, ... counts processed chunks; chunk index c = NC - 1 - it
+    if (warp < kTWarps) {
+        // ================= T: transform =================
+        PT_DECL
+        for (int it = 0; it < NC; ++it) {
+            const int s = it % kStages, c = NC - 1 - it;
+            uint8_t *qbuf = smem + s * kStageBytes;
+            mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
+            PT_MARK(0)
+            const int n_valid = N - c * kC;
+            if (n_valid >= kC) {
+                transform_stream<true>(qbuf, qbuf + kTile, pm + (it & 3) * 128, ee + (it & 3) * 128, kC, tid);
+            } else {
+                transform_stream<false>(qbuf, qbuf + kTile, pm + (it & 3) * 128, ee + (it & 3) * 128, n_valid, tid);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->t_done[s]);
+            PT_MARK(1)
+        }
+        PT_DUMP(status, 0, 2, tid == 0)
+    } else if (warp < kWarpE3) {
+        // ================= E1: state-gradient warps =================
+        float pm_prev = 1.f;
+        PT_DECL
+        for (int it = 0; it < NC; ++it) {
+            // ---- dS'' = (Pm_prev E) dS' (the accumulator, or dSN first) -> TMEM, bf16 copy -> dsbuf
+            mbar_wait(&ctl->t_done[it % kStages], (it / kStages) & 1, abort_flag);
+            PT_MARK(0)
+            const float factor = pm_prev * ee[(it & 3) * 128 + krow];
+            pm_prev = pm[(it & 3) * 128 + krow];
+            if (it > 0) {
+                mbar_wait(&ctl->barY1, (it - 1) & 1, abort_flag);    // dS' update done, dsbuf no longer read
+                tc_fence_after_sync();
+            }
+            PT_MARK(1)
+#pragma unroll 1
+            for (int part = 0; part < 4; ++part) {
+                uint32_t r[32];
+                if (it == 0) {
+                    if (dSN) {
+                        const float4 *src = reinterpret_cast<const float4 *>(dSN + ((size_t)u * kD + krow) * kD + 32 * part);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 v4 = __ldg(src + j);
+                            r[4 * j + 0] = __float_as_uint(v4.x); r[4 * j + 1] = __float_as_uint(v4.y);
+                            r[4 * j + 2] = __float_as_uint(v4.z); r[4 * j + 3] = __float_as_uint(v4.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    }
+                } else {
+                    tmem_ld32(tmem + lane_base + kColDS + 32 * part, r);
+                    tmem_wait_ld();
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
+                tmem_st32(tmem + lane_base + kColDS + 32 * part, r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    *reinterpret_cast<uint4 *>(dsbuf + (part >> 1) * kStateSlab + slab_chunk_off(krow, 4 * (part & 1) + j)) =
+                        pack8(r + 8 * j);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->m_done);
+            PT_MARK(2)
+
+            // ---- tril(A), tril(dA) -> operand slabs
+            mbar_wait(&ctl->barX, it & 1, abort_flag);
+            PT_MARK(3)
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int w = 0; w < 2; ++w) {
+                const uint32_t col = w ? kColDA : kColA;
+                uint8_t *dst = w ? dpbuf : pbuf;
+                tril_to_slab(tmem + lane_base + col, dst, sub, 0, lane);
+                tril_to_slab(tmem + lane_base + col + 32, dst, sub, 1, lane);
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->pd_ready);
+            PT_MARK(4)
+
+            // ---- R_k = sum_v dS''[k,v] S'[k,v] from the two bf16 copies
+            mbar_wait(&ctl->sfull, it & 1, abort_flag);
+            PT_MARK(5)
+            float racc = 0.f;
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t off = h * kStateSlab + slab_chunk_off(krow, j);
+                    const uint4 dw = *reinterpret_cast<const uint4 *>(dsbuf + off);
+                    const uint4 sw = *reinterpret_cast<const uint4 *>(sbuf + off);
+                    racc = fmaf(bf16_lo(dw.x), bf16_lo(sw.x), racc); racc = fmaf(bf16_hi(dw.x), bf16_hi(sw.x), racc);
+                    racc = fmaf(bf16_lo(dw.y), bf16_lo(sw.y), racc); racc = fmaf(bf16_hi(dw.y), bf16_hi(sw.y), racc);
+                    racc = fmaf(bf16_lo(dw.z), bf16_lo(sw.z), racc); racc = fmaf(bf16_hi(dw.z), bf16_hi(sw.z), racc);
+                    racc = fmaf(bf16_lo(dw.w), bf16_lo(sw.w), racc); racc = fmaf(bf16_hi(dw.w), bf16_hi(sw.w), racc);
+                }
+            }
+            rr[(it & 1) * 128 + krow] = racc;
+            mbar_arrive(&ctl->r_ready[it & 1]);
+            PT_MARK(6)
+        }
+        PT_DUMP(status, 2, 7, tid == kWarpE1 * 32)
+
+        // dS_0 = Diag(Pm of chunk 0) dS'
+        mbar_wait(&ctl->barY2, (NC - 1) & 1, abort_flag);
+        tc_fence_after_sync();
+        if (dS0) {
+#pragma unroll 1
+            for (int part = 0; part < 4; ++part) {
+                uint32_t r[32];
+                tmem_ld32(tmem + lane_base + kColDS + 32 * part, r);
+                tmem_wait_ld();
+                float4 *dst = reinterpret_cast<float4 *>(dS0 + ((size_t)u * kD + krow) * kD + 32 * part);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * pm_prev, __uint_as_float(r[4 * j + 1]) * pm_prev,
+                                         __uint_as_float(r[4 * j + 2]) * pm_prev, __uint_as_float(r[4 * j + 3]) * pm_prev);
+            }
+        }
+    } else if (warp < kWarpLoad) {
+        // ================= E3: output warps =================
+        const int half = (warp - kWarpE3) >> 2;                      // half of the chunk: local times [32 * half, +32)
+        const uint32_t tl = tmem + lane_base;
+        PT_DECL
+        for (int it = 0; it < NC; ++it) {
+            const int c = NC - 1 - it, s = it % kStages;
+            const int n_valid = min(kC, N - c * kC);
+            const uint8_t *qtile = smem + s * kStageBytes, *ktile = qtile + kTile;
+            const size_t row0 = (size_t)u * N + (size_t)c * kC;
+            mbar_wait(&ctl->barY2, it & 1, abort_flag);
+            PT_MARK(0)
+            tc_fence_after_sync();
+
+            // d_i = dV: lane = value dimension, columns = local times of this half
+#pragma unroll 1
+            for (int b = 0; b < 4; ++b) {
+                uint32_t r[8];
+                const int s0 = 32 * half + 8 * b;
+                tmem_ld8(tl + kColDV + s0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (s0 + j < n_valid) d_i[(row0 + s0 + j) * kD + krow] = __float2bfloat16_rn(__uint_as_float(r[j]));
+            }
+            PT_MARK(1)
+
+            // d_o and the parked part of d_f
+            float asum, esum;
+            if (half) phase_main<true>(tl, qtile, ktile, krow, f_gmem + row0 * kD + krow, d_o + row0 * kD + krow, n_valid, asum, esum);
+            else      phase_main<false>(tl, qtile, ktile, krow, f_gmem + row0 * kD + krow, d_o + row0 * kD + krow, n_valid, asum, esum);
+            mbar_arrive(&ctl->stage_read[s]);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->acc_free1);
+            if (half) xa[krow] = asum; else xe[krow] = esum;
+            PT_MARK(2)
+            mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
+            e3_sync();
+            PT_MARK(3)
+            const float K = rr[(it & 1) * 128 + krow] + xa[krow] + xe[krow];
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int b = 0; b < 4; ++b) {
+                uint32_t uu[8], rf[8];
+                const int t0 = 32 * half + 8 * b;
+                tmem_ld8(tl + kColDQ + t0, uu);
+                tmem_ld8(tl + kColDKi + t0, rf);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (t0 + j < n_valid)
+                        d_f[(row0 + t0 + j) * kD + krow] =
+                            __float2bfloat16_rn(fmaf(K, __uint_as_float(rf[j]), __uint_as_float(uu[j])));
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->acc_free2);
+            e3_sync();                                               // xa, xe are rewritten next iteration
+            PT_MARK(4)
+        }
+        PT_DUMP(status, 9, 5, tid == kWarpE3 * 32)
+    } else if (warp == kWarpLoad) {
+        // ================= L: TMA loads =================
         if (lane == 0) {
-            constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T
-            constexpr uint32_t idKX = idesc_bf16(128, 64, 0, 0);      // dS'' (K-major) x V (K-major); S' x dY
-            constexpr uint32_t idDV2 = idesc_bf16(64, 128, 0, 1);     // Ks (K-major) x dS'' (MN-major)
-            constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
-            constexpr uint32_t idDQ1 = idesc_bf16(128, 64, 1, 0);     // Ks^T (MN-major) x dA^T (dP K-major)
-            constexpr uint32_t idDKi = idesc_bf16(128, 64, 1, 1);     // Qs^T (MN-major) x dA (dP MN-major)
-            constexpr uint32_t idDV1 = idesc_bf16(64, 128, 1, 1);     // P^T (MN-major) x dY (MN-major)
-            // it = 0, 1, ... counts processed chunks; chunk index c = NC - 1 - it
-            auto issue_loads = [&](int it) {
-                const int s = it % kBwdStages, c = NC - 1 - it;
-                uint8_t *st = smem + s * kBwdStageBytes;
-                mbar_arrive_expect_tx(&ctl->full[s], kBwdStageBytes);
+            auto issue_stage = [&](int it) {
+                const int s = it % kStages, c = NC - 1 - it;
+                uint8_t *st = smem + s * kStageBytes;
+                mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
                 for (int b = 0; b < 2; ++b) {
                     tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
                     tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
@@ -221,295 +404,122 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tma_load_3d(st + 3 * kTile + b * kSlab, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
                 }
             };
-            auto issue_state_load = [&](int it) {
+            auto issue_state = [&](int it) {
                 const int c = NC - 1 - it;
                 mbar_arrive_expect_tx(&ctl->sfull, kStateTile);
                 for (int b = 0; b < 2; ++b)
                     tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, u * NC + c);
             };
-            for (int it = 0; it < kBwdStages && it < NC; ++it) issue_loads(it);
-            issue_state_load(0);
-            const uint32_t sa = smem_u32(sbuf), dsa = smem_u32(dsbuf), pa = smem_u32(pbuf), dpa = smem_u32(dpbuf);
-            for (int it = 0; it < NC; ++it) {
-                const uint32_t qa = smem_u32(smem + (it % kBwdStages) * kBwdStageBytes);
-                const uint32_t fa = qa + kTile, va = qa + 2 * kTile, ga = qa + 3 * kTile;
-                mbar_wait(&ctl->g1_ready, it & 1, abort_flag);
-                tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {            // A = Qs Ks^T
-                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                    mma_bf16_ss(tmem + kColA2, smem_desc_sw128(qa + koff, 16, 1024),
-                                smem_desc_sw128(fa + koff, 16, 1024), idA, kk > 0);
+            issue_stage(0);
+            issue_state(0);
+            if (NC > 1) issue_stage(1);
+            for (int it = 0; it + 1 < NC; ++it) {
+                // chunk `it` is finished with S' once its products and its R are done ...
+                mbar_wait(&ctl->barY2, it & 1, abort_flag);
+                mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
+                issue_state(it + 1);
+                // ... and with its stage once the output warps have read Qs and Ks
+                if (it + 2 < NC) {
+                    mbar_wait(&ctl->stage_read[it % kStages], (it / kStages) & 1, abort_flag);
+                    issue_stage(it + 2);
                 }
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {            // dA = dY V^T
-                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                    mma_bf16_ss(tmem + kColDA, smem_desc_sw128(ga + koff, 16, 1024),
-                                smem_desc_sw128(va + koff, 16, 1024), idA, kk > 0);
-                }
-                mma_commit(&ctl->bar1);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {            // dKs_inter^T = dS'' V^T
-                    const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
-                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                    mma_bf16_ss(tmem + kColDKx, smem_desc_sw128(dsa + ko_s, 16, 1024),
-                                smem_desc_sw128(va + koff, 16, 1024), idKX, kk > 0);
-                }
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {            // dV = Ks dS''
-                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                    mma_bf16_ss(tmem + kColDV, smem_desc_sw128(fa + koff, 16, 1024),
-                                smem_desc_sw128(dsa + kk * 2048, kStateSlab, 1024), idDV2, kk > 0);
-                }
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
-                    mma_bf16_ss(tmem + kColDS, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
-                                smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDS, 1);
-                mbar_wait(&ctl->pd_ready, it & 1, abort_flag);
-                tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)              // dQs^T = Ks^T dA^T
-                    mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(fa + kk * 2048, kSlab, 1024),
-                                smem_desc_sw128(dpa + kk * 32, 16, 1024), idDQ1, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {            //        + S' dY^T
-                    const uint32_t ko_s = (kk >> 2) * kStateSlab + (kk & 3) * 32;
-                    const uint32_t koff = (kk >> 2) * kSlab + (kk & 3) * 32;
-                    mma_bf16_ss(tmem + kColDQ, smem_desc_sw128(sa + ko_s, 16, 1024),
-                                smem_desc_sw128(ga + koff, 16, 1024), idKX, 1);
-                }
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
-                    mma_bf16_ss(tmem + kColDKi, smem_desc_sw128(qa + kk * 2048, kSlab, 1024),
-                                smem_desc_sw128(dpa + kk * 2048, kSlab, 1024), idDKi, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)              // dV += P^T dY
-                    mma_bf16_ss(tmem + kColDV, smem_desc_sw128(pa + kk * 2048, kSlab, 1024),
-                                smem_desc_sw128(ga + kk * 2048, kSlab, 1024), idDV1, 1);
-                mma_commit(&ctl->bar2);
-                // S' of this chunk is dead once the second group is complete: fetch the next one
-                mbar_wait(&ctl->bar2, it & 1, abort_flag);
-                if (it + 1 < NC) issue_state_load(it + 1);
-                // the raw-tile stage is dead once the workers have read Qs and Ks for d_o / d_f
-                mbar_wait(&ctl->f_done, it & 1, abort_flag);
-                if (it + kBwdStages < NC) issue_loads(it + kBwdStages);
             }
         }
     } else {
-        // ================= workers =================
-        const int sub = warp & 3, half = warp >> 2;
-        const uint32_t lane_base = static_cast<uint32_t>(32 * sub) << 16;
-        const int krow = 32 * sub + lane;
-        float pm_prev = 1.f;
-
-        // dS'' = (Pm_prev E) dS' (the accumulator, or dSN first), bf16 copy, partial sums of R
-        auto maintain = [&](bool first) {
-            const float factor = pm_prev * ee[krow];
-            pm_prev = pm[krow];
-            float racc = 0.f;
-            uint32_t r[32];
+        // ================= M: MMA issue =================
+        if (lane == 0) {
+            constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T (all K-major)
+            constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
+            constexpr uint32_t idKK = idesc_bf16(128, 64, 0, 0);      // dS'' x V^T, S' x dY^T (all K-major)
+            constexpr uint32_t idMK = idesc_bf16(128, 64, 1, 0);      // dS''^T (MN) x Ks^T (K);  Ks^T (MN) x dP^T (K)
+            constexpr uint32_t idMM = idesc_bf16(128, 64, 1, 1);      // Qs^T (MN) x dP (MN);  dY^T (MN) x P (MN)
+            // descriptors once; K steps and stage changes only add to the 14-bit start-address field
+            const uint32_t sm0 = smem_u32(smem);
+            const uint64_t dqk0 = smem_desc_sw128(sm0, 16, 1024), dqm0 = smem_desc_sw128(sm0, kSlab, 1024);
+            const uint64_t dfk0 = smem_desc_sw128(sm0 + kTile, 16, 1024), dfm0 = smem_desc_sw128(sm0 + kTile, kSlab, 1024);
+            const uint64_t dvk0 = smem_desc_sw128(sm0 + 2 * kTile, 16, 1024);
+            const uint64_t dgk0 = smem_desc_sw128(sm0 + 3 * kTile, 16, 1024), dgm0 = smem_desc_sw128(sm0 + 3 * kTile, kSlab, 1024);
+            const uint64_t dsk = smem_desc_sw128(smem_u32(sbuf), 16, 1024);
+            const uint64_t ddsk = smem_desc_sw128(smem_u32(dsbuf), 16, 1024), ddsm = smem_desc_sw128(smem_u32(dsbuf), kStateSlab, 1024);
+            const uint64_t dpm = smem_desc_sw128(smem_u32(pbuf), kSlab, 1024);
+            const uint64_t ddpk = smem_desc_sw128(smem_u32(dpbuf), 16, 1024), ddpm = smem_desc_sw128(smem_u32(dpbuf), kSlab, 1024);
+            auto kmaj = [](int kk) { return (uint64_t)(((kk >> 2) * kSlab + (kk & 3) * 32) >> 4); };          // [64][128] tile
+            auto kmaj_s = [](int kk) { return (uint64_t)(((kk >> 2) * kStateSlab + (kk & 3) * 32) >> 4); };   // [128][128] tile
+            PT_DECL
+            for (int it = 0; it < NC; ++it) {
+                const int s = it % kStages;
+                const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
+                const uint64_t dqk = dqk0 + so, dqm = dqm0 + so, dfk = dfk0 + so, dfm = dfm0 + so, dvk = dvk0 + so,
+                               dgk = dgk0 + so, dgm = dgm0 + so;
+                mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
+                mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
+                PT_MARK(0)
+                mbar_wait(&ctl->m_done, it & 1, abort_flag);
+                PT_MARK(1)
+                tc_fence_after_sync();
+                // ---- X
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                const int v0 = 64 * half + 32 * part;
-                if (first) {
-                    if (dSN) {
-                        const float4 *src = reinterpret_cast<const float4 *>(dSN + ((size_t)u * kD + krow) * kD + v0);
+                for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
+                    mma_bf16_ss(tmem + kColDS, dqm + (uint64_t)(kk * 128), dgm + (uint64_t)(kk * 128), idDS, 1);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 x = __ldg(src + j);
-                            r[4 * j + 0] = __float_as_uint(x.x); r[4 * j + 1] = __float_as_uint(x.y);
-                            r[4 * j + 2] = __float_as_uint(x.z); r[4 * j + 3] = __float_as_uint(x.w);
-                        }
-                    } else {
+                for (int kk = 0; kk < 8; ++kk)              // A = Qs Ks^T
+                    mma_bf16_ss(tmem + kColA, dqk + kmaj(kk), dfk + kmaj(kk), idA, kk > 0);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) r[j] = 0u;
-                    }
-                } else {
-                    tmem_ld32(tmem + lane_base + kColDS + v0, r);
-                    tmem_wait_ld();
-                }
-#pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
-                tmem_st32(tmem + lane_base + kColDS + v0, r);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t off = half * kStateSlab + slab_chunk_off(krow, 4 * part + j);
-                    const uint4 sw = *reinterpret_cast<const uint4 *>(sbuf + off);
-                    racc = fmaf(__uint_as_float(r[8 * j + 0]), bf16_lo(sw.x), racc);
-                    racc = fmaf(__uint_as_float(r[8 * j + 1]), bf16_hi(sw.x), racc);
-                    racc = fmaf(__uint_as_float(r[8 * j + 2]), bf16_lo(sw.y), racc);
-                    racc = fmaf(__uint_as_float(r[8 * j + 3]), bf16_hi(sw.y), racc);
-                    racc = fmaf(__uint_as_float(r[8 * j + 4]), bf16_lo(sw.z), racc);
-                    racc = fmaf(__uint_as_float(r[8 * j + 5]), bf16_hi(sw.z), racc);
-                    racc = fmaf(__uint_as_float(r[8 * j + 6]), bf16_lo(sw.w), racc);
-                    racc = fmaf(__uint_as_float(r[8 * j + 7]), bf16_hi(sw.w), racc);
-                    *reinterpret_cast<uint4 *>(dsbuf + off) = pack8(r + 8 * j);
-                }
-            }
-            rpart[half * 128 + krow] = racc;
-            tmem_wait_st();
-            tc_fence_before_sync();
-            fence_proxy_async_smem();
-            mbar_arrive(&ctl->g1_ready);
-        };
-
-        mbar_wait(&ctl->full[0], 0, abort_flag);
-        transform_chunk(smem, smem + kTile, tot, pm, ee, min(kC, N - (NC - 1) * kC), tid);
-        worker_sync();
-        mbar_wait(&ctl->sfull, 0, abort_flag);
-        maintain(true);
-        PT_DECL
-
-        for (int it = 0; it < NC; ++it) {
-            const int c = NC - 1 - it;
-            uint8_t *qbuf = smem + (it % kBwdStages) * kBwdStageBytes;
-            uint8_t *fbuf = qbuf + kTile;
-            const int n_valid = min(kC, N - c * kC);
-
-            // tril(A), tril(dA) -> shared memory
-            mbar_wait(&ctl->bar1, it & 1, abort_flag);
-            tc_fence_after_sync();
-            PT_MARK(0)
-            tril_to_slab(tmem + lane_base + kColA2 + 32 * half, pbuf, sub, half, lane);
-            tril_to_slab(tmem + lane_base + kColDA + 32 * half, dpbuf, sub, half, lane);
-            fence_proxy_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&ctl->pd_ready);
-            PT_MARK(1)
-
-            // next chunk's operands while the second MMA group runs
-            if (it + 1 < NC) {
-                const int s1 = (it + 1) % kBwdStages;
-                uint8_t *qn = smem + s1 * kBwdStageBytes;
-                mbar_wait(&ctl->full[s1], ((it + 1) / kBwdStages) & 1, abort_flag);
+                for (int kk = 0; kk < 8; ++kk)              // dA = dY V^T
+                    mma_bf16_ss(tmem + kColDA, dgk + kmaj(kk), dvk + kmaj(kk), idA, kk > 0);
+                mma_commit(&ctl->barX);
                 PT_MARK(2)
-                transform_chunk(qn, qn + kTile, tot, pm, ee, min(kC, N - (c - 1) * kC), tid);
-                worker_sync();
+                // ---- Y1
+                if (it > 0) {
+                    mbar_wait(&ctl->acc_free1, (it - 1) & 1, abort_flag);
+                    tc_fence_after_sync();
+                }
                 PT_MARK(3)
-            }
-
-            mbar_wait(&ctl->bar2, it & 1, abort_flag);
-            tc_fence_after_sync();
-            PT_MARK(4)
-
-            // d_i = dV
-            rows_to_global(tmem + lane_base + kColDV + 64 * half, d_i + ((size_t)u * N + (size_t)c * kC) * kD, sub,
-                           half, lane, n_valid);
-            PT_MARK(5)
-
-            // d_o and d_f: thread (krow, half) owns key dimension krow and local times 32*half .. 32*half+31
-            {
-                const int tb = 32 * half;
-                const size_t gbase = ((size_t)u * N + (size_t)c * kC + tb) * kD + krow;
-                const int kch = (krow & 63) >> 3;
-                const uint32_t kbase = (krow >> 6) * kSlab + tb * 128 + (krow & 7) * 2;
-                uint32_t xo[8];
 #pragma unroll
-                for (int jj = 0; jj < 8; ++jj) xo[jj] = kbase + ((kch ^ jj) << 4);    // (tb + j) & 7 == j & 7
-                float fv[32], m[32];
+                for (int kk = 0; kk < 8; ++kk)              // dKs_inter^T = dS'' V^T
+                    mma_bf16_ss(tmem + kColDKx, ddsk + kmaj_s(kk), dvk + kmaj(kk), idKK, kk > 0);
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    fv[j] = (tb + j < n_valid) ? __bfloat162float(f_gmem[gbase + (size_t)j * kD]) : 1.f;
-                if (half == 0) {
-                    float acc = 1.f;
-#pragma unroll
-                    for (int j = 31; j >= 0; --j) { m[j] = fmaxf(acc, kProdFloor); acc *= fv[j]; }
-                } else {
-                    float acc = 1.f;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) { acc *= fv[j]; m[j] = fmaxf(acc, kProdFloor); }
-                }
-                float a[32], dks[32], ev[32];
-                uint32_t r[32];
-                tmem_ld32(tmem + lane_base + kColDQ + tb, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float qs = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(qbuf + xo[j & 7] + j * 128));
-                    const float x = __uint_as_float(r[j]);
-                    a[j] = qs * x;
-                    const float mi = rcp_fast(m[j]);
-                    const float sq = half == 0 ? mi : m[j];
-                    m[j] = half == 0 ? m[j] : mi;            // from here on m holds exp(b_m - b_s)
-                    if (tb + j < n_valid) d_o[gbase + (size_t)j * kD] = __float2bfloat16_rn(x * sq);
-                }
-                tmem_ld32(tmem + lane_base + kColDKi + tb, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float ks = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(fbuf + xo[j & 7] + j * 128));
-                    const float x = __uint_as_float(r[j]);
-                    a[j] = fmaf(-ks, x, a[j]);
-                    dks[j] = x;
-                    ev[j] = ks;
-                }
-                mbar_arrive(&ctl->f_done);          // last read of this chunk's stage
-                tmem_ld32(tmem + lane_base + kColDKx + tb, r);
-                tmem_wait_ld();
-                float asum = 0.f, esum = 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float x = __uint_as_float(r[j]);
-                    dks[j] = (dks[j] + x) * m[j];
-                    ev[j] *= x;
-                    asum += a[j];
-                    esum += ev[j];
-                }
-                if (half == 1) xa[krow] = asum;       // each written by exactly one of the two threads of a key dim
-                if (half == 0) xe[krow] = esum;
-                const float R = rpart[krow] + rpart[128 + krow];
+                for (int kk = 0; kk < 8; ++kk)              // dV^T = dS''^T Ks^T
+                    mma_bf16_ss(tmem + kColDV, ddsm + (uint64_t)(kk * 128), dfk + kmaj(kk), idMK, kk > 0);
+                mma_commit(&ctl->barY1);
+                PT_MARK(4)
+                // ---- Y2
+                mbar_wait(&ctl->pd_ready, it & 1, abort_flag);
+                mbar_wait(&ctl->sfull, it & 1, abort_flag);
+                PT_MARK(5)
+                if (it > 0) mbar_wait(&ctl->acc_free2, (it - 1) & 1, abort_flag);
                 PT_MARK(6)
-                worker_sync();
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dQs^T = Ks^T dA^T
+                    mma_bf16_ss(tmem + kColDQ, dfm + (uint64_t)(kk * 128), ddpk + (uint64_t)(kk * 2), idMK, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)              //        + S' dY^T
+                    mma_bf16_ss(tmem + kColDQ, dsk + kmaj_s(kk), dgk + kmaj(kk), idKK, 1);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
+                    mma_bf16_ss(tmem + kColDKi, dqm + (uint64_t)(kk * 128), ddpm + (uint64_t)(kk * 128), idMM, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dV^T += dY^T A
+                    mma_bf16_ss(tmem + kColDV, dgm + (uint64_t)(kk * 128), dpm + (uint64_t)(kk * 128), idMM, 1);
+                mma_commit(&ctl->barY2);
                 PT_MARK(7)
-                float pre = (half == 1) ? xe[krow] : 0.f;
-                float suf = (half == 0) ? xa[krow] : 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {        // exclusive prefix sums of e
-                    const float e = ev[j];
-                    ev[j] = pre;
-                    pre += e;
-                }
-#pragma unroll
-                for (int j = 31; j >= 0; --j) {
-                    suf += a[j];
-                    const float dg = R + suf + ev[j];
-                    if (tb + j < n_valid)
-                        d_f[gbase + (size_t)j * kD] =
-                            __float2bfloat16_rn(fmaf(dg, rcp_fast(fmaxf(fv[j], kProdFloor)), -dks[j]));
-                }
             }
-            tc_fence_before_sync();
-            PT_MARK(8)
-
-            if (it + 1 < NC) {
-                mbar_wait(&ctl->sfull, (it + 1) & 1, abort_flag);
-                PT_MARK(9)
-                maintain(false);
-                PT_MARK(10)
-            }
-        }
-        PT_DUMP(status, 0, 12, tid == 0)
-
-        // dS_0 = Diag(Pm of chunk 0) dS'
-        if (dS0) {
-            tc_fence_after_sync();
-            uint32_t r[32];
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                const int v0 = 64 * half + 32 * part;
-                tmem_ld32(tmem + lane_base + kColDS + v0, r);
-                tmem_wait_ld();
-                float4 *dst = reinterpret_cast<float4 *>(dS0 + ((size_t)u * kD + krow) * kD + v0);
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    dst[j] = make_float4(__uint_as_float(r[4 * j + 0]) * pm_prev, __uint_as_float(r[4 * j + 1]) * pm_prev,
-                                         __uint_as_float(r[4 * j + 2]) * pm_prev, __uint_as_float(r[4 * j + 3]) * pm_prev);
-            }
+            PT_DUMP(status, 14, 8, true)
         }
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0 && *abort_flag) report_error(status, HGRN2_ERR_TIMEOUT, 2);
+    if (tid == 0 && *abort_flag) {
+        report_error(status, HGRN2_ERR_TIMEOUT, 2);
+        // loads may still be in flight towards this CTA's shared memory: give them time to land
+        for (int s = 0; s < kStages; ++s) {
+            const int last = ((NC - 1 - s) / kStages) * kStages + s;
+            if (s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
+        }
+        mbar_wait_drain(&ctl->sfull, (NC - 1) & 1, 20000000ull);
+    }
+    __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
@@ -522,9 +532,9 @@ cudaError_t launch_tc_bwd(const SeqArgs &a)
     if (!make_map(&mo, a.o, U, a.N, kC) || !make_map(&mf, a.f, U, a.N, kC) || !make_map(&mi, a.i, U, a.N, kC) ||
         !make_map(&mg, a.dy, U, a.N, kC) || !make_map(&ms, a.states, U * a.NC, kD, kD))
         return cudaErrorInvalidValue;
-    cudaError_t err = cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemBytes);
+    cudaError_t err = cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
-    tc_bwd_kernel<<<(unsigned)U, kThreads, kBwdSmemBytes, a.stream>>>(
+    tc_bwd_kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
         mo, mf, mi, mg, ms, static_cast<const __nv_bfloat16 *>(a.f), a.dSN, static_cast<__nv_bfloat16 *>(a.d_o),
         static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), a.dS0, a.N, a.NC, a.status);
     return cudaGetLastError();
