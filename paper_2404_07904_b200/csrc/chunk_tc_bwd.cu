@@ -23,11 +23,12 @@
 //   T   4 warps: raw o, f tiles -> Qs, Ks in place, one chunk ahead (two TMA stages);
 //   E1  4 warps: rescale the dS accumulator and publish its bf16 copy dS'' (the chain between
 //       chunks), causal masks of A and dA into operand slabs, R;
-//   E3  8 warps: outputs.  d_i from dV^T; d_o and d_f from dQs^T, dKs_intra^T, dKs_inter^T.  A
-//       thread owns (key dim, half of the chunk) and walks its 32 steps outwards from the middle,
-//       carrying the decay product and the running sums; what is still missing then is one constant
-//       per key dimension (R plus the other half's sums), so the almost finished d_f and 1/f are
-//       parked in the TMEM columns just read and completed after the two halves have exchanged sums;
+//   E3  8 warps: d_o and most of d_f from dQs^T, dKs_intra^T, dKs_inter^T.  A thread owns (key dim,
+//       half of the chunk) and walks its 32 steps outwards from the middle, carrying the decay
+//       product and the running sums; what is still missing then is one constant per key dimension
+//       (R plus the two halves' sums), so the almost finished d_f and 1/f are parked in the TMEM
+//       columns just read;
+//   O   4 warps: d_i from dV^T, and d_f completed from the parked values;
 //   L   1 warp: TMA loads (raw tiles, saved S');   M  1 warp: tcgen05.mma issue.
 // Per chunk the tensor pipe runs
 //   X : dS' += Qs^T dY | A | dA            (overlaps the outputs of the previous chunk)
@@ -44,10 +45,10 @@ namespace {
 
 using namespace tc;
 
-constexpr int kTWarps = 4, kE1Warps = 4, kE3Warps = 8;
-constexpr int kE1Threads = kE1Warps * 32, kE3Threads = kE3Warps * 32;
-constexpr int kWarpE1 = kTWarps, kWarpE3 = kWarpE1 + kE1Warps;
-constexpr int kWarpLoad = kWarpE3 + kE3Warps, kWarpMma = kWarpLoad + 1;
+constexpr int kTWarps = 4, kE1Warps = 4, kE3Warps = 8, kOWarps = 4;
+constexpr int kE1Threads = kE1Warps * 32, kE3Threads = kE3Warps * 32, kOThreads = kOWarps * 32;
+constexpr int kWarpE1 = kTWarps, kWarpE3 = kWarpE1 + kE1Warps, kWarpO = kWarpE3 + kE3Warps;
+constexpr int kWarpLoad = kWarpO + kOWarps, kWarpMma = kWarpLoad + 1;
 constexpr int kThreads = (kWarpMma + 1) * 32;
 
 constexpr int kStages = 2;
@@ -75,17 +76,17 @@ struct Ctl {
     uint64_t pd_ready;            // E1 -> M: tril(A), tril(dA) are in shared memory
     uint64_t barY1;               // tcgen05.commit -> E1: dS'' copy no longer read
     uint64_t barY2;               // tcgen05.commit -> E3, L: every product of the chunk complete
-    uint64_t r_ready[2];          // E1 -> E3, L: R of the chunk is in shared memory, S' no longer read by threads
+    uint64_t r_ready[2];          // E1 -> O, L: R of the chunk is in shared memory, S' no longer read by threads
                                   // (two barriers: the slower of the two waiters must not be lapped)
-    uint64_t acc_free1;           // E3 -> M: dKs_inter^T and dV^T have been read out
-    uint64_t acc_free2;           // E3 -> M: dQs^T and dKs_intra^T columns are free again
+    uint64_t acc_free1;           // E3 -> M: dKs_inter^T has been read out
+    uint64_t acc_freeV;           // O -> M: dV^T has been read out
+    uint64_t parked;              // E3 -> O: the parked values and the halves' sums are in place
+    uint64_t acc_free2;           // O -> M: dQs^T and dKs_intra^T columns are free again
     uint32_t tmem_base;
     int abort_flag;
 };
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
-
-__device__ __forceinline__ void e3_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // d_o and the nearly finished d_f of one thread: key dimension k, local times [32 * kUp, 32 * kUp + 32),
 // walked outwards from the middle of the chunk in blocks of eight.  Returns this half's sums of a and e.
@@ -187,7 +188,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->r_ready[0], kE1Threads);
         mbar_init(&ctl->r_ready[1], kE1Threads);
         mbar_init(&ctl->acc_free1, kE3Threads);
-        mbar_init(&ctl->acc_free2, kE3Threads);
+        mbar_init(&ctl->acc_freeV, kOThreads);
+        mbar_init(&ctl->parked, kE3Threads);
+        mbar_init(&ctl->acc_free2, kOThreads);
         ctl->abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
@@ -329,8 +332,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                                          __uint_as_float(r[4 * j + 2]) * pm_prev, __uint_as_float(r[4 * j + 3]) * pm_prev);
             }
         }
-    } else if (warp < kWarpLoad) {
-        // ================= E3: output warps =================
+    } else if (warp < kWarpO) {
+        // ================= E3: d_o and the parked part of d_f =================
         const int half = (warp - kWarpE3) >> 2;                      // half of the chunk: local times [32 * half, +32)
         const uint32_t tl = tmem + lane_base;
         PT_DECL
@@ -342,54 +345,65 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
             PT_MARK(0)
             tc_fence_after_sync();
-
-            // d_i = dV: lane = value dimension, columns = local times of this half
-#pragma unroll 1
-            for (int b = 0; b < 4; ++b) {
-                uint32_t r[8];
-                const int s0 = 32 * half + 8 * b;
-                tmem_ld8(tl + kColDV + s0, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (s0 + j < n_valid) d_i[(row0 + s0 + j) * kD + krow] = __float2bfloat16_rn(__uint_as_float(r[j]));
-            }
-            PT_MARK(1)
-
-            // d_o and the parked part of d_f
             float asum, esum;
             if (half) phase_main<true>(tl, qtile, ktile, krow, f_gmem + row0 * kD + krow, d_o + row0 * kD + krow, n_valid, asum, esum);
             else      phase_main<false>(tl, qtile, ktile, krow, f_gmem + row0 * kD + krow, d_o + row0 * kD + krow, n_valid, asum, esum);
             mbar_arrive(&ctl->stage_read[s]);
+            if (half) xa[krow] = asum; else xe[krow] = esum;
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_free1);
-            if (half) xa[krow] = asum; else xe[krow] = esum;
-            PT_MARK(2)
-            mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
-            e3_sync();
-            PT_MARK(3)
-            const float K = rr[(it & 1) * 128 + krow] + xa[krow] + xe[krow];
+            mbar_arrive(&ctl->parked);
+            PT_MARK(1)
+        }
+        PT_DUMP(status, 9, 2, tid == kWarpE3 * 32)
+    } else if (warp < kWarpLoad) {
+        // ================= O: d_i, and d_f completed from the parked values =================
+        const uint32_t tl = tmem + lane_base;
+        PT_DECL
+        for (int it = 0; it < NC; ++it) {
+            const int c = NC - 1 - it;
+            const int n_valid = min(kC, N - c * kC);
+            const size_t row0 = (size_t)u * N + (size_t)c * kC;
+            mbar_wait(&ctl->barY2, it & 1, abort_flag);
+            PT_MARK(0)
             tc_fence_after_sync();
+            // d_i = dV: lane = value dimension, columns = local times
 #pragma unroll 1
-            for (int b = 0; b < 4; ++b) {
-                uint32_t uu[8], rf[8];
-                const int t0 = 32 * half + 8 * b;
-                tmem_ld8(tl + kColDQ + t0, uu);
-                tmem_ld8(tl + kColDKi + t0, rf);
+            for (int b = 0; b < 8; ++b) {
+                uint32_t r[8];
+                tmem_ld8(tl + kColDV + 8 * b, r);
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
-                    if (t0 + j < n_valid)
-                        d_f[(row0 + t0 + j) * kD + krow] =
+                    if (8 * b + j < n_valid)
+                        d_i[(row0 + 8 * b + j) * kD + krow] = __float2bfloat16_rn(__uint_as_float(r[j]));
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->acc_freeV);
+            PT_MARK(1)
+            mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
+            mbar_wait(&ctl->parked, it & 1, abort_flag);
+            PT_MARK(2)
+            tc_fence_after_sync();
+            const float K = rr[(it & 1) * 128 + krow] + xa[krow] + xe[krow];
+#pragma unroll 1
+            for (int b = 0; b < 8; ++b) {
+                uint32_t uu[8], rf[8];
+                tmem_ld8(tl + kColDQ + 8 * b, uu);
+                tmem_ld8(tl + kColDKi + 8 * b, rf);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (8 * b + j < n_valid)
+                        d_f[(row0 + 8 * b + j) * kD + krow] =
                             __float2bfloat16_rn(fmaf(K, __uint_as_float(rf[j]), __uint_as_float(uu[j])));
             }
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_free2);
-            e3_sync();                                               // xa, xe are rewritten next iteration
-            PT_MARK(4)
+            PT_MARK(3)
         }
-        PT_DUMP(status, 9, 5, tid == kWarpE3 * 32)
+        PT_DUMP(status, 11, 4, tid == kWarpO * 32)
     } else if (warp == kWarpLoad) {
         // ================= L: TMA loads =================
         if (lane == 0) {
@@ -472,6 +486,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 // ---- Y1
                 if (it > 0) {
                     mbar_wait(&ctl->acc_free1, (it - 1) & 1, abort_flag);
+                    mbar_wait(&ctl->acc_freeV, (it - 1) & 1, abort_flag);
                     tc_fence_after_sync();
                 }
                 PT_MARK(3)
@@ -505,7 +520,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mma_commit(&ctl->barY2);
                 PT_MARK(7)
             }
-            PT_DUMP(status, 14, 8, true)
+            PT_DUMP(status, 15, 8, true)
         }
     }
     tc_fence_before_sync();
