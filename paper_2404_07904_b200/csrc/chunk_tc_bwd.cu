@@ -29,7 +29,9 @@
 //       (R plus the two halves' sums), so the almost finished d_f and 1/f are parked in the TMEM
 //       columns just read;
 //   O   4 warps: d_i from dV^T, and d_f completed from the parked values;
-//   L   1 warp: TMA loads (raw tiles, saved S');   M  1 warp: tcgen05.mma issue.
+//   L   1 warp: TMA loads (raw tiles, saved S');
+//   MX, MY1, MY2  1 warp each: tcgen05.mma issue of the three groups below (one lane issuing all 56
+//       products of a chunk is itself a bottleneck: its instruction stream is long and serial).
 // Per chunk the tensor pipe runs
 //   X : dS' += Qs^T dY | A | dA            (overlaps the outputs of the previous chunk)
 //   Y1: dKs_inter^T | dV^T = dS''^T Ks^T   (needs the previous chunk's dKs_inter^T, dV^T read out)
@@ -48,8 +50,9 @@ using namespace tc;
 constexpr int kTWarps = 4, kE1Warps = 4, kE3Warps = 8, kOWarps = 4;
 constexpr int kE1Threads = kE1Warps * 32, kE3Threads = kE3Warps * 32, kOThreads = kOWarps * 32;
 constexpr int kWarpE1 = kTWarps, kWarpE3 = kWarpE1 + kE1Warps, kWarpO = kWarpE3 + kE3Warps;
-constexpr int kWarpLoad = kWarpO + kOWarps, kWarpMma = kWarpLoad + 1;
-constexpr int kThreads = (kWarpMma + 1) * 32;
+constexpr int kWarpLoad = kWarpO + kOWarps, kWarpMmaX = kWarpLoad + 1, kWarpMmaY1 = kWarpLoad + 2,
+              kWarpMmaY2 = kWarpLoad + 3;
+constexpr int kThreads = (kWarpMmaY2 + 1) * 32;
 
 constexpr int kStages = 2;
 constexpr uint32_t kStageBytes = 4 * kTile;                       // q, f, v, dy
@@ -57,12 +60,11 @@ constexpr uint32_t kOffS = kStages * kStageBytes;                 // S' (bf16, f
 constexpr uint32_t kOffDS = kOffS + kStateTile;                   // bf16 copy of dS''
 constexpr uint32_t kOffP = kOffDS + kStateTile;                   // bf16 tril(A)
 constexpr uint32_t kOffDP = kOffP + kSlab;                        // bf16 tril(dA)
-constexpr uint32_t kOffPm = kOffDP + kSlab;                       // float pm[4][128]
-constexpr uint32_t kOffE = kOffPm + 4 * 128 * 4;                  // float ee[4][128]
-constexpr uint32_t kOffR = kOffE + 4 * 128 * 4;                   // float rr[2][128]
+constexpr uint32_t kOffF = kOffDP + kSlab;                        // uint32 fscr[16][256]: f strips of the E3 threads
+constexpr uint32_t kOffR = kOffF + 16 * 256 * 4;                  // float rr[2][128]
 constexpr uint32_t kOffX = kOffR + 2 * 128 * 4;                   // float xa[128], xe[128]
 constexpr uint32_t kOffCtl = kOffX + 2 * 128 * 4;
-constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024;
+constexpr uint32_t kSmemBytes = kOffCtl + 256;                    // no slack: the base must be 1024-byte aligned
 
 constexpr uint32_t kColDS = 0, kColA = 128, kColDA = 192, kColDQ = 256, kColDKi = 320, kColDKx = 384, kColDV = 448;
 
@@ -88,12 +90,36 @@ struct Ctl {
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
+// f of the 32 rows [t_first, t_first + 32) of one key dimension as raw bf16 bits, two rows per word, into
+// the thread's column of the scratch; rows at or beyond n_valid read as 1.  f_g points at (row 0 of the chunk,
+// column k).
+__device__ __forceinline__ void load_f_strip(const __nv_bfloat16 *f_g, int t_first, int n_valid, uint32_t *fs)
+{
+    const unsigned short *fp = reinterpret_cast<const unsigned short *>(f_g);
+#pragma unroll 1
+    for (int h = 0; h < 2; ++h) {
+        uint32_t w[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int t = t_first + 16 * h + 2 * i;
+            const uint32_t lo = (t < n_valid) ? fp[(size_t)t * kD] : 0x3F80u;
+            const uint32_t hi = (t + 1 < n_valid) ? fp[(size_t)(t + 1) * kD] : 0x3F80u;
+            w[i] = lo | (hi << 16);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) fs[(8 * h + i) * 256] = w[i];
+    }
+}
+
 // d_o and the nearly finished d_f of one thread: key dimension k, local times [32 * kUp, 32 * kUp + 32),
 // walked outwards from the middle of the chunk in blocks of eight.  Returns this half's sums of a and e.
-// f_g / do_g point at element (row 0 of the chunk, column k) of f and d_o in global memory.
+// do_g points at element (row 0 of the chunk, column k) of d_o in global memory.  fs points at this thread's
+// column of the f scratch (word i, stride 256 words, holds f of its rows 2i and 2i + 1 in row order), filled by
+// the thread itself while it waited for the products: narrow global loads inside the loop would put a round
+// trip to L2 on every block's dependent chain.
 template <bool kUp>
 __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qtile, const uint8_t *ktile, int k,
-                                           const __nv_bfloat16 *f_g, __nv_bfloat16 *do_g, int n_valid, float &asum,
+                                           const uint32_t *fs, __nv_bfloat16 *do_g, int n_valid, float &asum,
                                            float &esum)
 {
     const int kch = (k & 63) >> 3;
@@ -108,11 +134,17 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qt
         tmem_ld8(tmem_lane + kColDKi + t0, y);
         tmem_ld8(tmem_lane + kColDKx + t0, z);
         float fv[8], qs[8], ks[8];
+        const uint32_t *fb = fs + (kUp ? 4 * b : 12 - 4 * b) * 256;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t fw = fb[j * 256];
+            fv[2 * j] = bf16_lo(fw);
+            fv[2 * j + 1] = bf16_hi(fw);
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int t = t0 + j;
             const uint32_t off = kbase + t * 128 + ((kch ^ j) << 4);
-            fv[j] = (t < n_valid) ? __bfloat162float(f_g[(size_t)t * kD]) : 1.f;
             qs[j] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(qtile + off));
             ks[j] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(ktile + off));
         }
@@ -152,18 +184,21 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qt
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
-              const __grid_constant__ CUtensorMap map_saved, const __nv_bfloat16 *__restrict__ f_gmem,
+              const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ totals,
+              const __nv_bfloat16 *__restrict__ f_gmem,
               const float *__restrict__ dSN, __nv_bfloat16 *__restrict__ d_o, __nv_bfloat16 *__restrict__ d_f,
               __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N, int NC, StatusBlock *status)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
+    if (smem_u32(smem) & 1023u) {          // every byte is spoken for: the swizzled tiles need the base aligned
+        if (threadIdx.x == 0) report_error(status, HGRN2_ERR_CUDA, 3);
+        return;
+    }
     uint8_t *sbuf = smem + kOffS;
     uint8_t *dsbuf = smem + kOffDS;
     uint8_t *pbuf = smem + kOffP;
     uint8_t *dpbuf = smem + kOffDP;
-    float *pm = reinterpret_cast<float *>(smem + kOffPm);
-    float *ee = reinterpret_cast<float *>(smem + kOffE);
+    uint32_t *fscr = reinterpret_cast<uint32_t *>(smem + kOffF);
     float *rr = reinterpret_cast<float *>(smem + kOffR);
     float *xa = reinterpret_cast<float *>(smem + kOffX);
     float *xe = xa + 128;
@@ -218,10 +253,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
             PT_MARK(0)
             const int n_valid = N - c * kC;
+            // Pm and E of the chunk are not kept: the backward takes them from what the forward saved
             if (n_valid >= kC) {
-                transform_stream<true>(qbuf, qbuf + kTile, pm + (it & 3) * 128, ee + (it & 3) * 128, kC, tid);
+                transform_stream<true>(qbuf, qbuf + kTile, nullptr, nullptr, nullptr, nullptr, kC, tid);
             } else {
-                transform_stream<false>(qbuf, qbuf + kTile, pm + (it & 3) * 128, ee + (it & 3) * 128, n_valid, tid);
+                transform_stream<false>(qbuf, qbuf + kTile, nullptr, nullptr, nullptr, nullptr, n_valid, tid);
             }
             fence_proxy_async_smem();
             mbar_arrive(&ctl->t_done[s]);
@@ -230,14 +266,20 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         PT_DUMP(status, 0, 2, tid == 0)
     } else if (warp < kWarpE3) {
         // ================= E1: state-gradient warps =================
+        // Pm, E of every chunk come from the forward's saved totals, so this chain does not wait for T
         float pm_prev = 1.f;
+        const float *tot_u = totals + (size_t)u * NC * 2 * kD + krow;
+        float pm_c = __ldg(tot_u + (size_t)(NC - 1) * 2 * kD), ee_c = __ldg(tot_u + (size_t)(NC - 1) * 2 * kD + kD);
         PT_DECL
         for (int it = 0; it < NC; ++it) {
             // ---- dS'' = (Pm_prev E) dS' (the accumulator, or dSN first) -> TMEM, bf16 copy -> dsbuf
-            mbar_wait(&ctl->t_done[it % kStages], (it / kStages) & 1, abort_flag);
             PT_MARK(0)
-            const float factor = pm_prev * ee[(it & 3) * 128 + krow];
-            pm_prev = pm[(it & 3) * 128 + krow];
+            const float factor = pm_prev * ee_c;
+            pm_prev = pm_c;
+            if (it + 1 < NC) {
+                pm_c = __ldg(tot_u + (size_t)(NC - 2 - it) * 2 * kD);
+                ee_c = __ldg(tot_u + (size_t)(NC - 2 - it) * 2 * kD + kD);
+            }
             if (it > 0) {
                 mbar_wait(&ctl->barY1, (it - 1) & 1, abort_flag);    // dS' update done, dsbuf no longer read
                 tc_fence_after_sync();
@@ -279,6 +321,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
             // ---- tril(A), tril(dA) -> operand slabs
             mbar_wait(&ctl->barX, it & 1, abort_flag);
+            if (it > 0) mbar_wait(&ctl->barY2, (it - 1) & 1, abort_flag);   // the previous chunk's products have read P, dP
             PT_MARK(3)
             tc_fence_after_sync();
 #pragma unroll 1
@@ -342,12 +385,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int n_valid = min(kC, N - c * kC);
             const uint8_t *qtile = smem + s * kStageBytes, *ktile = qtile + kTile;
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
+            uint32_t *fs = fscr + (tid - kWarpE3 * 32);
+            load_f_strip(f_gmem + row0 * kD + krow, 32 * half, n_valid, fs);
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
             PT_MARK(0)
             tc_fence_after_sync();
             float asum, esum;
-            if (half) phase_main<true>(tl, qtile, ktile, krow, f_gmem + row0 * kD + krow, d_o + row0 * kD + krow, n_valid, asum, esum);
-            else      phase_main<false>(tl, qtile, ktile, krow, f_gmem + row0 * kD + krow, d_o + row0 * kD + krow, n_valid, asum, esum);
+            if (half) phase_main<true>(tl, qtile, ktile, krow, fs, d_o + row0 * kD + krow, n_valid, asum, esum);
+            else      phase_main<false>(tl, qtile, ktile, krow, fs, d_o + row0 * kD + krow, n_valid, asum, esum);
             mbar_arrive(&ctl->stage_read[s]);
             if (half) xa[krow] = asum; else xe[krow] = esum;
             tmem_wait_st();
@@ -439,39 +484,38 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 }
             }
         }
-    } else {
-        // ================= M: MMA issue =================
-        if (lane == 0) {
-            constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T (all K-major)
-            constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
-            constexpr uint32_t idKK = idesc_bf16(128, 64, 0, 0);      // dS'' x V^T, S' x dY^T (all K-major)
-            constexpr uint32_t idMK = idesc_bf16(128, 64, 1, 0);      // dS''^T (MN) x Ks^T (K);  Ks^T (MN) x dP^T (K)
-            constexpr uint32_t idMM = idesc_bf16(128, 64, 1, 1);      // Qs^T (MN) x dP (MN);  dY^T (MN) x P (MN)
-            // descriptors once; K steps and stage changes only add to the 14-bit start-address field
-            const uint32_t sm0 = smem_u32(smem);
-            const uint64_t dqk0 = smem_desc_sw128(sm0, 16, 1024), dqm0 = smem_desc_sw128(sm0, kSlab, 1024);
-            const uint64_t dfk0 = smem_desc_sw128(sm0 + kTile, 16, 1024), dfm0 = smem_desc_sw128(sm0 + kTile, kSlab, 1024);
-            const uint64_t dvk0 = smem_desc_sw128(sm0 + 2 * kTile, 16, 1024);
-            const uint64_t dgk0 = smem_desc_sw128(sm0 + 3 * kTile, 16, 1024), dgm0 = smem_desc_sw128(sm0 + 3 * kTile, kSlab, 1024);
-            const uint64_t dsk = smem_desc_sw128(smem_u32(sbuf), 16, 1024);
-            const uint64_t ddsk = smem_desc_sw128(smem_u32(dsbuf), 16, 1024), ddsm = smem_desc_sw128(smem_u32(dsbuf), kStateSlab, 1024);
-            const uint64_t dpm = smem_desc_sw128(smem_u32(pbuf), kSlab, 1024);
-            const uint64_t ddpk = smem_desc_sw128(smem_u32(dpbuf), 16, 1024), ddpm = smem_desc_sw128(smem_u32(dpbuf), kSlab, 1024);
-            auto kmaj = [](int kk) { return (uint64_t)(((kk >> 2) * kSlab + (kk & 3) * 32) >> 4); };          // [64][128] tile
-            auto kmaj_s = [](int kk) { return (uint64_t)(((kk >> 2) * kStateSlab + (kk & 3) * 32) >> 4); };   // [128][128] tile
-            PT_DECL
+    } else if (lane == 0) {
+        // ================= MX, MY1, MY2: MMA issue =================
+        constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T (all K-major)
+        constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
+        constexpr uint32_t idKK = idesc_bf16(128, 64, 0, 0);      // dS'' x V^T, S' x dY^T (all K-major)
+        constexpr uint32_t idMK = idesc_bf16(128, 64, 1, 0);      // dS''^T (MN) x Ks^T (K);  Ks^T (MN) x dP^T (K)
+        constexpr uint32_t idMM = idesc_bf16(128, 64, 1, 1);      // Qs^T (MN) x dP (MN);  dY^T (MN) x P (MN)
+        // descriptors once; K steps and stage changes only add to the 14-bit start-address field
+        const uint32_t sm0 = smem_u32(smem);
+        const uint64_t dqk0 = smem_desc_sw128(sm0, 16, 1024), dqm0 = smem_desc_sw128(sm0, kSlab, 1024);
+        const uint64_t dfk0 = smem_desc_sw128(sm0 + kTile, 16, 1024), dfm0 = smem_desc_sw128(sm0 + kTile, kSlab, 1024);
+        const uint64_t dvk0 = smem_desc_sw128(sm0 + 2 * kTile, 16, 1024);
+        const uint64_t dgk0 = smem_desc_sw128(sm0 + 3 * kTile, 16, 1024), dgm0 = smem_desc_sw128(sm0 + 3 * kTile, kSlab, 1024);
+        const uint64_t dsk = smem_desc_sw128(smem_u32(sbuf), 16, 1024);
+        const uint64_t ddsk = smem_desc_sw128(smem_u32(dsbuf), 16, 1024), ddsm = smem_desc_sw128(smem_u32(dsbuf), kStateSlab, 1024);
+        const uint64_t dpm = smem_desc_sw128(smem_u32(pbuf), kSlab, 1024);
+        const uint64_t ddpk = smem_desc_sw128(smem_u32(dpbuf), 16, 1024), ddpm = smem_desc_sw128(smem_u32(dpbuf), kSlab, 1024);
+        auto kmaj = [](int kk) { return (uint64_t)(((kk >> 2) * kSlab + (kk & 3) * 32) >> 4); };          // [64][128] tile
+        auto kmaj_s = [](int kk) { return (uint64_t)(((kk >> 2) * kStateSlab + (kk & 3) * 32) >> 4); };   // [128][128] tile
+        PT_DECL
+        if (warp == kWarpMmaX) {
             for (int it = 0; it < NC; ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
-                const uint64_t dqk = dqk0 + so, dqm = dqm0 + so, dfk = dfk0 + so, dfm = dfm0 + so, dvk = dvk0 + so,
-                               dgk = dgk0 + so, dgm = dgm0 + so;
+                const uint64_t dqk = dqk0 + so, dqm = dqm0 + so, dfk = dfk0 + so, dvk = dvk0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
                 mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
                 PT_MARK(0)
-                mbar_wait(&ctl->m_done, it & 1, abort_flag);
+                mbar_wait(&ctl->m_done, it & 1, abort_flag);          // dS'' in TMEM
+                if (it > 0) mbar_wait(&ctl->pd_ready, (it - 1) & 1, abort_flag);   // A, dA of the previous chunk read out
                 PT_MARK(1)
                 tc_fence_after_sync();
-                // ---- X
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
                     mma_bf16_ss(tmem + kColDS, dqm + (uint64_t)(kk * 128), dgm + (uint64_t)(kk * 128), idDS, 1);
@@ -483,13 +527,23 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     mma_bf16_ss(tmem + kColDA, dgk + kmaj(kk), dvk + kmaj(kk), idA, kk > 0);
                 mma_commit(&ctl->barX);
                 PT_MARK(2)
-                // ---- Y1
+            }
+            PT_DUMP(status, 15, 3, true)
+        } else if (warp == kWarpMmaY1) {
+            for (int it = 0; it < NC; ++it) {
+                const int s = it % kStages;
+                const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
+                const uint64_t dfk = dfk0 + so, dvk = dvk0 + so;
+                mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
+                mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
+                mbar_wait(&ctl->m_done, it & 1, abort_flag);          // bf16 dS'' in shared memory
+                PT_MARK(0)
                 if (it > 0) {
                     mbar_wait(&ctl->acc_free1, (it - 1) & 1, abort_flag);
                     mbar_wait(&ctl->acc_freeV, (it - 1) & 1, abort_flag);
-                    tc_fence_after_sync();
                 }
-                PT_MARK(3)
+                PT_MARK(1)
+                tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)              // dKs_inter^T = dS'' V^T
                     mma_bf16_ss(tmem + kColDKx, ddsk + kmaj_s(kk), dvk + kmaj(kk), idKK, kk > 0);
@@ -497,13 +551,20 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 for (int kk = 0; kk < 8; ++kk)              // dV^T = dS''^T Ks^T
                     mma_bf16_ss(tmem + kColDV, ddsm + (uint64_t)(kk * 128), dfk + kmaj(kk), idMK, kk > 0);
                 mma_commit(&ctl->barY1);
-                PT_MARK(4)
-                // ---- Y2
-                mbar_wait(&ctl->pd_ready, it & 1, abort_flag);
+                PT_MARK(2)
+            }
+            PT_DUMP(status, 18, 3, true)
+        } else {
+            for (int it = 0; it < NC; ++it) {
+                const int s = it % kStages;
+                const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
+                const uint64_t dqm = dqm0 + so, dfm = dfm0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
+                mbar_wait(&ctl->pd_ready, it & 1, abort_flag);        // tril(A), tril(dA); implies X and T of the chunk
                 mbar_wait(&ctl->sfull, it & 1, abort_flag);
-                PT_MARK(5)
+                PT_MARK(0)
+                mbar_wait(&ctl->barY1, it & 1, abort_flag);           // dV^T += ... must follow dV^T = ...
                 if (it > 0) mbar_wait(&ctl->acc_free2, (it - 1) & 1, abort_flag);
-                PT_MARK(6)
+                PT_MARK(1)
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dQs^T = Ks^T dA^T
@@ -518,9 +579,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 for (int kk = 0; kk < 4; ++kk)              // dV^T += dY^T A
                     mma_bf16_ss(tmem + kColDV, dgm + (uint64_t)(kk * 128), dpm + (uint64_t)(kk * 128), idMM, 1);
                 mma_commit(&ctl->barY2);
-                PT_MARK(7)
+                PT_MARK(2)
             }
-            PT_DUMP(status, 15, 8, true)
+            PT_DUMP(status, 21, 3, true)
         }
     }
     tc_fence_before_sync();
@@ -550,7 +611,9 @@ cudaError_t launch_tc_bwd(const SeqArgs &a)
     cudaError_t err = cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     tc_bwd_kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
-        mo, mf, mi, mg, ms, static_cast<const __nv_bfloat16 *>(a.f), a.dSN, static_cast<__nv_bfloat16 *>(a.d_o),
+        mo, mf, mi, mg, ms,
+        reinterpret_cast<const float *>(reinterpret_cast<const char *>(a.states) + U * a.NC * kSavedStateBytes),
+        static_cast<const __nv_bfloat16 *>(a.f), a.dSN, static_cast<__nv_bfloat16 *>(a.d_o),
         static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), a.dS0, a.N, a.NC, a.status);
     return cudaGetLastError();
 }

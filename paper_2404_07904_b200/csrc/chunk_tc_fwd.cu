@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
               const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
-              int want_y, int want_saved, int N, int NC, StatusBlock *status)
+              float *__restrict__ totals, int want_y, int want_saved, int N, int NC, StatusBlock *status)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -132,10 +132,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
             PT_MARK(0)
             const int n_valid = N - c * kC;
+            float *tg = totals ? totals + ((size_t)u * NC + c) * 2 * kD : nullptr;     // Pm, E of the chunk for the backward
             if (n_valid >= kC) {
-                transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, kC, tt);
+                transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
+                                       kC, tt);
             } else {
-                transform_stream<false>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, n_valid, tt);
+                transform_stream<false>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
+                                        n_valid, tt);
             }
             fence_proxy_async_smem();
             mbar_arrive(&ctl->t_done[s]);
@@ -408,7 +411,7 @@ bool tc_chunk_supported(int C) { return C == kC; }
 size_t tc_saved_bytes(const hgrn2_desc *d, int C)
 {
     const size_t NC = ((size_t)d->N + C - 1) / C;
-    return (size_t)d->B * d->H * NC * kD * kD * sizeof(__nv_bfloat16);
+    return (size_t)d->B * d->H * NC * (kSavedStateBytes + kSavedTotalsBytes);
 }
 
 cudaError_t launch_tc_fwd(const SeqArgs &a)
@@ -425,7 +428,9 @@ cudaError_t launch_tc_fwd(const SeqArgs &a)
         return cudaErrorInvalidValue;
     cudaError_t err = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
-    tc_fwd_kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, a.S0, a.SN, a.y != nullptr,
+    float *totals = a.states ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes)
+                             : nullptr;
+    tc_fwd_kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, a.S0, a.SN, totals, a.y != nullptr,
                                                                    a.states != nullptr, a.N, a.NC, a.status);
     return cudaGetLastError();
 }

@@ -33,6 +33,10 @@ constexpr uint32_t kStateTile = 2 * kStateSlab;
 constexpr float kProdFloor = 7.888609052210118e-31f;   // 2^-100
 constexpr uint32_t kTmemCols = 512;
 constexpr int kTransformThreads = 128;          // threads that run transform_stream together
+// Saved-for-backward buffer of the tensor-core path, per (unit, chunk): the bf16 state S' in the mid
+// frame ([128][128]), then, after all states, the decay totals Pm[128], E[128] (float) of every chunk.
+constexpr size_t kSavedStateBytes = (size_t)kD * kD * 2;
+constexpr size_t kSavedTotalsBytes = 2 * kD * sizeof(float);
 
 // Optional per-role cycle counters of CTA 0 (development aid; compiled out unless HGRN2_PHASE_TIMING
 // is defined).  Totals land in the padding words of the status block.
@@ -70,10 +74,12 @@ __device__ __forceinline__ uint4 pack8(const uint32_t *r)
 // handled in batches of eight, and the loads of the next batch are issued before the stores of the
 // current one (the tiles are rewritten in place, so the compiler would otherwise serialise every
 // load behind the previous row's stores).  Pm (product over rows 0..31) and E (product over rows
-// 32..63) of the chunk are left in pm[128] and ee[128].  Rows at or beyond n_valid are the neutral
-// token f = 1, o = 0.
+// 32..63) of the chunk are left in pm[128] and ee[128] (shared memory) and / or pm_g[128], ee_g[128]
+// (global memory); either pair may be null.  Rows at or beyond n_valid are the neutral token
+// f = 1, o = 0.
 template <bool kFull, bool kUp>
-__device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, float *tot, int n_valid, int p)
+__device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, float *tot, float *tot_g, int n_valid,
+                                               int p)
 {
     const int col = 2 * p;
     const int jch = (col & 63) >> 3;
@@ -120,15 +126,17 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
             *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0) * sk0, (1.f - f1) * sk1);
         }
     }
-    *reinterpret_cast<float2 *>(tot + col) = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
+    const float2 t2 = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
+    if (tot) *reinterpret_cast<float2 *>(tot + col) = t2;
+    if (tot_g) *reinterpret_cast<float2 *>(tot_g + col) = t2;
 }
 
 template <bool kFull>
-__device__ __forceinline__ void transform_stream(uint8_t *qbuf, uint8_t *fbuf, float *pm, float *ee, int n_valid,
-                                                 int tid)
+__device__ __forceinline__ void transform_stream(uint8_t *qbuf, uint8_t *fbuf, float *pm, float *ee, float *pm_g,
+                                                 float *ee_g, int n_valid, int tid)
 {
-    if (tid >> 6) transform_half<kFull, true>(qbuf, fbuf, ee, n_valid, tid & 63);
-    else          transform_half<kFull, false>(qbuf, fbuf, pm, n_valid, tid & 63);
+    if (tid >> 6) transform_half<kFull, true>(qbuf, fbuf, ee, ee_g, n_valid, tid & 63);
+    else          transform_half<kFull, false>(qbuf, fbuf, pm, pm_g, n_valid, tid & 63);
 }
 
 // Causal mask + bf16 of 32 columns (32 * half ...) of one 64 x 64 fp32 accumulator in the M = 64

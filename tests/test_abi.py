@@ -60,7 +60,7 @@ def test_bf16_128_goes_to_tensor_cores_unless_forced(lib):
     assert binding.path_of(forced) == "alu"
     assert binding.path_of(d) == "tcgen05"
     assert binding.chunk_of(d) == 64
-    assert binding.saved_bytes(d) == 8 * 16 * 32 * 128 * 128 * 2          # bf16 chunk-start states
+    assert binding.saved_bytes(d) == 8 * 16 * 32 * (128 * 128 * 2 + 2 * 128 * 4)   # per chunk: bf16 state + decay totals
     assert binding.workspace_bytes(binding.make_desc(8, 16, 2048, 128, 128, binding.HGRN2_BF16, chunk=32)) == 0
     assert binding.path_of(binding.make_desc(1, 1, 64, 128, 64, binding.HGRN2_BF16)) == "alu"
     assert binding.path_of(binding.make_desc(1, 1, 64, 128, 128, binding.HGRN2_F32)) == "alu"
