@@ -33,8 +33,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (None until a capture of that kernel exists).
-NCU_TRAFFIC_BYTES = {"fwd": None, "bwd": None, "step": None}
+# profiles/ (captured on the same workloads the bench times: lm_2048 and the full decode batch).
+NCU_TRAFFIC_BYTES = {"fwd": 201.40e6 + 155.01e6, "bwd": 406.98e6 + 172.10e6, "step": 271.60e6 + 212.48e6}
 
 
 def load_peaks():
@@ -87,7 +87,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -376,12 +376,13 @@ def run_cuda(args):
     from oracle import ref
     ref.build()
     cores = ref.num_threads()
-    n_units = max(1, min(cores, w.B * w.H))
-    reps = 2
-    cpu_value, cpu_dt, cores = time_oracle(w, reps, 1, n_units)
+    n_units = w.B * w.H                       # the whole workload per repetition
+    _, probe_dt, cores = time_oracle(w, 1, 0, n_units)
+    reps = int(min(12, max(2, round(12.0 / max(probe_dt, 1e-3)))))      # about 12 s of CPU work
+    cpu_value, cpu_dt, cores = time_oracle(w, reps, 0, n_units)
     cpu_baseline = {"value": cpu_value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                    "sample": f"{n_units} of {w.B * w.H} (batch, head) units of lm_2048 (N={w.N}), fwd+bwd in fp64, "
-                              f"{reps} timed repetitions of {cpu_dt:.2f} s, scaled by tokens"}
+                    "sample": f"all {n_units} (batch, head) units of lm_2048 (N={w.N}), fwd+bwd in fp64, "
+                              f"{reps} timed repetitions of {cpu_dt:.2f} s after one untimed"}
 
     line = {
         "metric": "HGRN2 layer fwd+bwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
@@ -404,7 +405,7 @@ def run_cuda(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--only", default="all", choices=["all", "train", "decode"],

@@ -74,7 +74,8 @@ typedef struct hgrn2_desc {
 } hgrn2_desc;
 
 /* Bytes of the `saved` buffer that hgrn2_fwd fills for hgrn2_bwd: the state at the
- * start of every chunk (derived from Eq. 3 by unrolling C steps).  0 on a bad desc. */
+ * start of every chunk (derived from Eq. 3 by unrolling C steps) and, on the tensor-core
+ * path, the two per-chunk decay totals of every key dimension.  0 on a bad desc. */
 size_t hgrn2_saved_bytes(const hgrn2_desc *desc);
 
 /* Bytes of the workspace `ws` every call takes: a 256-byte status block followed by
@@ -129,7 +130,7 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
  *               status word of the call is copied there on the stream, for hgrn2_poll.
  * Limits and caveats
  *   - hgrn2_workspace_bytes(desc) - 256 must not exceed HGRN2_STATIC_SCRATCH_BYTES (bf16 d = 128:
- *     B*H*ceil(N/64) <= 1024 chunk states); larger problems return HGRN2_ERR_WORKSPACE and nothing
+ *     B*H*ceil(N/64) <= 992 chunks of 33 KB each); larger problems return HGRN2_ERR_WORKSPACE and nothing
  *     is launched.  Use hgrn2_bwd with a caller-owned workspace for those.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in
  *     it.  Each call clears the status block and overwrites every state it later reads, so stale
