@@ -122,8 +122,11 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
             if (!kUp) { a0 *= f0; a1 *= f1; }
             const float sq0 = kUp ? m0 : i0, sq1 = kUp ? m1 : i1;
             const float sk0 = kUp ? i0 : m0, sk1 = kUp ? i1 : m1;
-            *reinterpret_cast<uint32_t *>(qbuf + off) = pack_bf16(bf16_lo(qw[j]) * sq0, bf16_hi(qw[j]) * sq1);
-            *reinterpret_cast<uint32_t *>(fbuf + off) = pack_bf16((1.f - f0) * sk0, (1.f - f1) * sk1);
+            // packed bf16 arithmetic: the scale factors are rounded to bf16 first, then one bf16x2 multiply
+            // (resp. fused multiply-add for k = 1 - f) produces the operand pair
+            const uint32_t sqp = pack_bf16(sq0, sq1), skp = pack_bf16(sk0, sk1);
+            *reinterpret_cast<uint32_t *>(qbuf + off) = mul_bf16x2(qw[j], sqp);
+            *reinterpret_cast<uint32_t *>(fbuf + off) = fma_bf16x2(fw[j], skp ^ 0x80008000u, skp);
         }
     }
     const float2 t2 = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
