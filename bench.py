@@ -34,7 +34,7 @@ NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (captured on the same workloads the bench times: lm_2048 and the full decode batch).
-NCU_TRAFFIC_BYTES = {"fwd": 201.40e6 + 155.01e6, "bwd": 406.98e6 + 172.10e6, "step": 271.60e6 + 212.48e6}
+NCU_TRAFFIC_BYTES = {"fwd": 201.41e6 + 154.41e6, "bwd": 406.93e6 + 170.11e6, "step": 271.60e6 + 212.48e6}
 
 
 def load_peaks():
@@ -231,6 +231,54 @@ def run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks,
     return decode
 
 
+def run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf):
+    """fwd + bwd on the long-context and the larger-layer workloads (reported, not the headline): same recipe,
+    same calls, 10 timed steps each after 3 warm-ups.  Rank 0 only."""
+    import torch
+    out = []
+    if rank != 0:
+        return out
+    for name, gamma in (("long_16k", None), ("lm_2560", 0.9)):
+        w = W.CONFIGS[name]
+        inp = W.make_inputs(w, gamma=gamma)
+        t = {k: (None if v is None else torch.from_numpy(v).to(dev)) for k, v in inp.items()}
+        o, f, i, dy = (t[k].to(bf) for k in ("o", "f", "i", "dy"))
+        S0, dSN = t["S0"], t["dSN"]
+        del inp, t
+        desc = binding.make_desc(w.B, w.H, w.N, w.dk, w.dv, binding.HGRN2_BF16, w.chunk, 0)
+        saved = binding.alloc_saved(desc, dev)
+        ws = binding.alloc_workspace(desc, dev)
+        y = torch.empty_like(i); d_o = torch.empty_like(o); d_f = torch.empty_like(o); d_i = torch.empty_like(i)
+        SN = torch.empty((w.B, w.H, w.dk, w.dv), dtype=torch.float32, device=dev) if w.has_S0 else None
+        dS0 = torch.empty_like(SN) if SN is not None else None
+
+        def fwd():
+            binding.hgrn2_fwd(o, f, i, S0, y=y, SN=SN, saved=saved, ws=ws, want_final_state=SN is not None)
+
+        def bwd():
+            binding.hgrn2_bwd(o, f, i, S0, dy, dSN, saved, d_o=d_o, d_f=d_f, d_i=d_i, dS0=dS0, ws=ws,
+                              want_dS0=dS0 is not None)
+
+        def step():
+            fwd(); bwd()
+
+        for _ in range(3):
+            step()
+        n = 10
+        ms = timed(step, n) / n
+        ms_f = timed(fwd, n) / n
+        ms_b = timed(bwd, n) / n
+        ab = train_bytes(w)
+        state_bytes = 4 * w.B * w.H * w.dk * w.dv * 4 if w.has_S0 else 0
+        t_hbm = (ab["fwd"] + ab["bwd"] + state_bytes) / (peaks["hbm_gbs"] * 1e9)
+        out.append({"workload": name, "B": w.B, "H": w.H, "N": w.N, "gamma": w.gamma if gamma is None else gamma,
+                    "units": w.B * w.H, "ms_per_step": ms, "fwd_ms": ms_f, "bwd_ms": ms_b,
+                    "tokens_per_s": w.tokens / (ms * 1e-3), "frac_of_hbm_roofline": t_hbm * 1e3 / ms})
+        del o, f, i, dy, saved, ws, y, d_o, d_f, d_i
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -364,6 +412,7 @@ def run_cuda(args):
             print(json.dumps({"only": "train", "ms_per_step": ms_step, "kernels": kern}), flush=True)
         return 0
     decode = run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks, peak_kind, bf)
+    others = run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf) if not args.skip_others else []
 
     if world > 1:
         dist.barrier()
@@ -389,7 +438,7 @@ def run_cuda(args):
         "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": workload_config(w, path),
-        "roofline": roofline, "cpu_baseline": cpu_baseline, "decode": decode,
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "decode": decode, "other_workloads": others,
         "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in host.values()),
                 "d2h_bytes_per_step": sum(v.numel() * v.element_size() for v in host_out.values())},
@@ -411,6 +460,7 @@ def main():
     ap.add_argument("--only", default="all", choices=["all", "train", "decode"],
                     help="restrict the run to one part (for profiling); the JSON line is printed for 'all' only")
     ap.add_argument("--decode-steps", type=int, default=0, help="decode calls to time (0 = the workload's 512)")
+    ap.add_argument("--skip-others", action="store_true", help="do not time the long-context and larger-layer workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -241,11 +241,6 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn_major, 
            (static_cast<uint32_t>(M >> 4) << 24);
 }
 
-// ---- register re-partitioning between roles --------------------------------------------------------
-// Executed by all four warps of an aligned group of four; N is a multiple of 8.
-template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-
 // ---- small helpers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
