@@ -78,9 +78,10 @@ typedef struct hgrn2_desc {
  * path, the two per-chunk decay totals of every key dimension.  0 on a bad desc. */
 size_t hgrn2_saved_bytes(const hgrn2_desc *desc);
 
-/* Bytes of the workspace `ws` every call takes: a 256-byte status block followed by
- * room for the chunk states that hgrn2_bwd re-creates when it is given saved = NULL.
- * 0 on a bad desc. */
+/* Bytes of the workspace `ws` every call takes: a 256-byte status block, room for the
+ * saved data that hgrn2_bwd re-creates when it is given saved = NULL and, when the batch
+ * has too few (batch, head) units to fill the GPU, scratch for running each sequence as
+ * several segments (the size therefore depends on the current device).  0 on a bad desc. */
 size_t hgrn2_workspace_bytes(const hgrn2_desc *desc);
 
 /* Forward over a whole sequence (Eq. 3 unrolled chunk by chunk; training and prefill).

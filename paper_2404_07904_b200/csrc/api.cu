@@ -12,6 +12,7 @@ bool        tc_supported(const hgrn2_desc *d);
 int         tc_default_chunk();
 bool        tc_chunk_supported(int C);
 size_t      tc_saved_bytes(const hgrn2_desc *d, int C);
+size_t      tc_segment_scratch_bytes(const hgrn2_desc *d, int C);
 cudaError_t launch_tc_fwd(const SeqArgs &a);
 cudaError_t launch_tc_bwd(const SeqArgs &a);
 }  // namespace hgrn2
@@ -68,9 +69,12 @@ size_t saved_bytes_for(const hgrn2_desc *d, int C)
     return (size_t)d->B * d->H * NC * d->dk * d->dv * sizeof(float);
 }
 
-void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream)
+void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream, void *ws)
 {
     memset(&a, 0, sizeof(a));
+    // workspace layout: status block | room for re-created saved data | segment scratch (tensor-core path)
+    if (use_tc(d) && tc_segment_scratch_bytes(d, C) != 0)
+        a.seg_scratch = static_cast<char *>(ws) + sizeof(StatusBlock) + saved_bytes_for(d, C);
     a.B = d->B; a.H = d->H; a.N = d->N; a.dk = d->dk; a.dv = d->dv; a.C = C;
     a.NC = (d->N + C - 1) / C;
     a.io = d->io;
@@ -100,7 +104,7 @@ size_t hgrn2_workspace_bytes(const hgrn2_desc *desc)
 {
     const int C = resolve_chunk(desc);
     if (C == 0) return 0;
-    return sizeof(StatusBlock) + saved_bytes_for(desc, C);
+    return sizeof(StatusBlock) + saved_bytes_for(desc, C) + (use_tc(desc) ? tc_segment_scratch_bytes(desc, C) : 0);
 }
 
 const char *hgrn2_status_string(hgrn2_status s)
@@ -132,7 +136,7 @@ hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, con
     if (st != HGRN2_OK) return st;
 
     SeqArgs a;
-    fill_args(a, desc, C, cuda_stream);
+    fill_args(a, desc, C, cuda_stream, ws);
     a.o = o; a.f = f; a.i = i; a.S0 = S0; a.y = y; a.SN = SN;
     a.states = static_cast<float *>(saved);
     a.status = static_cast<StatusBlock *>(ws);
@@ -165,7 +169,7 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
     if (st != HGRN2_OK) return st;
 
     SeqArgs a;
-    fill_args(a, desc, C, cuda_stream);
+    fill_args(a, desc, C, cuda_stream, ws);
     a.o = o; a.f = f; a.i = i; a.S0 = S0; a.dy = dy; a.dSN = dSN;
     a.d_o = d_o; a.d_f = d_f; a.d_i = d_i; a.dS0 = dS0;
     a.status = static_cast<StatusBlock *>(ws);

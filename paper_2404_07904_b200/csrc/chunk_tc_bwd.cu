@@ -181,6 +181,9 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qt
     esum = H;
 }
 
+// kDsOnly: run the state-gradient chain alone (dS_0 from dS_N and dy; no other output), for sequences split
+// into segments.  A template parameter, not a flag: the full kernel is sensitive to its instruction footprint.
+template <bool kDsOnly>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
@@ -318,6 +321,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             fence_proxy_async_smem();
             mbar_arrive(&ctl->m_done);
             PT_MARK(2)
+            if (kDsOnly) continue;                                   // state-gradient chain only
 
             // ---- tril(A), tril(dA) -> operand slabs
             mbar_wait(&ctl->barX, it & 1, abort_flag);
@@ -382,6 +386,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         PT_DECL
         for (int it = 0; it < NC; ++it) {
             const int c = NC - 1 - it, s = it % kStages;
+            if (kDsOnly) {                                           // nothing to output: just hand the stage back
+                mbar_wait(&ctl->barY2, it & 1, abort_flag);
+                mbar_arrive(&ctl->stage_read[s]);
+                continue;
+            }
             const int n_valid = min(kC, N - c * kC);
             const uint8_t *qtile = smem + s * kStageBytes, *ktile = qtile + kTile;
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
@@ -406,7 +415,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         // ================= O: d_i, and d_f completed from the parked values =================
         const uint32_t tl = tmem + lane_base;
         PT_DECL
-        for (int it = 0; it < NC; ++it) {
+        for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
             const int c = NC - 1 - it;
             const int n_valid = min(kC, N - c * kC);
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
@@ -470,13 +479,15 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, u * NC + c);
             };
             issue_stage(0);
-            issue_state(0);
+            if (!kDsOnly) issue_state(0);
             if (NC > 1) issue_stage(1);
             for (int it = 0; it + 1 < NC; ++it) {
                 // chunk `it` is finished with S' once its products and its R are done ...
                 mbar_wait(&ctl->barY2, it & 1, abort_flag);
-                mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
-                issue_state(it + 1);
+                if (!kDsOnly) {
+                    mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
+                    issue_state(it + 1);
+                }
                 // ... and with its stage once the output warps have read Qs and Ks
                 if (it + 2 < NC) {
                     mbar_wait(&ctl->stage_read[it % kStages], (it / kStages) & 1, abort_flag);
@@ -513,24 +524,30 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
                 PT_MARK(0)
                 mbar_wait(&ctl->m_done, it & 1, abort_flag);          // dS'' in TMEM
-                if (it > 0) mbar_wait(&ctl->pd_ready, (it - 1) & 1, abort_flag);   // A, dA of the previous chunk read out
+                if (it > 0 && !kDsOnly) mbar_wait(&ctl->pd_ready, (it - 1) & 1, abort_flag);   // A, dA of the previous chunk read out
                 PT_MARK(1)
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
                     mma_bf16_ss(tmem + kColDS, dqm + (uint64_t)(kk * 128), dgm + (uint64_t)(kk * 128), idDS, 1);
+                if constexpr (kDsOnly) {                    // state-gradient chain only: stand in for the other groups
+                    mma_commit(&ctl->barX);
+                    mma_commit(&ctl->barY1);
+                    mma_commit(&ctl->barY2);
+                } else {
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)              // A = Qs Ks^T
-                    mma_bf16_ss(tmem + kColA, dqk + kmaj(kk), dfk + kmaj(kk), idA, kk > 0);
+                    for (int kk = 0; kk < 8; ++kk)          // A = Qs Ks^T
+                        mma_bf16_ss(tmem + kColA, dqk + kmaj(kk), dfk + kmaj(kk), idA, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)              // dA = dY V^T
-                    mma_bf16_ss(tmem + kColDA, dgk + kmaj(kk), dvk + kmaj(kk), idA, kk > 0);
-                mma_commit(&ctl->barX);
+                    for (int kk = 0; kk < 8; ++kk)          // dA = dY V^T
+                        mma_bf16_ss(tmem + kColDA, dgk + kmaj(kk), dvk + kmaj(kk), idA, kk > 0);
+                    mma_commit(&ctl->barX);
+                }
                 PT_MARK(2)
             }
             PT_DUMP(status, 15, 3, true)
         } else if (warp == kWarpMmaY1) {
-            for (int it = 0; it < NC; ++it) {
+            for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
                 const uint64_t dfk = dfk0 + so, dvk = dvk0 + so;
@@ -555,7 +572,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
             PT_DUMP(status, 18, 3, true)
         } else {
-            for (int it = 0; it < NC; ++it) {
+            for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
                 const uint64_t dqm = dqm0 + so, dfm = dfm0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
@@ -593,7 +610,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int last = ((NC - 1 - s) / kStages) * kStages + s;
             if (s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
         }
-        mbar_wait_drain(&ctl->sfull, (NC - 1) & 1, 20000000ull);
+        if (!kDsOnly) mbar_wait_drain(&ctl->sfull, (NC - 1) & 1, 20000000ull);
     }
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
@@ -601,21 +618,70 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
 }  // namespace
 
+// ---- sequences split into segments (see chunk_tc_fwd.cu) ----------------------------------------------
+// Total decay of every segment from the forward's saved per-chunk totals: lam[ur][k] = prod_c Pm E.
+__global__ void seg_decay_kernel(const float *__restrict__ totals, float *__restrict__ lam, int chunks_per_seg)
+{
+    const size_t ur = blockIdx.x;
+    const int k = threadIdx.x;
+    const float *t = totals + ur * chunks_per_seg * 2 * kD + k;
+    float p = 1.f;
+    for (int c = 0; c < chunks_per_seg; ++c) p *= t[(size_t)c * 2 * kD] * t[(size_t)c * 2 * kD + kD];
+    lam[ur * kD + k] = p;
+}
+// Chains the segments in reverse: dS_end[r] = gradient w.r.t. the state at the end of segment r.
+__global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const float *__restrict__ G_loc,
+                                       const float *__restrict__ lam, float *__restrict__ dS_end,
+                                       float *__restrict__ dS0, int G)
+{
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
+    const size_t u = e / (kD * kD);
+    const int k = (int)((e / kD) % kD);
+    const size_t kv = e % (kD * kD);
+    float D = dSN ? dSN[e] : 0.f;
+    for (int r = G - 1; r >= 0; --r) {
+        const size_t ur = u * G + r;
+        dS_end[ur * kD * kD + kv] = D;
+        D = fmaf(lam[ur * kD + k], D, G_loc[ur * kD * kD + kv]);
+    }
+    if (dS0) dS0[e] = D;
+}
+
+int segments_for(uint64_t U, int N, int NC);     // chunk_tc_fwd.cu
+
+static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly)
+{
+    CUtensorMap mo, mf, mi, mg, ms;
+    if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
+        !make_map(&mg, a.dy, U, N, kC) || !make_map(&ms, a.states, U * NC, kD, kD))
+        return cudaErrorInvalidValue;
+    auto kernel = kDsOnly ? tc_bwd_kernel<true> : tc_bwd_kernel<false>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (err != cudaSuccess) return err;
+    kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
+        mo, mf, mi, mg, ms,
+        reinterpret_cast<const float *>(reinterpret_cast<const char *>(a.states) + U * NC * kSavedStateBytes),
+        static_cast<const __nv_bfloat16 *>(a.f), dSN, static_cast<__nv_bfloat16 *>(a.d_o),
+        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_tc_bwd(const SeqArgs &a)
 {
     const uint64_t U = (uint64_t)a.B * a.H;
-    CUtensorMap mo, mf, mi, mg, ms;
-    if (!make_map(&mo, a.o, U, a.N, kC) || !make_map(&mf, a.f, U, a.N, kC) || !make_map(&mi, a.i, U, a.N, kC) ||
-        !make_map(&mg, a.dy, U, a.N, kC) || !make_map(&ms, a.states, U * a.NC, kD, kD))
-        return cudaErrorInvalidValue;
-    cudaError_t err = cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    const int G = a.seg_scratch ? segments_for(U, a.N, a.NC) : 1;
+    if (G == 1) return launch_bwd_once(a, U, a.N, a.NC, a.dSN, a.dS0, false);
+    // scratch: G_local [U*G][128][128], dS_end [U*G][128][128], Lambda [U*G][128]
+    float *G_loc = static_cast<float *>(a.seg_scratch);
+    float *dS_end = G_loc + U * G * kD * kD;
+    float *lam = dS_end + U * G * kD * kD;
+    const float *totals = reinterpret_cast<const float *>(reinterpret_cast<const char *>(a.states) + U * a.NC * kSavedStateBytes);
+    cudaError_t err = launch_bwd_once(a, U * G, a.N / G, a.NC / G, nullptr, G_loc, true);     // state-gradient chains only
     if (err != cudaSuccess) return err;
-    tc_bwd_kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
-        mo, mf, mi, mg, ms,
-        reinterpret_cast<const float *>(reinterpret_cast<const char *>(a.states) + U * a.NC * kSavedStateBytes),
-        static_cast<const __nv_bfloat16 *>(a.f), a.dSN, static_cast<__nv_bfloat16 *>(a.d_o),
-        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), a.dS0, a.N, a.NC, a.status);
-    return cudaGetLastError();
+    seg_decay_kernel<<<(unsigned)(U * G), kD, 0, a.stream>>>(totals, lam, a.NC / G);
+    seg_combine_bwd_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.dSN, G_loc, lam, dS_end, a.dS0, G);
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    return launch_bwd_once(a, U * G, a.N / G, a.NC / G, dS_end, nullptr, false);
 }
 
 }  // namespace hgrn2

@@ -69,11 +69,15 @@ struct Ctl {
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
+// kSegDecay: also write the product of f over the whole (sub)sequence per key dimension to seg_decay (used when
+// sequences are split into segments).  A template parameter: the kernel is sensitive to its instruction footprint.
+template <bool kSegDecay>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
               const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
-              float *__restrict__ totals, int want_y, int want_saved, int N, int NC, StatusBlock *status)
+              float *__restrict__ totals, float *__restrict__ seg_decay, int want_y, int want_saved, int N, int NC,
+              StatusBlock *status)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -151,6 +155,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         const int krow = 32 * sub + lane;
         const int v0 = 64 * half;
         float e_prev = 1.f;
+        float lam = 1.f;                                             // product of f over the whole sequence, this key dim
         PT_DECL
         for (int c = 0; c < NC; ++c) {
             // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk) back into TMEM
@@ -158,6 +163,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             PT_MARK(0)
             const float factor = e_prev * pm[(c & 3) * 128 + krow];
             e_prev = ee[(c & 3) * 128 + krow];
+            if (kSegDecay) lam *= pm[(c & 3) * 128 + krow] * e_prev;
             uint32_t r[64];
             if (c == 0) {
                 if (S0) {
@@ -202,6 +208,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             PT_MARK(4)
         }
         PT_DUMP(status, 2, 5, tid == kWarpE1 * 32)
+
+        if (kSegDecay && half == 0) seg_decay[(size_t)u * kD + krow] = lam;
 
         // S_N = Diag(E_last) S''
         mbar_wait(&ctl->barS, (NC - 1) & 1, abort_flag);
@@ -414,25 +422,93 @@ size_t tc_saved_bytes(const hgrn2_desc *d, int C)
     return (size_t)d->B * d->H * NC * (kSavedStateBytes + kSavedTotalsBytes);
 }
 
+// ---- sequences split into segments ----------------------------------------------------------------------
+// One CTA per unit leaves most SMs idle when there are few units (a 16K-token batch of two sequences has
+// 32).  The recurrence is linear in the state, so a sequence can be cut into G segments that run as separate
+// CTAs: (1) every segment runs state-only from a zero state, giving its local end state and its total decay
+// Lambda = prod f; (2) a small kernel chains them, S_start[r+1] = Diag(Lambda[r]) S_start[r] + S_local[r];
+// (3) every segment runs in full from its S_start.  Token (r, t) of unit u is token t of "unit" u * G + r of a
+// [U * G][N / G][128] view of the same memory, so the kernel itself does not know about segments.
+__global__ void seg_combine_kernel(const float *__restrict__ S0, const float *__restrict__ S_loc,
+                                   const float *__restrict__ lam, float *__restrict__ S_start, float *__restrict__ SN,
+                                   int G)
+{
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
+    const size_t u = e / (kD * kD);
+    const int k = (int)((e / kD) % kD);
+    const size_t kv = e % (kD * kD);
+    float S = S0 ? S0[e] : 0.f;
+    for (int r = 0; r < G; ++r) {
+        const size_t ur = u * G + r;
+        S_start[ur * kD * kD + kv] = S;
+        S = fmaf(lam[ur * kD + k], S, S_loc[ur * kD * kD + kv]);
+    }
+    if (SN) SN[e] = S;
+}
+
+int sm_count()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return n;
+}
+
+// Number of segments per sequence (1 = do not split): as many as fill the SMs, at most 8, dividing the chunk
+// count, each at least 8 chunks long; only for sequences made of whole chunks.
+int segments_for(uint64_t U, int N, int NC)
+{
+    if (U == 0 || N % kC != 0) return 1;
+    int G = (int)(sm_count() / (int)U);
+    if (G > 8) G = 8;
+    while (G >= 2 && (NC % G != 0 || NC / G < 8)) --G;
+    return G >= 2 ? G : 1;
+}
+
+size_t tc_segment_scratch_bytes(const hgrn2_desc *d, int C)
+{
+    const uint64_t U = (uint64_t)d->B * d->H;
+    const int NC = (d->N + C - 1) / C;
+    const int G = segments_for(U, d->N, NC);
+    return G > 1 ? (size_t)U * G * (2 * kD * kD + kD) * sizeof(float) : 0;
+}
+
+static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *S0, float *SN, float *seg_decay,
+                                   bool want_y, bool want_saved)
+{
+    CUtensorMap mo, mf, mi, my, ms;
+    // tensor maps need a valid base even for outputs that are not wanted: point those at an input
+    const void *ybase = want_y ? a.y : a.i;
+    const void *sbase = want_saved ? static_cast<const void *>(a.states) : a.i;
+    const uint64_t srows = want_saved ? (uint64_t)kD : (uint64_t)N;
+    const uint64_t sunits = want_saved ? U * NC : U;
+    if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
+        !make_map(&my, ybase, U, N, kC) || !make_map(&ms, sbase, sunits, srows, want_saved ? kD : kC))
+        return cudaErrorInvalidValue;
+    auto kernel = seg_decay ? tc_fwd_kernel<true> : tc_fwd_kernel<false>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (err != cudaSuccess) return err;
+    float *totals = want_saved ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * NC * kSavedStateBytes)
+                               : nullptr;
+    kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, seg_decay, want_y,
+                                                                   want_saved, N, NC, a.status);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_tc_fwd(const SeqArgs &a)
 {
     const uint64_t U = (uint64_t)a.B * a.H;
-    CUtensorMap mo, mf, mi, my, ms;
-    // tensor maps need a valid base even for outputs that are not wanted: point those at an input
-    const void *ybase = a.y ? a.y : a.i;
-    const void *sbase = a.states ? static_cast<const void *>(a.states) : a.i;
-    const uint64_t srows = a.states ? (uint64_t)kD : (uint64_t)a.N;
-    const uint64_t sunits = a.states ? U * a.NC : U;
-    if (!make_map(&mo, a.o, U, a.N, kC) || !make_map(&mf, a.f, U, a.N, kC) || !make_map(&mi, a.i, U, a.N, kC) ||
-        !make_map(&my, ybase, U, a.N, kC) || !make_map(&ms, sbase, sunits, srows, a.states ? kD : kC))
-        return cudaErrorInvalidValue;
-    cudaError_t err = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    const int G = a.seg_scratch ? segments_for(U, a.N, a.NC) : 1;
+    if (G == 1) return launch_fwd_once(a, U, a.N, a.NC, a.S0, a.SN, nullptr, a.y != nullptr, a.states != nullptr);
+    // scratch: S_local [U*G][128][128], S_start [U*G][128][128], Lambda [U*G][128]
+    float *S_loc = static_cast<float *>(a.seg_scratch);
+    float *S_start = S_loc + U * G * kD * kD;
+    float *lam = S_start + U * G * kD * kD;
+    cudaError_t err = launch_fwd_once(a, U * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false);
     if (err != cudaSuccess) return err;
-    float *totals = a.states ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes)
-                             : nullptr;
-    tc_fwd_kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, a.S0, a.SN, totals, a.y != nullptr,
-                                                                   a.states != nullptr, a.N, a.NC, a.status);
-    return cudaGetLastError();
+    seg_combine_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.S0, S_loc, lam, S_start, a.SN, G);
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    return launch_fwd_once(a, U * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, a.y != nullptr, a.states != nullptr);
 }
 
 }  // namespace hgrn2

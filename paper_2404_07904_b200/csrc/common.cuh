@@ -55,6 +55,7 @@ struct SeqArgs {
     void *d_o, *d_f, *d_i;        // bwd out
     float *dS0;                   // nullable
     StatusBlock *status;
+    void *seg_scratch;            // tensor-core path: scratch for sequences split into segments (nullable)
     cudaStream_t stream;
 };
 

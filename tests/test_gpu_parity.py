@@ -161,6 +161,20 @@ def test_bf16_recompute_matches_saved():
         np.testing.assert_array_equal(a[k], b[k])
 
 
+def test_few_units_split_into_segments():
+    # 4 units of 32 chunks: too few to fill the GPU, so each sequence runs as several segments chained through
+    # their boundary states (forward) and boundary state gradients (backward); all outputs against the oracle
+    w = W.scaled(W.CONFIGS["long_16k"], B=1, H=4, N=2048, seed=77)
+    d = binding.make_desc(w.B, w.H, w.N, w.dk, w.dv, binding.HGRN2_BF16)
+    assert binding.workspace_bytes(d) > 256 + binding.saved_bytes(d), "segment scratch expected in the workspace"
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "bf16")
+    _check_units(inp, got, [(0, 0), (0, 3)], 2e-2, "segments")
+    got2 = G.gpu_fwd_bwd(inp, "bf16", use_saved=False)
+    for k in got:
+        np.testing.assert_array_equal(got[k], got2[k])
+
+
 def test_config2_full_size_sampled_units():
     w = W.CONFIGS["lm_2048"]
     inp = W.make_inputs(w)
