@@ -183,7 +183,9 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qt
 
 // kDsOnly: run the state-gradient chain alone (dS_0 from dS_N and dy; no other output), for sequences split
 // into segments.  A template parameter, not a flag: the full kernel is sensitive to its instruction footprint.
-template <bool kDsOnly>
+// kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens); when false,
+// every per-row validity test below folds away.
+template <bool kDsOnly, bool kRagged>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
@@ -255,7 +257,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             uint8_t *qbuf = smem + s * kStageBytes;
             mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
             PT_MARK(0)
-            const int n_valid = N - c * kC;
+            const int n_valid = kRagged ? N - c * kC : kC;
             // Pm and E of the chunk are not kept: the backward takes them from what the forward saved
             if (n_valid >= kC) {
                 transform_stream<true>(qbuf, qbuf + kTile, nullptr, nullptr, nullptr, nullptr, kC, tid);
@@ -391,7 +393,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mbar_arrive(&ctl->stage_read[s]);
                 continue;
             }
-            const int n_valid = min(kC, N - c * kC);
+            const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
             const uint8_t *qtile = smem + s * kStageBytes, *ktile = qtile + kTile;
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
             uint32_t *fs = fscr + (tid - kWarpE3 * 32);
@@ -417,7 +419,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         PT_DECL
         for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
             const int c = NC - 1 - it;
-            const int n_valid = min(kC, N - c * kC);
+            const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
             PT_MARK(0)
@@ -655,7 +657,9 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
         !make_map(&mg, a.dy, U, N, kC) || !make_map(&ms, a.states, U * NC, kD, kD))
         return cudaErrorInvalidValue;
-    auto kernel = kDsOnly ? tc_bwd_kernel<true> : tc_bwd_kernel<false>;
+    const bool ragged = N % kC != 0;
+    auto kernel = kDsOnly ? (ragged ? tc_bwd_kernel<true, true> : tc_bwd_kernel<true, false>)
+                          : (ragged ? tc_bwd_kernel<false, true> : tc_bwd_kernel<false, false>);
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(

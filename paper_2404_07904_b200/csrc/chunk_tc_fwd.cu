@@ -71,7 +71,8 @@ static_assert(kSmemBytes <= 232448, "shared memory budget");
 
 // kSegDecay: also write the product of f over the whole (sub)sequence per key dimension to seg_decay (used when
 // sequences are split into segments).  A template parameter: the kernel is sensitive to its instruction footprint.
-template <bool kSegDecay>
+// kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens).
+template <bool kSegDecay, bool kRagged>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
@@ -135,7 +136,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             uint8_t *qbuf = smem + s * kStageBytes;
             mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
             PT_MARK(0)
-            const int n_valid = N - c * kC;
+            const int n_valid = kRagged ? N - c * kC : kC;
             float *tg = totals ? totals + ((size_t)u * NC + c) * 2 * kD : nullptr;     // Pm, E of the chunk for the backward
             if (n_valid >= kC) {
                 transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
@@ -485,7 +486,9 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
         !make_map(&my, ybase, U, N, kC) || !make_map(&ms, sbase, sunits, srows, want_saved ? kD : kC))
         return cudaErrorInvalidValue;
-    auto kernel = seg_decay ? tc_fwd_kernel<true> : tc_fwd_kernel<false>;
+    const bool ragged = N % kC != 0;
+    auto kernel = seg_decay ? (ragged ? tc_fwd_kernel<true, true> : tc_fwd_kernel<true, false>)
+                            : (ragged ? tc_fwd_kernel<false, true> : tc_fwd_kernel<false, false>);
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * NC * kSavedStateBytes)
