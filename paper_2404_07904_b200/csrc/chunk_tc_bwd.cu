@@ -149,28 +149,49 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qt
             ks[j] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(ktile + off));
         }
         tmem_wait_ld();
-        float u[8], rf[8];
+        // scale factors along the walk (sequential in the running product), 1/f
+        float sq[8], sk[8], rf[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int j = kUp ? i : 7 - i;                      // visiting order: away from the middle
-            const int t = t0 + j;
             if (kUp) cp *= fv[j];
             const float m = fmaxf(cp, kProdFloor);
             const float mi = rcp_fast(m);
             if (!kUp) cp *= fv[j];
-            const float sq = kUp ? m : mi, sk = kUp ? mi : m;
-            const float xx = __uint_as_float(x[j]), yy = __uint_as_float(y[j]), zz = __uint_as_float(z[j]);
-            if (t < n_valid) do_g[(size_t)t * kD] = __float2bfloat16_rn(xx * sq);
-            const float a = fmaf(qs[j], xx, -ks[j] * yy);
-            const float e = ks[j] * zz;
-            const float dk = (yy + zz) * sk;
+            sq[j] = kUp ? m : mi;
+            sk[j] = kUp ? mi : m;
             rf[j] = rcp_fast(fmaxf(fv[j], kProdFloor));
+        }
+        // element-wise part, two rows per instruction (packed fp32)
+        float a[8], e[8], dk[8];
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const int j = 2 * p;
+            const float2 X = make_float2(__uint_as_float(x[j]), __uint_as_float(x[j + 1]));
+            const float2 Y = make_float2(__uint_as_float(y[j]), __uint_as_float(y[j + 1]));
+            const float2 Z = make_float2(__uint_as_float(z[j]), __uint_as_float(z[j + 1]));
+            const float2 QS = make_float2(qs[j], qs[j + 1]), KS = make_float2(ks[j], ks[j + 1]);
+            const float2 dox = mul2(X, make_float2(sq[j], sq[j + 1]));
+            const float2 a2 = sub2(mul2(QS, X), mul2(KS, Y));
+            const float2 e2 = mul2(KS, Z);
+            const float2 dk2 = mul2(add2(Y, Z), make_float2(sk[j], sk[j + 1]));
+            if (t0 + j < n_valid) do_g[(size_t)(t0 + j) * kD] = __float2bfloat16_rn(dox.x);
+            if (t0 + j + 1 < n_valid) do_g[(size_t)(t0 + j + 1) * kD] = __float2bfloat16_rn(dox.y);
+            a[j] = a2.x; a[j + 1] = a2.y;
+            e[j] = e2.x; e[j + 1] = e2.y;
+            dk[j] = dk2.x; dk[j + 1] = dk2.y;
+        }
+        // running sums along the walk
+        float u[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int j = kUp ? i : 7 - i;
             if (kUp) {              // rows after the middle: sums over the rows strictly before t
-                u[j] = fmaf(H - G, rf[j], -dk);
-                G += a; H += e;
+                u[j] = fmaf(H - G, rf[j], -dk[j]);
+                G += a[j]; H += e[j];
             } else {                // rows before the middle: sums over the rows from t on
-                G += a; H += e;
-                u[j] = fmaf(G - H, rf[j], -dk);
+                G += a[j]; H += e[j];
+                u[j] = fmaf(G - H, rf[j], -dk[j]);
             }
         }
         // park u and 1/f in the columns just read
@@ -311,7 +332,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tmem_wait_ld();
                 }
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
+                for (int j = 0; j < 32; j += 2) scale2(r[j], r[j + 1], factor);
                 tmem_st32(tmem + lane_base + kColDS + 32 * part, r);
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
