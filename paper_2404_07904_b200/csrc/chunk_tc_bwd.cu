@@ -278,6 +278,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             uint8_t *qbuf = smem + s * kStageBytes;
             mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
             PT_MARK(0)
+            PT_STAMP(status, 1, tid == 0 && it == 16) PT_STAMP(status, 20, tid == 0 && it == 18)
             const int n_valid = kRagged ? N - c * kC : kC;
             // Pm and E of the chunk are not kept: the backward takes them from what the forward saved
             if (n_valid >= kC) {
@@ -288,6 +289,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             fence_proxy_async_smem();
             mbar_arrive(&ctl->t_done[s]);
             PT_MARK(1)
+            PT_STAMP(status, 2, tid == 0 && it == 16)
         }
         PT_DUMP(status, 0, 2, tid == 0)
     } else if (warp < kWarpE3) {
@@ -311,6 +313,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 tc_fence_after_sync();
             }
             PT_MARK(1)
+            PT_STAMP(status, 5, tid == kWarpE1 * 32 && it == 16)
 #pragma unroll 1
             for (int part = 0; part < 4; ++part) {
                 uint32_t r[32];
@@ -344,6 +347,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             fence_proxy_async_smem();
             mbar_arrive(&ctl->m_done);
             PT_MARK(2)
+            PT_STAMP(status, 6, tid == kWarpE1 * 32 && it == 16)
             if (kDsOnly) continue;                                   // state-gradient chain only
 
             // ---- tril(A), tril(dA) -> operand slabs
@@ -351,6 +355,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             if (it > 0) mbar_wait(&ctl->barY2, (it - 1) & 1, abort_flag);   // the previous chunk's products have read P, dP
             PT_MARK(3)
             tc_fence_after_sync();
+            PT_STAMP(status, 7, tid == kWarpE1 * 32 && it == 16)
 #pragma unroll 1
             for (int w = 0; w < 2; ++w) {
                 const uint32_t col = w ? kColDA : kColA;
@@ -362,6 +367,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             tc_fence_before_sync();
             mbar_arrive(&ctl->pd_ready);
             PT_MARK(4)
+            PT_STAMP(status, 8, tid == kWarpE1 * 32 && it == 16)
 
             // ---- R_k = sum_v dS''[k,v] S'[k,v] from the two bf16 copies
             mbar_wait(&ctl->sfull, it & 1, abort_flag);
@@ -383,6 +389,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             rr[(it & 1) * 128 + krow] = racc;
             mbar_arrive(&ctl->r_ready[it & 1]);
             PT_MARK(6)
+            PT_STAMP(status, 9, tid == kWarpE1 * 32 && it == 16)
         }
         PT_DUMP(status, 2, 7, tid == kWarpE1 * 32)
 
@@ -423,6 +430,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             PT_MARK(0)
             tc_fence_after_sync();
             float asum, esum;
+            PT_STAMP(status, 14, tid == kWarpE3 * 32 && it == 16)
             if (half) phase_main<true>(tl, qtile, ktile, krow, fs, d_o + row0 * kD + krow, n_valid, asum, esum);
             else      phase_main<false>(tl, qtile, ktile, krow, fs, d_o + row0 * kD + krow, n_valid, asum, esum);
             mbar_arrive(&ctl->stage_read[s]);
@@ -432,6 +440,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_arrive(&ctl->acc_free1);
             mbar_arrive(&ctl->parked);
             PT_MARK(1)
+            PT_STAMP(status, 15, tid == kWarpE3 * 32 && it == 16)
         }
         PT_DUMP(status, 9, 2, tid == kWarpE3 * 32)
     } else if (warp < kWarpLoad) {
@@ -444,6 +453,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
             PT_MARK(0)
+            PT_STAMP(status, 16, tid == kWarpO * 32 && it == 16)
             tc_fence_after_sync();
             // d_i = dV: lane = value dimension, columns = local times
 #pragma unroll 1
@@ -459,9 +469,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_freeV);
             PT_MARK(1)
+            PT_STAMP(status, 17, tid == kWarpO * 32 && it == 16)
             mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
             mbar_wait(&ctl->parked, it & 1, abort_flag);
             PT_MARK(2)
+            PT_STAMP(status, 18, tid == kWarpO * 32 && it == 16)
             tc_fence_after_sync();
             const float K = rr[(it & 1) * 128 + krow] + xa[krow] + xe[krow];
 #pragma unroll 1
@@ -479,6 +491,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_free2);
             PT_MARK(3)
+            PT_STAMP(status, 19, tid == kWarpO * 32 && it == 16)
         }
         PT_DUMP(status, 11, 4, tid == kWarpO * 32)
     } else if (warp == kWarpLoad) {
@@ -510,11 +523,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 if (!kDsOnly) {
                     mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
                     issue_state(it + 1);
+                    PT_STAMP(status, 22, it == 15)
                 }
                 // ... and with its stage once the output warps have read Qs and Ks
                 if (it + 2 < NC) {
                     mbar_wait(&ctl->stage_read[it % kStages], (it / kStages) & 1, abort_flag);
                     issue_stage(it + 2);
+                    PT_STAMP(status, 0, it == 14) PT_STAMP(status, 21, it == 16)
                 }
             }
         }
@@ -549,6 +564,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mbar_wait(&ctl->m_done, it & 1, abort_flag);          // dS'' in TMEM
                 if (it > 0 && !kDsOnly) mbar_wait(&ctl->pd_ready, (it - 1) & 1, abort_flag);   // A, dA of the previous chunk read out
                 PT_MARK(1)
+                PT_STAMP(status, 3, it == 16)
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
@@ -567,6 +583,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     mma_commit(&ctl->barX);
                 }
                 PT_MARK(2)
+                PT_STAMP(status, 4, it == 16)
             }
             PT_DUMP(status, 15, 3, true)
         } else if (warp == kWarpMmaY1) {
@@ -583,6 +600,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     mbar_wait(&ctl->acc_freeV, (it - 1) & 1, abort_flag);
                 }
                 PT_MARK(1)
+                PT_STAMP(status, 10, it == 16)
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)              // dKs_inter^T = dS'' V^T
@@ -602,9 +620,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mbar_wait(&ctl->pd_ready, it & 1, abort_flag);        // tril(A), tril(dA); implies X and T of the chunk
                 mbar_wait(&ctl->sfull, it & 1, abort_flag);
                 PT_MARK(0)
+                PT_STAMP(status, 11, it == 16)
                 mbar_wait(&ctl->barY1, it & 1, abort_flag);           // dV^T += ... must follow dV^T = ...
                 if (it > 0) mbar_wait(&ctl->acc_free2, (it - 1) & 1, abort_flag);
                 PT_MARK(1)
+                PT_STAMP(status, 12, it == 16)
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dQs^T = Ks^T dA^T
@@ -620,6 +640,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     mma_bf16_ss(tmem + kColDV, dgm + (uint64_t)(kk * 128), dpm + (uint64_t)(kk * 128), idMM, 1);
                 mma_commit(&ctl->barY2);
                 PT_MARK(2)
+                PT_STAMP(status, 13, it == 16)
             }
             PT_DUMP(status, 21, 3, true)
         }

@@ -44,7 +44,9 @@ constexpr size_t kSavedTotalsBytes = 2 * kD * sizeof(float);
 #define PT_DECL long long pt_t0 = clock64(); long long pt_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
 #define PT_MARK(i) { const long long pt_t = clock64(); pt_acc[i] += pt_t - pt_t0; pt_t0 = pt_t; }
 #define PT_DUMP(st, base, n, cond) if ((cond) && blockIdx.x == 0 && (st) != nullptr) { for (int pt_i = 0; pt_i < (n); ++pt_i) (st)->pad[(base) + pt_i] = (int)(pt_acc[pt_i] >> 4); }
+#define PT_STAMP(st, idx, cond) if (blockIdx.x == 0 && (cond) && (st) != nullptr) (st)->pad[30 + (idx)] = (int)(clock64() & 0x3fffffff);
 #else
+#define PT_STAMP(st, idx, cond)
 #define PT_DECL
 #define PT_MARK(i)
 #define PT_DUMP(st, base, n, cond)
