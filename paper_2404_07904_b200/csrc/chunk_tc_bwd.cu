@@ -55,13 +55,15 @@ constexpr int kWarpLoad = kWarpO + kOWarps, kWarpMmaX = kWarpLoad + 1, kWarpMmaY
 constexpr int kThreads = (kWarpMmaY2 + 1) * 32;
 
 constexpr int kStages = 2;
-constexpr uint32_t kStageBytes = 4 * kTile;                       // q, f, v, dy
-constexpr uint32_t kOffS = kStages * kStageBytes;                 // S' (bf16, from the forward)
+constexpr uint32_t kStageBytes = 3 * kTile;                       // q, f, dy: free again when the chunk's products are done
+constexpr uint32_t kOffV = kStages * kStageBytes;                 // v: one buffer, free when X and Y1 of the chunk are done
+constexpr uint32_t kOffS = kOffV + kTile;                         // S' (bf16, from the forward)
 constexpr uint32_t kOffDS = kOffS + kStateTile;                   // bf16 copy of dS''
 constexpr uint32_t kOffP = kOffDS + kStateTile;                   // bf16 tril(A)
 constexpr uint32_t kOffDP = kOffP + kSlab;                        // bf16 tril(dA)
-constexpr uint32_t kOffF = kOffDP + kSlab;                        // uint32 fscr[16][256]: f strips of the E3 threads
-constexpr uint32_t kOffR = kOffF + 16 * 256 * 4;                  // float rr[2][128]
+constexpr uint32_t kOffRawO = kOffDP + kSlab;                     // raw o and f of the chunk, plain [64][128] bf16, for
+constexpr uint32_t kOffRawF = kOffRawO + kTile;                   // the output warps (the stage holds Qs, Ks by then)
+constexpr uint32_t kOffR = kOffRawF + kTile;                      // float rr[2][128]
 constexpr uint32_t kOffX = kOffR + 2 * 128 * 4;                   // float xa[128], xe[128]
 constexpr uint32_t kOffCtl = kOffX + 2 * 128 * 4;
 constexpr uint32_t kSmemBytes = kOffCtl + 256;                    // no slack: the base must be 1024-byte aligned
@@ -69,8 +71,10 @@ constexpr uint32_t kSmemBytes = kOffCtl + 256;                    // no slack: t
 constexpr uint32_t kColDS = 0, kColA = 128, kColDA = 192, kColDQ = 256, kColDKi = 320, kColDKx = 384, kColDV = 448;
 
 struct Ctl {
-    uint64_t full[kStages];       // TMA (raw tiles) -> T, M
-    uint64_t stage_read[kStages]; // E3 -> L: Qs, Ks of the stage have been read for the last time
+    uint64_t full[kStages];       // TMA (o, f, dy tiles) -> T, M
+    uint64_t vfull;               // TMA (v tile) -> M
+    uint64_t rawfull;             // TMA (second, unswizzled copy of o and f) -> E3
+    uint64_t raw_read;            // E3 -> L: the raw copies have been read for the last time
     uint64_t t_done[kStages];     // T -> M, E1
     uint64_t sfull;               // TMA (saved S') -> E1, M
     uint64_t m_done;              // E1 -> M: dS'' is in TMEM and in shared memory
@@ -90,40 +94,16 @@ struct Ctl {
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
-// f of the 32 rows [t_first, t_first + 32) of one key dimension as raw bf16 bits, two rows per word, into
-// the thread's column of the scratch; rows at or beyond n_valid read as 1.  f_g points at (row 0 of the chunk,
-// column k).
-__device__ __forceinline__ void load_f_strip(const __nv_bfloat16 *f_g, int t_first, int n_valid, uint32_t *fs)
-{
-    const unsigned short *fp = reinterpret_cast<const unsigned short *>(f_g);
-#pragma unroll 1
-    for (int h = 0; h < 2; ++h) {
-        uint32_t w[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int t = t_first + 16 * h + 2 * i;
-            const uint32_t lo = (t < n_valid) ? fp[(size_t)t * kD] : 0x3F80u;
-            const uint32_t hi = (t + 1 < n_valid) ? fp[(size_t)(t + 1) * kD] : 0x3F80u;
-            w[i] = lo | (hi << 16);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) fs[(8 * h + i) * 256] = w[i];
-    }
-}
-
 // d_o and the nearly finished d_f of one thread: key dimension k, local times [32 * kUp, 32 * kUp + 32),
 // walked outwards from the middle of the chunk in blocks of eight.  Returns this half's sums of a and e.
-// do_g points at element (row 0 of the chunk, column k) of d_o in global memory.  fs points at this thread's
-// column of the f scratch (word i, stride 256 words, holds f of its rows 2i and 2i + 1 in row order), filled by
-// the thread itself while it waited for the products: narrow global loads inside the loop would put a round
-// trip to L2 on every block's dependent chain.
-template <bool kUp>
-__device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qtile, const uint8_t *ktile, int k,
-                                           const uint32_t *fs, __nv_bfloat16 *do_g, int n_valid, float &asum,
-                                           float &esum)
+// do_g points at element (row 0 of the chunk, column k) of d_o in global memory.  oraw, fraw: the chunk's raw
+// o and f as plain [64][128] bf16 tiles (rows beyond the end of the sequence read as zero there, so f is
+// patched to the neutral 1).  Qs and Ks are recomputed from them with the transform's own roundings, so the
+// operand stage does not have to be held until the outputs are done.
+template <bool kUp, bool kRagged>
+__device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat16 *oraw, const __nv_bfloat16 *fraw,
+                                           int k, __nv_bfloat16 *do_g, int n_valid, float &asum, float &esum)
 {
-    const int kch = (k & 63) >> 3;
-    const uint32_t kbase = (k >> 6) * kSlab + (k & 7) * 2;
     float cp = 1.f;                 // running product of f between the middle and the current row
     float G = 0.f, H = 0.f;         // running sums of a and e over the rows visited so far
 #pragma unroll 1
@@ -133,20 +113,15 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qt
         tmem_ld8(tmem_lane + kColDQ + t0, x);
         tmem_ld8(tmem_lane + kColDKi + t0, y);
         tmem_ld8(tmem_lane + kColDKx + t0, z);
-        float fv[8], qs[8], ks[8];
-        const uint32_t *fb = fs + (kUp ? 4 * b : 12 - 4 * b) * 256;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t fw = fb[j * 256];
-            fv[2 * j] = bf16_lo(fw);
-            fv[2 * j + 1] = bf16_hi(fw);
-        }
+        uint32_t fw[8], qw[8];         // raw bf16 bits
+        float fv[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int t = t0 + j;
-            const uint32_t off = kbase + t * 128 + ((kch ^ j) << 4);
-            qs[j] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(qtile + off));
-            ks[j] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(ktile + off));
+            fw[j] = reinterpret_cast<const unsigned short *>(fraw)[t * kD + k];
+            qw[j] = reinterpret_cast<const unsigned short *>(oraw)[t * kD + k];
+            if (kRagged && t >= n_valid) fw[j] = 0x3F80u;
+            fv[j] = __uint_as_float(fw[j] << 16);
         }
         tmem_wait_ld();
         // scale factors along the walk (sequential in the running product), 1/f
@@ -170,13 +145,18 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const uint8_t *qt
             const float2 X = make_float2(__uint_as_float(x[j]), __uint_as_float(x[j + 1]));
             const float2 Y = make_float2(__uint_as_float(y[j]), __uint_as_float(y[j + 1]));
             const float2 Z = make_float2(__uint_as_float(z[j]), __uint_as_float(z[j + 1]));
-            const float2 QS = make_float2(qs[j], qs[j + 1]), KS = make_float2(ks[j], ks[j + 1]);
+            // Qs, Ks of the two rows exactly as the transform warps rounded them for the products: the terms
+            // of a cancel in pairs along the chunk only if both sides use the same operand values
+            const uint32_t sqp = pack_bf16(sq[j], sq[j + 1]), skp = pack_bf16(sk[j], sk[j + 1]);
+            const uint32_t qsp = mul_bf16x2(qw[j] | (qw[j + 1] << 16), sqp);
+            const uint32_t ksp = fma_bf16x2(fw[j] | (fw[j + 1] << 16), skp ^ 0x80008000u, skp);
+            const float2 QS = make_float2(bf16_lo(qsp), bf16_hi(qsp)), KS = make_float2(bf16_lo(ksp), bf16_hi(ksp));
             const float2 dox = mul2(X, make_float2(sq[j], sq[j + 1]));
             const float2 a2 = sub2(mul2(QS, X), mul2(KS, Y));
             const float2 e2 = mul2(KS, Z);
             const float2 dk2 = mul2(add2(Y, Z), make_float2(sk[j], sk[j + 1]));
-            if (t0 + j < n_valid) do_g[(size_t)(t0 + j) * kD] = __float2bfloat16_rn(dox.x);
-            if (t0 + j + 1 < n_valid) do_g[(size_t)(t0 + j + 1) * kD] = __float2bfloat16_rn(dox.y);
+            if (!kRagged || t0 + j < n_valid) do_g[(size_t)(t0 + j) * kD] = __float2bfloat16_rn(dox.x);
+            if (!kRagged || t0 + j + 1 < n_valid) do_g[(size_t)(t0 + j + 1) * kD] = __float2bfloat16_rn(dox.y);
             a[j] = a2.x; a[j + 1] = a2.y;
             e[j] = e2.x; e[j + 1] = e2.y;
             dk[j] = dk2.x; dk[j + 1] = dk2.y;
@@ -210,8 +190,8 @@ template <bool kDsOnly, bool kRagged>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
-              const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ totals,
-              const __nv_bfloat16 *__restrict__ f_gmem,
+              const __grid_constant__ CUtensorMap map_saved, const __grid_constant__ CUtensorMap map_o_raw,
+              const __grid_constant__ CUtensorMap map_f_raw, const float *__restrict__ totals,
               const float *__restrict__ dSN, __nv_bfloat16 *__restrict__ d_o, __nv_bfloat16 *__restrict__ d_f,
               __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N, int NC, StatusBlock *status)
 {
@@ -224,7 +204,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     uint8_t *dsbuf = smem + kOffDS;
     uint8_t *pbuf = smem + kOffP;
     uint8_t *dpbuf = smem + kOffDP;
-    uint32_t *fscr = reinterpret_cast<uint32_t *>(smem + kOffF);
+    const __nv_bfloat16 *oraw = reinterpret_cast<const __nv_bfloat16 *>(smem + kOffRawO);
+    const __nv_bfloat16 *fraw = reinterpret_cast<const __nv_bfloat16 *>(smem + kOffRawF);
+    uint8_t *vbuf = smem + kOffV;
     float *rr = reinterpret_cast<float *>(smem + kOffR);
     float *xa = reinterpret_cast<float *>(smem + kOffX);
     float *xe = xa + 128;
@@ -237,9 +219,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->stage_read[s], kE3Threads);
             mbar_init(&ctl->t_done[s], kTransformThreads);
         }
+        mbar_init(&ctl->vfull, 1);
+        mbar_init(&ctl->rawfull, 1);
+        mbar_init(&ctl->raw_read, kE3Threads);
         mbar_init(&ctl->sfull, 1);
         mbar_init(&ctl->m_done, kE1Threads);
         mbar_init(&ctl->barX, 1);
@@ -259,6 +243,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         tma_prefetch_desc(&map_i);
         tma_prefetch_desc(&map_dy);
         tma_prefetch_desc(&map_saved);
+        tma_prefetch_desc(&map_o_raw);
+        tma_prefetch_desc(&map_f_raw);
     }
     if (warp == 0) tmem_alloc(&ctl->tmem_base, kTmemCols);
     tc_fence_before_sync();
@@ -414,26 +400,19 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         const int half = (warp - kWarpE3) >> 2;                      // half of the chunk: local times [32 * half, +32)
         const uint32_t tl = tmem + lane_base;
         PT_DECL
-        for (int it = 0; it < NC; ++it) {
-            const int c = NC - 1 - it, s = it % kStages;
-            if (kDsOnly) {                                           // nothing to output: just hand the stage back
-                mbar_wait(&ctl->barY2, it & 1, abort_flag);
-                mbar_arrive(&ctl->stage_read[s]);
-                continue;
-            }
+        for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
+            const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
-            const uint8_t *qtile = smem + s * kStageBytes, *ktile = qtile + kTile;
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
-            uint32_t *fs = fscr + (tid - kWarpE3 * 32);
-            load_f_strip(f_gmem + row0 * kD + krow, 32 * half, n_valid, fs);
+            mbar_wait(&ctl->rawfull, it & 1, abort_flag);
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
             PT_MARK(0)
             tc_fence_after_sync();
             float asum, esum;
             PT_STAMP(status, 14, tid == kWarpE3 * 32 && it == 16)
-            if (half) phase_main<true>(tl, qtile, ktile, krow, fs, d_o + row0 * kD + krow, n_valid, asum, esum);
-            else      phase_main<false>(tl, qtile, ktile, krow, fs, d_o + row0 * kD + krow, n_valid, asum, esum);
-            mbar_arrive(&ctl->stage_read[s]);
+            if (half) phase_main<true, kRagged>(tl, oraw, fraw, krow, d_o + row0 * kD + krow, n_valid, asum, esum);
+            else      phase_main<false, kRagged>(tl, oraw, fraw, krow, d_o + row0 * kD + krow, n_valid, asum, esum);
+            mbar_arrive(&ctl->raw_read);
             if (half) xa[krow] = asum; else xe[krow] = esum;
             tmem_wait_st();
             tc_fence_before_sync();
@@ -504,9 +483,20 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 for (int b = 0; b < 2; ++b) {
                     tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
                     tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + 3 * kTile + b * kSlab, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
                 }
+                for (int b = 0; b < 2; ++b)
+                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
+            };
+            auto issue_v = [&](int it) {
+                const int c = NC - 1 - it;
+                mbar_arrive_expect_tx(&ctl->vfull, kTile);
+                for (int b = 0; b < 2; ++b) tma_load_3d(vbuf + b * kSlab, &map_i, &ctl->vfull, 64 * b, c * kC, u);
+            };
+            auto issue_raw = [&](int it) {
+                const int c = NC - 1 - it;
+                mbar_arrive_expect_tx(&ctl->rawfull, 2 * kTile);
+                tma_load_3d(smem + kOffRawO, &map_o_raw, &ctl->rawfull, 0, c * kC, u);
+                tma_load_3d(smem + kOffRawF, &map_f_raw, &ctl->rawfull, 0, c * kC, u);
             };
             auto issue_state = [&](int it) {
                 const int c = NC - 1 - it;
@@ -515,21 +505,28 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, u * NC + c);
             };
             issue_stage(0);
-            if (!kDsOnly) issue_state(0);
+            if (!kDsOnly) {
+                issue_v(0);
+                issue_state(0);
+                issue_raw(0);
+            }
             if (NC > 1) issue_stage(1);
+            // Every buffer is refilled as soon as its last reader of chunk `it` is done; the waits below are in
+            // the order in which those readers finish.
             for (int it = 0; it + 1 < NC; ++it) {
-                // chunk `it` is finished with S' once its products and its R are done ...
-                mbar_wait(&ctl->barY2, it & 1, abort_flag);
                 if (!kDsOnly) {
-                    mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
-                    issue_state(it + 1);
-                    PT_STAMP(status, 22, it == 15)
+                    mbar_wait(&ctl->barX, it & 1, abort_flag);       // dA = dY V^T ...
+                    mbar_wait(&ctl->barY1, it & 1, abort_flag);      // ... and dKs_inter^T = dS'' V^T have read v
+                    issue_v(it + 1);
+                    mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);   // R has read S' ...
                 }
-                // ... and with its stage once the output warps have read Qs and Ks
-                if (it + 2 < NC) {
-                    mbar_wait(&ctl->stage_read[it % kStages], (it / kStages) & 1, abort_flag);
-                    issue_stage(it + 2);
-                    PT_STAMP(status, 0, it == 14) PT_STAMP(status, 21, it == 16)
+                mbar_wait(&ctl->barY2, it & 1, abort_flag);          // ... and so have the chunk's products;
+                if (!kDsOnly) issue_state(it + 1);
+                if (it + 2 < NC) issue_stage(it + 2);                // o, f, dy of the stage are free as well
+                PT_STAMP(status, 0, it == 14) PT_STAMP(status, 21, it == 16) PT_STAMP(status, 22, it == 15)
+                if (!kDsOnly) {
+                    mbar_wait(&ctl->raw_read, it & 1, abort_flag);   // the output warps are done with raw o, f
+                    issue_raw(it + 1);
                 }
             }
         }
@@ -544,8 +541,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         const uint32_t sm0 = smem_u32(smem);
         const uint64_t dqk0 = smem_desc_sw128(sm0, 16, 1024), dqm0 = smem_desc_sw128(sm0, kSlab, 1024);
         const uint64_t dfk0 = smem_desc_sw128(sm0 + kTile, 16, 1024), dfm0 = smem_desc_sw128(sm0 + kTile, kSlab, 1024);
-        const uint64_t dvk0 = smem_desc_sw128(sm0 + 2 * kTile, 16, 1024);
-        const uint64_t dgk0 = smem_desc_sw128(sm0 + 3 * kTile, 16, 1024), dgm0 = smem_desc_sw128(sm0 + 3 * kTile, kSlab, 1024);
+        const uint64_t dvk = smem_desc_sw128(smem_u32(vbuf), 16, 1024);
+        const uint64_t dgk0 = smem_desc_sw128(sm0 + 2 * kTile, 16, 1024), dgm0 = smem_desc_sw128(sm0 + 2 * kTile, kSlab, 1024);
         const uint64_t dsk = smem_desc_sw128(smem_u32(sbuf), 16, 1024);
         const uint64_t ddsk = smem_desc_sw128(smem_u32(dsbuf), 16, 1024), ddsm = smem_desc_sw128(smem_u32(dsbuf), kStateSlab, 1024);
         const uint64_t dpm = smem_desc_sw128(smem_u32(pbuf), kSlab, 1024);
@@ -557,12 +554,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             for (int it = 0; it < NC; ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
-                const uint64_t dqk = dqk0 + so, dqm = dqm0 + so, dfk = dfk0 + so, dvk = dvk0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
+                const uint64_t dqk = dqk0 + so, dqm = dqm0 + so, dfk = dfk0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
                 mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
                 PT_MARK(0)
                 mbar_wait(&ctl->m_done, it & 1, abort_flag);          // dS'' in TMEM
                 if (it > 0 && !kDsOnly) mbar_wait(&ctl->pd_ready, (it - 1) & 1, abort_flag);   // A, dA of the previous chunk read out
+                if (!kDsOnly) mbar_wait(&ctl->vfull, it & 1, abort_flag);
                 PT_MARK(1)
                 PT_STAMP(status, 3, it == 16)
                 tc_fence_after_sync();
@@ -590,10 +588,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
-                const uint64_t dfk = dfk0 + so, dvk = dvk0 + so;
+                const uint64_t dfk = dfk0 + so;
                 mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->m_done, it & 1, abort_flag);          // bf16 dS'' in shared memory
+                mbar_wait(&ctl->vfull, it & 1, abort_flag);
                 PT_MARK(0)
                 if (it > 0) {
                     mbar_wait(&ctl->acc_free1, (it - 1) & 1, abort_flag);
@@ -654,7 +653,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int last = ((NC - 1 - s) / kStages) * kStages + s;
             if (s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
         }
-        if (!kDsOnly) mbar_wait_drain(&ctl->sfull, (NC - 1) & 1, 20000000ull);
+        if (!kDsOnly) {
+            mbar_wait_drain(&ctl->sfull, (NC - 1) & 1, 20000000ull);
+            mbar_wait_drain(&ctl->vfull, (NC - 1) & 1, 20000000ull);
+            mbar_wait_drain(&ctl->rawfull, (NC - 1) & 1, 20000000ull);
+        }
     }
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
@@ -695,9 +698,10 @@ int segments_for(uint64_t U, int N, int NC);     // chunk_tc_fwd.cu
 
 static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly)
 {
-    CUtensorMap mo, mf, mi, mg, ms;
+    CUtensorMap mo, mf, mi, mg, ms, mor, mfr;
     if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
-        !make_map(&mg, a.dy, U, N, kC) || !make_map(&ms, a.states, U * NC, kD, kD))
+        !make_map(&mg, a.dy, U, N, kC) || !make_map(&ms, a.states, U * NC, kD, kD) ||
+        !make_map_plain(&mor, a.o, U, N, kC) || !make_map_plain(&mfr, a.f, U, N, kC))
         return cudaErrorInvalidValue;
     const bool ragged = N % kC != 0;
     auto kernel = kDsOnly ? (ragged ? tc_bwd_kernel<true, true> : tc_bwd_kernel<true, false>)
@@ -705,9 +709,9 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
-        mo, mf, mi, mg, ms,
+        mo, mf, mi, mg, ms, mor, mfr,
         reinterpret_cast<const float *>(reinterpret_cast<const char *>(a.states) + U * NC * kSavedStateBytes),
-        static_cast<const __nv_bfloat16 *>(a.f), dSN, static_cast<__nv_bfloat16 *>(a.d_o),
+        dSN, static_cast<__nv_bfloat16 *>(a.d_o),
         static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status);
     return cudaGetLastError();
 }

@@ -197,5 +197,19 @@ inline bool make_map(CUtensorMap *m, const void *base, uint64_t U, uint64_t rows
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same tensor as whole-width tiles of [box_rows][128] without swizzle (rows of 256 bytes, in order).
+inline bool make_map_plain(CUtensorMap *m, const void *base, uint64_t U, uint64_t rows, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {128, rows, U};
+    cuuint64_t strides[2] = {256, rows * 256};
+    cuuint32_t box[3] = {128, box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace tc
 }  // namespace hgrn2
