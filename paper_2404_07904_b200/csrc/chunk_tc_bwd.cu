@@ -37,8 +37,8 @@
 //   Y1: dKs_inter^T | dV^T = dS''^T Ks^T   (needs the previous chunk's dKs_inter^T, dV^T read out)
 //   Y2: dQs^T | dKs_intra^T | dV^T += dY^T A   (needs tril(A), tril(dA), S', and the parked values consumed)
 //
-// Tensor-memory plan (512 columns, no spare): dS [0,128); A [128,192), dA [192,256) in the M = 64
-// layout; dQs^T [256,320); dKs_intra^T [320,384); dKs_inter^T [384,448); dV^T [448,512).
+// Tensor-memory plan (512 columns, no spare): dS [0,128); A [128,192) in lanes 0..63 and dA [192,256) in
+// lanes 64..127 (products of the stacked operand (Qs; dY), M = 128); dQs^T [256,320); dKs_intra^T [320,384); dKs_inter^T [384,448); dV^T [448,512).
 #include "tc_chunk.cuh"
 
 namespace hgrn2 {
@@ -55,7 +55,11 @@ constexpr int kWarpLoad = kWarpO + kOWarps, kWarpMmaX = kWarpLoad + 1, kWarpMmaY
 constexpr int kThreads = (kWarpMmaY2 + 1) * 32;
 
 constexpr int kStages = 2;
-constexpr uint32_t kStageBytes = 3 * kTile;                       // q, f, dy: free again when the chunk's products are done
+constexpr uint32_t kStageBytes = 3 * kTile;                       // q, dy, f: free again when the chunk's products are done
+// Stage layout: [q slab 0][dy slab 0][q slab 1][dy slab 1][f slab 0][f slab 1].  With the slabs of q and dy
+// interleaved, (Qs; dY) also reads as ONE 128-row K-major operand whose slabs are 16 KB apart.
+constexpr uint32_t kSS = 2 * kSlab;                               // distance between the two slabs of the q and dy tiles
+constexpr uint32_t kOffQ = 0, kOffG = kSlab, kOffK = 2 * kTile;
 constexpr uint32_t kOffV = kStages * kStageBytes;                 // v: one buffer, free when X and Y1 of the chunk are done
 constexpr uint32_t kOffS = kOffV + kTile;                         // S' (bf16, from the forward)
 constexpr uint32_t kOffDS = kOffS + kStateTile;                   // bf16 copy of dS''
@@ -78,8 +82,8 @@ struct Ctl {
     uint64_t t_done[kStages];     // T -> M, E1
     uint64_t sfull;               // TMA (saved S') -> E1, M
     uint64_t m_done;              // E1 -> M: dS'' is in TMEM and in shared memory
-    uint64_t barX;                // tcgen05.commit -> E1: dS' update, A, dA complete
-    uint64_t pd_ready;            // E1 -> M: tril(A), tril(dA) are in shared memory
+    uint64_t barX;                // tcgen05.commit -> E1, E3, L: dS' update, A, dA complete
+    uint64_t pd_ready;            // E3 -> M: tril(A), tril(dA) are in shared memory
     uint64_t barY1;               // tcgen05.commit -> E1: dS'' copy no longer read
     uint64_t barY2;               // tcgen05.commit -> E3, L: every product of the chunk complete
     uint64_t r_ready[2];          // E1 -> O, L: R of the chunk is in shared memory, S' no longer read by threads
@@ -227,7 +231,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->sfull, 1);
         mbar_init(&ctl->m_done, kE1Threads);
         mbar_init(&ctl->barX, 1);
-        mbar_init(&ctl->pd_ready, kE1Threads);
+        mbar_init(&ctl->pd_ready, kE3Threads);
         mbar_init(&ctl->barY1, 1);
         mbar_init(&ctl->barY2, 1);
         mbar_init(&ctl->r_ready[0], kE1Threads);
@@ -268,9 +272,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int n_valid = kRagged ? N - c * kC : kC;
             // Pm and E of the chunk are not kept: the backward takes them from what the forward saved
             if (n_valid >= kC) {
-                transform_stream<true>(qbuf, qbuf + kTile, nullptr, nullptr, nullptr, nullptr, kC, tid);
+                transform_stream<true, kSS, kSlab>(qbuf + kOffQ, qbuf + kOffK, nullptr, nullptr, nullptr, nullptr, kC, tid);
             } else {
-                transform_stream<false>(qbuf, qbuf + kTile, nullptr, nullptr, nullptr, nullptr, n_valid, tid);
+                transform_stream<false, kSS, kSlab>(qbuf + kOffQ, qbuf + kOffK, nullptr, nullptr, nullptr, nullptr, n_valid, tid);
             }
             fence_proxy_async_smem();
             mbar_arrive(&ctl->t_done[s]);
@@ -295,7 +299,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 ee_c = __ldg(tot_u + (size_t)(NC - 2 - it) * 2 * kD + kD);
             }
             if (it > 0) {
-                mbar_wait(&ctl->barY1, (it - 1) & 1, abort_flag);    // dS' update done, dsbuf no longer read
+                mbar_wait(&ctl->barX, (it - 1) & 1, abort_flag);     // dS' of the previous chunk is complete
+                mbar_wait(&ctl->barY1, (it - 1) & 1, abort_flag);    // its dS'' copy is no longer read
                 tc_fence_after_sync();
             }
             PT_MARK(1)
@@ -336,28 +341,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             PT_STAMP(status, 6, tid == kWarpE1 * 32 && it == 16)
             if (kDsOnly) continue;                                   // state-gradient chain only
 
-            // ---- tril(A), tril(dA) -> operand slabs
-            mbar_wait(&ctl->barX, it & 1, abort_flag);
-            if (it > 0) mbar_wait(&ctl->barY2, (it - 1) & 1, abort_flag);   // the previous chunk's products have read P, dP
-            PT_MARK(3)
-            tc_fence_after_sync();
-            PT_STAMP(status, 7, tid == kWarpE1 * 32 && it == 16)
-#pragma unroll 1
-            for (int w = 0; w < 2; ++w) {
-                const uint32_t col = w ? kColDA : kColA;
-                uint8_t *dst = w ? dpbuf : pbuf;
-                tril_to_slab(tmem + lane_base + col, dst, sub, 0, lane);
-                tril_to_slab(tmem + lane_base + col + 32, dst, sub, 1, lane);
-            }
-            fence_proxy_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&ctl->pd_ready);
-            PT_MARK(4)
-            PT_STAMP(status, 8, tid == kWarpE1 * 32 && it == 16)
-
             // ---- R_k = sum_v dS''[k,v] S'[k,v] from the two bf16 copies
             mbar_wait(&ctl->sfull, it & 1, abort_flag);
-            PT_MARK(5)
+            PT_MARK(3)
             float racc = 0.f;
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
@@ -374,10 +360,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
             rr[(it & 1) * 128 + krow] = racc;
             mbar_arrive(&ctl->r_ready[it & 1]);
-            PT_MARK(6)
+            PT_MARK(4)
             PT_STAMP(status, 9, tid == kWarpE1 * 32 && it == 16)
         }
-        PT_DUMP(status, 2, 7, tid == kWarpE1 * 32)
+        PT_DUMP(status, 2, 5, tid == kWarpE1 * 32)
 
         // dS_0 = Diag(Pm of chunk 0) dS'
         mbar_wait(&ctl->barY2, (NC - 1) & 1, abort_flag);
@@ -404,9 +390,23 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
             const size_t row0 = (size_t)u * N + (size_t)c * kC;
+            // ---- tril(A), tril(dA) -> operand slabs, one 32 x 32 block per warp.  The
+            // previous chunk's products have read the slabs: this role waited for them before its outputs.
+            mbar_wait(&ctl->barX, it & 1, abort_flag);
+            PT_MARK(0)
+            PT_STAMP(status, 7, tid == kWarpE3 * 32 && it == 16)
+            tc_fence_after_sync();
+            // rows of A sit in lanes 0..63, rows of dA in lanes 64..127: a warp converts 32 rows x 32 columns
+            tril_row_block(tl + (sub < 2 ? kColA : kColDA) + 32 * half, sub < 2 ? pbuf : dpbuf, krow & 63, half);
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->pd_ready);
+            PT_MARK(1)
+            PT_STAMP(status, 8, tid == kWarpE3 * 32 && it == 16)
+            // ---- outputs
             mbar_wait(&ctl->rawfull, it & 1, abort_flag);
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
-            PT_MARK(0)
+            PT_MARK(2)
             tc_fence_after_sync();
             float asum, esum;
             PT_STAMP(status, 14, tid == kWarpE3 * 32 && it == 16)
@@ -418,10 +418,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_free1);
             mbar_arrive(&ctl->parked);
-            PT_MARK(1)
+            PT_MARK(3)
             PT_STAMP(status, 15, tid == kWarpE3 * 32 && it == 16)
         }
-        PT_DUMP(status, 9, 2, tid == kWarpE3 * 32)
+        PT_DUMP(status, 7, 4, tid == kWarpE3 * 32)
     } else if (warp < kWarpLoad) {
         // ================= O: d_i, and d_f completed from the parked values =================
         const uint32_t tl = tmem + lane_base;
@@ -481,11 +481,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 uint8_t *st = smem + s * kStageBytes;
                 mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
                 for (int b = 0; b < 2; ++b) {
-                    tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kOffQ + b * kSS, &map_o, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kOffK + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
                 }
                 for (int b = 0; b < 2; ++b)
-                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kOffG + b * kSS, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
             };
             auto issue_v = [&](int it) {
                 const int c = NC - 1 - it;
@@ -532,29 +532,29 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         }
     } else if (lane == 0) {
         // ================= MX, MY1, MY2: MMA issue =================
-        constexpr uint32_t idA = idesc_bf16(64, 64, 0, 0);        // Qs x Ks^T, dY x V^T (all K-major)
         constexpr uint32_t idDS = idesc_bf16(128, 128, 1, 1);     // Qs^T (MN-major) x dY (MN-major)
         constexpr uint32_t idKK = idesc_bf16(128, 64, 0, 0);      // dS'' x V^T, S' x dY^T (all K-major)
         constexpr uint32_t idMK = idesc_bf16(128, 64, 1, 0);      // dS''^T (MN) x Ks^T (K);  Ks^T (MN) x dP^T (K)
         constexpr uint32_t idMM = idesc_bf16(128, 64, 1, 1);      // Qs^T (MN) x dP (MN);  dY^T (MN) x P (MN)
         // descriptors once; K steps and stage changes only add to the 14-bit start-address field
         const uint32_t sm0 = smem_u32(smem);
-        const uint64_t dqk0 = smem_desc_sw128(sm0, 16, 1024), dqm0 = smem_desc_sw128(sm0, kSlab, 1024);
-        const uint64_t dfk0 = smem_desc_sw128(sm0 + kTile, 16, 1024), dfm0 = smem_desc_sw128(sm0 + kTile, kSlab, 1024);
+        const uint64_t dqk0 = smem_desc_sw128(sm0 + kOffQ, 16, 1024), dqm0 = smem_desc_sw128(sm0 + kOffQ, kSS, 1024);
+        const uint64_t dfk0 = smem_desc_sw128(sm0 + kOffK, 16, 1024), dfm0 = smem_desc_sw128(sm0 + kOffK, kSlab, 1024);
         const uint64_t dvk = smem_desc_sw128(smem_u32(vbuf), 16, 1024);
-        const uint64_t dgk0 = smem_desc_sw128(sm0 + 2 * kTile, 16, 1024), dgm0 = smem_desc_sw128(sm0 + 2 * kTile, kSlab, 1024);
+        const uint64_t dgk0 = smem_desc_sw128(sm0 + kOffG, 16, 1024), dgm0 = smem_desc_sw128(sm0 + kOffG, kSS, 1024);
         const uint64_t dsk = smem_desc_sw128(smem_u32(sbuf), 16, 1024);
         const uint64_t ddsk = smem_desc_sw128(smem_u32(dsbuf), 16, 1024), ddsm = smem_desc_sw128(smem_u32(dsbuf), kStateSlab, 1024);
         const uint64_t dpm = smem_desc_sw128(smem_u32(pbuf), kSlab, 1024);
         const uint64_t ddpk = smem_desc_sw128(smem_u32(dpbuf), 16, 1024), ddpm = smem_desc_sw128(smem_u32(dpbuf), kSlab, 1024);
         auto kmaj = [](int kk) { return (uint64_t)(((kk >> 2) * kSlab + (kk & 3) * 32) >> 4); };          // [64][128] tile
+        auto kmaj_i = [](int kk) { return (uint64_t)(((kk >> 2) * kSS + (kk & 3) * 32) >> 4); };          // interleaved q / dy tile
         auto kmaj_s = [](int kk) { return (uint64_t)(((kk >> 2) * kStateSlab + (kk & 3) * 32) >> 4); };   // [128][128] tile
         PT_DECL
         if (warp == kWarpMmaX) {
             for (int it = 0; it < NC; ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
-                const uint64_t dqk = dqk0 + so, dqm = dqm0 + so, dfk = dfk0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
+                const uint64_t dqk = dqk0 + so, dqm = dqm0 + so, dfk = dfk0 + so, dgm = dgm0 + so;
                 mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
                 PT_MARK(0)
@@ -572,12 +572,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     mma_commit(&ctl->barY1);
                     mma_commit(&ctl->barY2);
                 } else {
+                    // (Qs; dY) as one 128-row operand: (Qs; dY) Ks^T has A in lanes 0..63 and (Qs; dY) V^T has dA
+                    // in lanes 64..127 (the other halves are not used), so every lane carries a row to mask
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)          // A = Qs Ks^T
-                        mma_bf16_ss(tmem + kColA, dqk + kmaj(kk), dfk + kmaj(kk), idA, kk > 0);
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_bf16_ss(tmem + kColA, dqk + kmaj_i(kk), dfk + kmaj(kk), idKK, kk > 0);
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)          // dA = dY V^T
-                        mma_bf16_ss(tmem + kColDA, dgk + kmaj(kk), dvk + kmaj(kk), idA, kk > 0);
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_bf16_ss(tmem + kColDA, dqk + kmaj_i(kk), dvk + kmaj(kk), idKK, kk > 0);
                     mma_commit(&ctl->barX);
                 }
                 PT_MARK(2)
@@ -630,7 +632,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     mma_bf16_ss(tmem + kColDQ, dfm + (uint64_t)(kk * 128), ddpk + (uint64_t)(kk * 2), idMK, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)              //        + S' dY^T
-                    mma_bf16_ss(tmem + kColDQ, dsk + kmaj_s(kk), dgk + kmaj(kk), idKK, 1);
+                    mma_bf16_ss(tmem + kColDQ, dsk + kmaj_s(kk), dgk + kmaj_i(kk), idKK, 1);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
                     mma_bf16_ss(tmem + kColDKi, dqm + (uint64_t)(kk * 128), ddpm + (uint64_t)(kk * 128), idMM, kk > 0);

@@ -79,13 +79,14 @@ __device__ __forceinline__ uint4 pack8(const uint32_t *r)
 // 32..63) of the chunk are left in pm[128] and ee[128] (shared memory) and / or pm_g[128], ee_g[128]
 // (global memory); either pair may be null.  Rows at or beyond n_valid are the neutral token
 // f = 1, o = 0.
-template <bool kFull, bool kUp>
+template <bool kFull, bool kUp, uint32_t kQSlabStride, uint32_t kFSlabStride>
 __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, float *tot, float *tot_g, int n_valid,
                                                int p)
 {
     const int col = 2 * p;
     const int jch = (col & 63) >> 3;
-    const uint32_t base = (col >> 6) * kSlab + (col & 7) * 2;
+    const uint32_t base = (col >> 6) * kQSlabStride + (col & 7) * 2;
+    if (kFSlabStride != kQSlabStride && (col >> 6)) fbuf -= kQSlabStride - kFSlabStride;   // offsets below are the q tile's
     uint32_t xo[8];
 #pragma unroll
     for (int jj = 0; jj < 8; ++jj) xo[jj] = base + ((jch ^ jj) << 4);
@@ -136,12 +137,13 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
     if (tot_g) *reinterpret_cast<float2 *>(tot_g + col) = t2;
 }
 
-template <bool kFull>
+// kQSlabStride, kFSlabStride: distance in bytes between the two 64-column slabs of the q tile and of the f tile.
+template <bool kFull, uint32_t kQSlabStride = kSlab, uint32_t kFSlabStride = kSlab>
 __device__ __forceinline__ void transform_stream(uint8_t *qbuf, uint8_t *fbuf, float *pm, float *ee, float *pm_g,
                                                  float *ee_g, int n_valid, int tid)
 {
-    if (tid >> 6) transform_half<kFull, true>(qbuf, fbuf, ee, ee_g, n_valid, tid & 63);
-    else          transform_half<kFull, false>(qbuf, fbuf, pm, pm_g, n_valid, tid & 63);
+    if (tid >> 6) transform_half<kFull, true, kQSlabStride, kFSlabStride>(qbuf, fbuf, ee, ee_g, n_valid, tid & 63);
+    else          transform_half<kFull, false, kQSlabStride, kFSlabStride>(qbuf, fbuf, pm, pm_g, n_valid, tid & 63);
 }
 
 // Causal mask + bf16 of 32 columns (32 * half ...) of one 64 x 64 fp32 accumulator in the M = 64
@@ -161,6 +163,30 @@ __device__ __forceinline__ void tril_to_slab(uint32_t taddr, uint8_t *dstbuf, in
             for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? r[8 * j + q] : 0u;
             *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = pack8(x);
         }
+    }
+}
+
+// Causal mask + bf16 of columns [32 * half, +32) of row t of a 64 x 64 fp32 accumulator whose rows sit one per
+// TMEM lane (taddr = this thread's lane, first of the 32 columns) into a K-major slab.  The 32 threads of the
+// warp hold 32 consecutive rows; a block that lies wholly above the diagonal is zero and is not read.
+__device__ __forceinline__ void tril_row_block(uint32_t taddr, uint8_t *dstbuf, int t, int half)
+{
+    if (32 * half > (t | 31)) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
+    uint32_t r[32];
+    tmem_ld32(taddr, r);
+    tmem_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int s0 = 32 * half + 8 * j;
+        uint32_t x[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) x[q] = (s0 + q <= t) ? r[8 * j + q] : 0u;
+        *reinterpret_cast<uint4 *>(dstbuf + slab_chunk_off(t, 4 * half + j)) = pack8(x);
     }
 }
 
