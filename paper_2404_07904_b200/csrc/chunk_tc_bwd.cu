@@ -619,10 +619,15 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
                 const uint64_t dqm = dqm0 + so, dfm = dfm0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
                 mbar_wait(&ctl->pd_ready, it & 1, abort_flag);        // tril(A), tril(dA); implies X and T of the chunk
-                mbar_wait(&ctl->sfull, it & 1, abort_flag);
+                mbar_wait(&ctl->barY1, it & 1, abort_flag);           // dV^T += ... must follow dV^T = ...
                 PT_MARK(0)
                 PT_STAMP(status, 11, it == 16)
-                mbar_wait(&ctl->barY1, it & 1, abort_flag);           // dV^T += ... must follow dV^T = ...
+                tc_fence_after_sync();
+                // dV^T first: it does not touch the columns that still hold the previous chunk's parked values
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)              // dV^T += dY^T A
+                    mma_bf16_ss(tmem + kColDV, dgm + (uint64_t)(kk * 128), dpm + (uint64_t)(kk * 128), idMM, 1);
+                mbar_wait(&ctl->sfull, it & 1, abort_flag);
                 if (it > 0) mbar_wait(&ctl->acc_free2, (it - 1) & 1, abort_flag);
                 PT_MARK(1)
                 PT_STAMP(status, 12, it == 16)
@@ -636,9 +641,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
                     mma_bf16_ss(tmem + kColDKi, dqm + (uint64_t)(kk * 128), ddpm + (uint64_t)(kk * 128), idMM, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)              // dV^T += dY^T A
-                    mma_bf16_ss(tmem + kColDV, dgm + (uint64_t)(kk * 128), dpm + (uint64_t)(kk * 128), idMM, 1);
                 mma_commit(&ctl->barY2);
                 PT_MARK(2)
                 PT_STAMP(status, 13, it == 16)
