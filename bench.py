@@ -226,6 +226,31 @@ def run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks,
               "roofline": {"bound": "hbm", "kernel": "hgrn2_step", "achieved": dec_gbps, "peak": peaks["hbm_gbs"],
                            "unit": "GB/s", "frac": dec_gbps / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES["step"],
                            "peak_source": f"of {peak_kind}", "frac_nominal": dec_gbps / NOMINAL["hbm_gbs"]}}
+    # ---- the same tokens, 8 per launch (hgrn2_step_multi): the state crosses HBM once per 8 tokens -------
+    TM = 8
+    if T >= TM:
+        nl = T // TM
+        seq = {k: gates[k][:nl * TM].reshape(nl, TM, wd.B, wd.H, -1).permute(0, 2, 3, 1, 4).contiguous() for k in gates}
+        ym = torch.empty((nl, wd.B, wd.H, TM, wd.dv), dtype=bf, device=dev)
+        S.copy_(torch.from_numpy(S0))
+
+        def decode_multi():
+            for l in range(nl):
+                binding.hgrn2_step_multi(seq["o"][l], seq["f"][l], seq["i"][l], S, y=ym[l])
+
+        binding.hgrn2_step_multi(seq["o"][0], seq["f"][0], seq["i"][0], S, y=ym[0])
+        S.copy_(torch.from_numpy(S0))
+        ms_l = max_over_ranks(timed(decode_multi, 1)) / nl
+        if rank == 0:       # same arithmetic in the same order: identical to the one-token calls
+            same = torch.equal(ym.permute(0, 3, 1, 2, 4).reshape(nl * TM, wd.B, wd.H, wd.dv), yd[:nl * TM])
+            assert same, "multi-token step differs from single steps"
+        gate_bytes = decode_bytes(wd) - 2 * wd.B * wd.H * wd.dk * wd.dv * 4
+        mb = 2 * wd.B * wd.H * wd.dk * wd.dv * 4 + TM * gate_bytes
+        decode["multi_token"] = {"tokens_per_launch": TM, "launches": nl, "us_per_launch": ms_l * 1e3,
+                                 "us_per_token_step": ms_l * 1e3 / TM,
+                                 "tokens_per_s": world * wd.B * TM / (ms_l * 1e-3),
+                                 "achieved_GBps": mb / (ms_l * 1e-3) / 1e9,
+                                 "algorithmic_bytes_per_launch": mb}
     if args.only == "decode" and rank == 0:
         print(json.dumps({"only": "decode", "decode": decode}), flush=True)
     return decode

@@ -154,6 +154,17 @@ hgrn2_status hgrn2_bwd_static_scratch(const hgrn2_desc *desc, const void *o, con
 hgrn2_status hgrn2_step(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
                         float *S, void *y, void *cuda_stream);
 
+/* desc->N successive decode steps in one launch (Eq. 3 applied N times; multi-token or speculative decoding):
+ * the state of a unit is read once, stays on chip across the tokens and is written once, so the state traffic
+ * per token falls N-fold (constant-size state, Section 1).  Results equal N calls of hgrn2_step bit for bit.
+ *   o, f [B][H][N][dk], i [B][H][N][dv] in (desc->io), device memory, 16-byte aligned, caller-owned
+ *   S    [B][H][dk][dv] float32, updated in place to the state after the last token
+ *   y    [B][H][N][dv] out (desc->io), y_t computed from the state after token t
+ * Supported: dk = dv in {64, 128}; anything else returns HGRN2_ERR_UNSUPPORTED.  N = 0 is a no-op.
+ * Errors: HGRN2_ERR_INVALID_ARG (null pointer, bad descriptor), HGRN2_ERR_ALIGNMENT, HGRN2_ERR_CUDA (launch). */
+hgrn2_status hgrn2_step_multi(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                              float *S, void *y, void *cuda_stream);
+
 /* Reads the device status word of `ws` (a device pointer) with a blocking copy.  Call it
  * after synchronising the stream the work ran on.  Returns HGRN2_OK, HGRN2_ERR_TIMEOUT,
  * HGRN2_ERR_DOMAIN, or HGRN2_ERR_CUDA if the copy itself failed. */

@@ -26,7 +26,7 @@ STATUS_NAMES = {
 # Every symbol include/hgrn2.h declares.
 EXPORTS = (
     "hgrn2_saved_bytes", "hgrn2_workspace_bytes", "hgrn2_fwd", "hgrn2_bwd", "hgrn2_step",
-    "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path", "hgrn2_bwd_static_scratch",
+    "hgrn2_step_multi", "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path", "hgrn2_bwd_static_scratch",
 )
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
@@ -77,6 +77,8 @@ def load() -> ctypes.CDLL:
     lib.hgrn2_bwd_static_scratch.argtypes = [dp] + [vp] * 12
     lib.hgrn2_step.restype = ctypes.c_int
     lib.hgrn2_step.argtypes = [dp] + [vp] * 6
+    lib.hgrn2_step_multi.restype = ctypes.c_int
+    lib.hgrn2_step_multi.argtypes = [dp] + [vp] * 6
     _lib = lib
     return lib
 
@@ -211,6 +213,19 @@ def hgrn2_step(o, f, i, S, *, y=None, stream=None):
         y = torch.empty((B, H, dv), dtype=o.dtype, device=o.device)
     code = load().hgrn2_step(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S), _ptr(y), _stream(stream))
     _check(code, "hgrn2_step")
+    return y
+
+
+def hgrn2_step_multi(o, f, i, S, *, y=None, stream=None):
+    """T successive decode steps in one launch on [B, H, T, d] gates; S [B, H, dk, dv] float32 is updated in
+    place to the state after the last token.  Returns y [B, H, T, dv]."""
+    B, H, T, dk = o.shape
+    dv = i.shape[-1]
+    desc = make_desc(B, H, T, dk, dv, _io_code(o))
+    if y is None:
+        y = torch.empty((B, H, T, dv), dtype=o.dtype, device=o.device)
+    code = load().hgrn2_step_multi(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S), _ptr(y), _stream(stream))
+    _check(code, "hgrn2_step_multi")
     return y
 
 

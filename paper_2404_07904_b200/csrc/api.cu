@@ -214,6 +214,23 @@ hgrn2_status hgrn2_step(const hgrn2_desc *desc, const void *o, const void *f, co
     return launch_step(a) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
 }
 
+hgrn2_status hgrn2_step_multi(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                              float *S, void *y, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    if (!step_multi_supported(desc->dk, desc->dv)) return HGRN2_ERR_UNSUPPORTED;
+    const bool empty = (size_t)desc->B * desc->H * desc->N == 0;
+    if (empty) return HGRN2_OK;                                  // no token: the state stays as it is
+    const void *req[] = {o, f, i, S, y};
+    hgrn2_status st = check_ptrs(req, 5, nullptr, 0);
+    if (st != HGRN2_OK) return st;
+    StepArgs a;
+    a.B = desc->B; a.H = desc->H; a.dk = desc->dk; a.dv = desc->dv; a.io = desc->io; a.T = desc->N;
+    a.o = o; a.f = f; a.i = i; a.S = S; a.y = y;
+    a.stream = static_cast<cudaStream_t>(cuda_stream);
+    return launch_step_multi(a) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
 hgrn2_status hgrn2_poll(const void *ws)
 {
     if (!ws) return HGRN2_ERR_INVALID_ARG;

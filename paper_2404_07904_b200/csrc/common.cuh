@@ -61,6 +61,7 @@ struct SeqArgs {
 
 struct StepArgs {
     int B, H, dk, dv, io;
+    int T = 1;             // tokens per launch (launch_step_multi)
     const void *o, *f, *i;
     float *S;
     void *y;
@@ -68,6 +69,8 @@ struct StepArgs {
 };
 
 cudaError_t launch_step(const StepArgs &a);
+bool        step_multi_supported(int dk, int dv);
+cudaError_t launch_step_multi(const StepArgs &a);
 int         alu_default_chunk(int dk, int dv);
 bool        alu_chunk_supported(int dk, int dv, int C);
 cudaError_t launch_alu_fwd(const SeqArgs &a);

@@ -96,6 +96,13 @@ def test_host_side_argument_errors_launch_nothing(lib):
     # step args: o f i S y stream
     assert lib.hgrn2_step(ctypes.byref(d), *[ctypes.c_void_p(p) for p in [ok, ok, ok, 0, ok, 0]]) == 1
     assert lib.hgrn2_step(ctypes.byref(d), *[ctypes.c_void_p(p) for p in [ok, ok + 1, ok, ok, ok, 0]]) == 3
+    # multi-token step: same arguments; N tokens; d_k = d_v in {64, 128} only
+    assert lib.hgrn2_step_multi(ctypes.byref(d), *[ctypes.c_void_p(p) for p in [ok, ok, ok, 0, ok, 0]]) == 1
+    assert lib.hgrn2_step_multi(ctypes.byref(d), *[ctypes.c_void_p(p) for p in [ok, ok + 1, ok, ok, ok, 0]]) == 3
+    odd = binding.make_desc(1, 1, 4, 32, 64, binding.HGRN2_F32)
+    assert lib.hgrn2_step_multi(ctypes.byref(odd), *[ctypes.c_void_p(p) for p in [ok, ok, ok, ok, ok, 0]]) == 2
+    none = binding.make_desc(1, 1, 0, 64, 64, binding.HGRN2_F32)
+    assert lib.hgrn2_step_multi(ctypes.byref(none), *[ctypes.c_void_p(0)] * 6) == 0      # no token: no-op
     assert lib.hgrn2_poll(None) == 1
 
 

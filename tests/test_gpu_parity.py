@@ -54,6 +54,47 @@ def test_step_continues_prefill_state():
     assert G.rel_err(Sm.cpu().numpy(), SN_ref) <= 2e-2
 
 
+@pytest.mark.parametrize("B,H,d,io,T", [(3, 2, 128, "bf16", 7), (2, 3, 64, "f32", 5), (1, 1, 128, "f32", 1),
+                                        (2, 2, 64, "bf16", 16)])
+def test_step_multi_matches_oracle_and_single_steps(B, H, d, io, T):
+    # T tokens in one launch: against the oracle's T single steps, and bit for bit against T calls of hgrn2_step
+    w = W.scaled(W.CONFIGS["decode"], B=B, H=H, dk=d, dv=d, io=io)
+    dd = W.make_decode_inputs(w, steps=T)
+    tdt = torch.float32 if io == "f32" else torch.bfloat16
+    seq = {k: torch.from_numpy(np.ascontiguousarray(np.moveaxis(dd[k], 0, 2))).cuda().to(tdt) for k in ("o", "f", "i")}
+    Sbuf, S = G.canary((B, H, d, d), torch.float32)
+    S.copy_(torch.from_numpy(dd["S0"]))
+    ybuf, y = G.canary((B, H, T, d), tdt)
+    binding.hgrn2_step_multi(seq["o"], seq["f"], seq["i"], S, y=y)
+    S1 = torch.from_numpy(dd["S0"]).cuda()
+    S_ref = dd["S0"].astype(np.float64)
+    for t in range(T):
+        y1 = binding.hgrn2_step(seq["o"][:, :, t].contiguous(), seq["f"][:, :, t].contiguous(),
+                                seq["i"][:, :, t].contiguous(), S1)
+        assert torch.equal(y1, y[:, :, t])
+        y_ref = ref.hgrn2_step(dd["o"][t], dd["f"][t], dd["i"][t], S_ref)
+        assert G.rel_err(y[:, :, t].float().cpu().numpy(), y_ref) <= G.TOL[io]
+    assert torch.equal(S1, S)
+    assert G.rel_err(S.cpu().numpy(), S_ref) <= 1e-5
+    assert G.canary_ok(ybuf) and G.canary_ok(Sbuf)
+
+
+def test_step_multi_continues_prefill_state():
+    # forward over m tokens, then ONE multi-token step over the rest from its S_N == forward over all tokens
+    w = W.scaled(W.CONFIGS["lm_2048"], B=2, H=2, N=200, has_S0=True)
+    inp = W.make_inputs(w)
+    t = G.to_dev(inp, "bf16")
+    m = 150
+    _, Sm, _, ws, _ = binding.hgrn2_fwd(t["o"][:, :, :m].contiguous(), t["f"][:, :, :m].contiguous(),
+                                        t["i"][:, :, :m].contiguous(), t["S0"], save_for_backward=False)
+    y = binding.hgrn2_step_multi(t["o"][:, :, m:].contiguous(), t["f"][:, :, m:].contiguous(),
+                                 t["i"][:, :, m:].contiguous(), Sm)
+    torch.cuda.synchronize()
+    y_ref, SN_ref = ref.hgrn2_fwd(inp["o"], inp["f"], inp["i"], inp["S0"])
+    assert G.rel_err(y.float().cpu().numpy(), y_ref[:, :, m:]) <= 2e-2
+    assert G.rel_err(Sm.cpu().numpy(), SN_ref) <= 2e-2
+
+
 # ---------------------------------------------------------------- config 1 and the fp32 path
 def test_config1_tiny_f32():
     w = W.CONFIGS["tiny_f32"]
