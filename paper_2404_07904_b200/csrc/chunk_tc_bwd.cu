@@ -698,7 +698,6 @@ __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const floa
     if (dS0) dS0[e] = D;
 }
 
-int segments_for(uint64_t U, int N, int NC);     // chunk_tc_fwd.cu
 
 static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly)
 {
@@ -714,28 +713,39 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
         mo, mf, mi, mg, ms, mor, mfr,
-        reinterpret_cast<const float *>(reinterpret_cast<const char *>(a.states) + U * NC * kSavedStateBytes),
-        dSN, static_cast<__nv_bfloat16 *>(a.d_o),
+        a.totals, dSN, static_cast<__nv_bfloat16 *>(a.d_o),
         static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status);
     return cudaGetLastError();
 }
 
-cudaError_t launch_tc_bwd(const SeqArgs &a)
+cudaError_t launch_tc_bwd(const SeqArgs &a0)
 {
-    const uint64_t U = (uint64_t)a.B * a.H;
-    const int G = a.seg_scratch ? segments_for(U, a.N, a.NC) : 1;
-    if (G == 1) return launch_bwd_once(a, U, a.N, a.NC, a.dSN, a.dS0, false);
-    // scratch: G_local [U*G][128][128], dS_end [U*G][128][128], Lambda [U*G][128]
-    float *G_loc = static_cast<float *>(a.seg_scratch);
-    float *dS_end = G_loc + U * G * kD * kD;
-    float *lam = dS_end + U * G * kD * kD;
-    const float *totals = reinterpret_cast<const float *>(reinterpret_cast<const char *>(a.states) + U * a.NC * kSavedStateBytes);
-    cudaError_t err = launch_bwd_once(a, U * G, a.N / G, a.NC / G, nullptr, G_loc, true);     // state-gradient chains only
-    if (err != cudaSuccess) return err;
-    seg_decay_kernel<<<(unsigned)(U * G), kD, 0, a.stream>>>(totals, lam, a.NC / G);
-    seg_combine_bwd_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.dSN, G_loc, lam, dS_end, a.dS0, G);
-    if ((err = cudaGetLastError()) != cudaSuccess) return err;
-    return launch_bwd_once(a, U * G, a.N / G, a.NC / G, dS_end, nullptr, false);
+    const uint64_t U = (uint64_t)a0.B * a0.H;
+    SeqArgs a = a0;
+    a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
+    const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
+    cudaError_t err = cudaSuccess;
+    if (plan.main_units) {
+        const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
+        err = launch_bwd_once(m, plan.main_units, a.N, a.NC, m.dSN, m.dS0, false);
+        if (err != cudaSuccess) return err;
+    }
+    if (plan.tail_units) {
+        const SeqArgs t = tc_slice_units(a, plan.main_units, plan.tail_units);
+        const uint64_t Ut = plan.tail_units;
+        const int G = plan.G;
+        // scratch: G_local [Ut*G][128][128], dS_end [Ut*G][128][128], Lambda [Ut*G][128]
+        float *G_loc = static_cast<float *>(a.seg_scratch);
+        float *dS_end = G_loc + Ut * G * kD * kD;
+        float *lam = dS_end + Ut * G * kD * kD;
+        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, G_loc, true);     // state-gradient chains only
+        if (err != cudaSuccess) return err;
+        seg_decay_kernel<<<(unsigned)(Ut * G), kD, 0, a.stream>>>(t.totals, lam, a.NC / G);
+        seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false);
+    }
+    return err;
 }
 
 }  // namespace hgrn2

@@ -466,12 +466,58 @@ int segments_for(uint64_t U, int N, int NC)
     return G >= 2 ? G : 1;
 }
 
+// Few units (no more than SMs): all of them are split.  More units than SMs: the units beyond the last full
+// wave of CTAs would keep a few SMs busy for a whole sequence while the rest idle, so those - when they are at
+// most half a wave - are split as well and run after the full waves.
+SegPlan tc_seg_plan(uint64_t U, int N, int NC)
+{
+    SegPlan p{U, 0, 1};
+    const uint64_t sms = (uint64_t)sm_count();
+    if (U == 0 || sms == 0) return p;
+    if (U <= sms) {
+        const int G = segments_for(U, N, NC);
+        if (G > 1) p = SegPlan{0, U, G};
+        return p;
+    }
+    const uint64_t r = U % sms;
+    if (r > 0 && 2 * r <= sms) {
+        const int G = segments_for(r, N, NC);
+        if (G > 1) p = SegPlan{U - r, r, G};
+    }
+    return p;
+}
+
+// The same call restricted to units [u0, u0 + n): every per-unit pointer advanced (bf16 sequence tensors,
+// fp32 states; a.totals must be set).  The result has B = n, H = 1.
+SeqArgs tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n)
+{
+    SeqArgs s = a;
+    s.B = (int)n;
+    s.H = 1;
+    const size_t seq = (size_t)u0 * a.N * kD * 2, st = (size_t)u0 * kD * kD;
+    auto adv = [](const void *p, size_t bytes) { return p ? static_cast<const char *>(p) + bytes : nullptr; };
+    s.o = adv(a.o, seq); s.f = adv(a.f, seq); s.i = adv(a.i, seq); s.dy = adv(a.dy, seq);
+    s.y = const_cast<char *>(static_cast<const char *>(adv(a.y, seq)));
+    s.d_o = const_cast<char *>(static_cast<const char *>(adv(a.d_o, seq)));
+    s.d_f = const_cast<char *>(static_cast<const char *>(adv(a.d_f, seq)));
+    s.d_i = const_cast<char *>(static_cast<const char *>(adv(a.d_i, seq)));
+    s.S0 = a.S0 ? a.S0 + st : nullptr;
+    s.SN = a.SN ? a.SN + st : nullptr;
+    s.dSN = a.dSN ? a.dSN + st : nullptr;
+    s.dS0 = a.dS0 ? a.dS0 + st : nullptr;
+    if (a.states) {
+        s.states = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + (size_t)u0 * a.NC * kSavedStateBytes);
+        s.totals = a.totals + (size_t)u0 * a.NC * 2 * kD;
+    }
+    return s;
+}
+
 size_t tc_segment_scratch_bytes(const hgrn2_desc *d, int C)
 {
     const uint64_t U = (uint64_t)d->B * d->H;
     const int NC = (d->N + C - 1) / C;
-    const int G = segments_for(U, d->N, NC);
-    return G > 1 ? (size_t)U * G * (2 * kD * kD + kD) * sizeof(float) : 0;
+    const SegPlan p = tc_seg_plan(U, d->N, NC);
+    return p.tail_units ? (size_t)p.tail_units * p.G * (2 * kD * kD + kD) * sizeof(float) : 0;
 }
 
 static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *S0, float *SN, float *seg_decay,
@@ -491,27 +537,40 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
                             : (ragged ? tc_fwd_kernel<false, true> : tc_fwd_kernel<false, false>);
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
-    float *totals = want_saved ? reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * NC * kSavedStateBytes)
-                               : nullptr;
+    float *totals = want_saved ? a.totals : nullptr;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, seg_decay, want_y,
                                                                    want_saved, N, NC, a.status);
     return cudaGetLastError();
 }
 
-cudaError_t launch_tc_fwd(const SeqArgs &a)
+cudaError_t launch_tc_fwd(const SeqArgs &a0)
 {
-    const uint64_t U = (uint64_t)a.B * a.H;
-    const int G = a.seg_scratch ? segments_for(U, a.N, a.NC) : 1;
-    if (G == 1) return launch_fwd_once(a, U, a.N, a.NC, a.S0, a.SN, nullptr, a.y != nullptr, a.states != nullptr);
-    // scratch: S_local [U*G][128][128], S_start [U*G][128][128], Lambda [U*G][128]
-    float *S_loc = static_cast<float *>(a.seg_scratch);
-    float *S_start = S_loc + U * G * kD * kD;
-    float *lam = S_start + U * G * kD * kD;
-    cudaError_t err = launch_fwd_once(a, U * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false);
-    if (err != cudaSuccess) return err;
-    seg_combine_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.S0, S_loc, lam, S_start, a.SN, G);
-    if ((err = cudaGetLastError()) != cudaSuccess) return err;
-    return launch_fwd_once(a, U * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, a.y != nullptr, a.states != nullptr);
+    const uint64_t U = (uint64_t)a0.B * a0.H;
+    SeqArgs a = a0;
+    if (a.states) a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
+    const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
+    const bool want_y = a.y != nullptr, want_saved = a.states != nullptr;
+    cudaError_t err = cudaSuccess;
+    if (plan.main_units) {
+        const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
+        err = launch_fwd_once(m, plan.main_units, a.N, a.NC, m.S0, m.SN, nullptr, want_y, want_saved);
+        if (err != cudaSuccess) return err;
+    }
+    if (plan.tail_units) {
+        const SeqArgs t = tc_slice_units(a, plan.main_units, plan.tail_units);
+        const uint64_t Ut = plan.tail_units;
+        const int G = plan.G;
+        // scratch: S_local [Ut*G][128][128], S_start [Ut*G][128][128], Lambda [Ut*G][128]
+        float *S_loc = static_cast<float *>(a.seg_scratch);
+        float *S_start = S_loc + Ut * G * kD * kD;
+        float *lam = S_start + Ut * G * kD * kD;
+        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false);
+        if (err != cudaSuccess) return err;
+        seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, want_y, want_saved);
+    }
+    return err;
 }
 
 }  // namespace hgrn2

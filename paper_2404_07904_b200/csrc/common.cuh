@@ -56,6 +56,7 @@ struct SeqArgs {
     float *dS0;                   // nullable
     StatusBlock *status;
     void *seg_scratch;            // tensor-core path: scratch for sequences split into segments (nullable)
+    float *totals = nullptr;      // tensor-core path: per-chunk decay totals inside the saved data (set by its launchers)
     cudaStream_t stream;
 };
 
@@ -67,6 +68,15 @@ struct StepArgs {
     void *y;
     cudaStream_t stream;
 };
+
+// Tensor-core path, few or left-over units: which units run whole and which are split into G segments each.
+struct SegPlan {
+    uint64_t main_units;   // units [0, main_units) run as one CTA each
+    uint64_t tail_units;   // units [main_units, main_units + tail_units) are split into G segments each
+    int G;
+};
+SegPlan     tc_seg_plan(uint64_t U, int N, int NC);
+SeqArgs     tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n);
 
 cudaError_t launch_step(const StepArgs &a);
 bool        step_multi_supported(int dk, int dv);

@@ -216,6 +216,22 @@ def test_few_units_split_into_segments():
         np.testing.assert_array_equal(got[k], got2[k])
 
 
+def test_units_beyond_the_last_full_wave_are_split():
+    # a few more units than SMs: the left-over units run as segments after the full wave; units from both
+    # parts against the oracle, with initial state and final-state gradient so the slices' offsets are exercised
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    H = sms + 3
+    w = W.scaled(W.CONFIGS["long_16k"], B=1, H=H, N=1024, seed=78)
+    d = binding.make_desc(w.B, w.H, w.N, w.dk, w.dv, binding.HGRN2_BF16)
+    assert binding.workspace_bytes(d) > 256 + binding.saved_bytes(d), "segment scratch expected in the workspace"
+    inp = W.make_inputs(w)
+    got = G.gpu_fwd_bwd(inp, "bf16")
+    _check_units(inp, got, [(0, 0), (0, sms - 1), (0, sms), (0, H - 1)], 2e-2, "left-over units")
+    got2 = G.gpu_fwd_bwd(inp, "bf16", use_saved=False)
+    for k in got:
+        np.testing.assert_array_equal(got[k], got2[k])
+
+
 def test_config2_full_size_sampled_units():
     w = W.CONFIGS["lm_2048"]
     inp = W.make_inputs(w)
