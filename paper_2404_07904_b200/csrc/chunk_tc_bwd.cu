@@ -94,6 +94,7 @@ struct Ctl {
     uint64_t acc_free2;           // O -> M: dQs^T and dKs_intra^T columns are free again
     uint32_t tmem_base;
     int abort_flag;
+    int o_done;                   // O -> T: final passes finished so far, counted per warp (pacing only)
 };
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -241,6 +242,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->parked, kE3Threads);
         mbar_init(&ctl->acc_free2, kOThreads);
         ctl->abort_flag = 0;
+        ctl->o_done = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
         tma_prefetch_desc(&map_f);
@@ -267,6 +269,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int s = it % kStages, c = NC - 1 - it;
             uint8_t *qbuf = smem + s * kStageBytes;
             mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
+            // Pacing, not a data dependence: the transform of chunk `it` starts only when the final d_f pass of
+            // chunk it - 2 is over.  Its tiles are there well before, but run earlier it shares the issue slots
+            // with the output phase and that final pass, the longest stretch of the per-chunk loop (measured:
+            // starting as soon as the tiles land costs 2 %, starting even earlier, via an L2 prefetch, 15 %).
+            if (!kDsOnly && it >= 2) {
+                if (lane == 0) count_wait(&ctl->o_done, kOWarps * (it - 1), abort_flag);   // one poller per warp
+                __syncwarp();
+            }
             PT_MARK(0)
             PT_STAMP(status, 1, tid == 0 && it == 16) PT_STAMP(status, 20, tid == 0 && it == 18)
             const int n_valid = kRagged ? N - c * kC : kC;
@@ -469,6 +479,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_free2);
+            __syncwarp();
+            if (lane == 0) atomicAdd(&ctl->o_done, 1);
             PT_MARK(3)
             PT_STAMP(status, 19, tid == kWarpO * 32 && it == 16)
         }

@@ -93,6 +93,24 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parit
     return true;
 }
 
+// Bounded wait until a counter in shared memory, which only ever grows, has reached `target`.  Unlike an
+// mbarrier phase it cannot be missed by a waiter that arrives late, so it suits pure pacing hints between roles
+// that exchange no data.
+static __device__ __noinline__ bool count_wait(volatile int *counter, int target, volatile int *abort_flag)
+{
+    if (*counter >= target) return true;
+    if (*abort_flag) return false;
+    const unsigned long long t0 = globaltimer_ns();
+    while (*counter < target) {
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+    return true;
+}
+
 // Bounded wait that ignores the abort flag: used on the way out of a kernel to let copies that are
 // still in flight land before the shared memory they target is given up.
 __device__ __forceinline__ bool mbar_wait_drain(uint64_t *bar, uint32_t parity, unsigned long long limit_ns)
