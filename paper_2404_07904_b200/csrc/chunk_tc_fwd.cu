@@ -11,9 +11,9 @@
 //       bf16 copy S' for Y = Qs S' and for the saved-state store;
 //   E2  4 output warps: causal mask of A into an operand slab, Y into a staging tile;
 //   L   1 warp: TMA loads of o, f, i;
-//   MS  1 warp: tcgen05.mma issue of the state update S' += Ks^T V;
-//   MY  1 warp: tcgen05.mma issue of A = Qs Ks^T, Y = Qs S', Y += tril(A) V, and the TMA store of S'
-//       (the saved chunk state) straight from the operand copy;
+//   MS  1 warp: tcgen05.mma issue of the state update S' += Ks^T V, then the TMA store of S' (the saved
+//       chunk state) straight from the operand copy;
+//   MY  1 warp: tcgen05.mma issue of A = Qs Ks^T, Y = Qs S', Y += tril(A) V;
 //   ST  1 warp: TMA stores of the Y tiles.
 // Hand-offs are mbarriers; every wait is bounded (tc_common.cuh).
 //
@@ -56,7 +56,7 @@ struct Ctl {
     uint64_t m_tmem;             // E1 -> MS: the accumulator holds S' of the chunk
     uint64_t m_done;             // E1 -> MY: the bf16 copy of S' is in shared memory
     uint64_t barS;               // tcgen05.commit -> E1: state update complete
-    uint64_t barS2;              // tcgen05.commit -> E1: Y = Qs S' complete and stored, S' copy reusable
+    uint64_t barS2;              // tcgen05.commit (MY) + MS -> E1: Y = Qs S' complete, S' stored: copy reusable
     uint64_t barA[2];            // tcgen05.commit -> E2: A is complete
     uint64_t p_ready[2];         // E2 -> MY: tril(A) is in shared memory
     uint64_t barY[2];            // tcgen05.commit -> E2: Y is complete
@@ -102,7 +102,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->m_tmem, kE1Threads);
         mbar_init(&ctl->m_done, kE1Threads);
         mbar_init(&ctl->barS, 1);
-        mbar_init(&ctl->barS2, 1);
+        mbar_init(&ctl->barS2, 2);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&ctl->barA[b], 1);
             mbar_init(&ctl->p_ready[b], kE2Threads);
@@ -316,8 +316,20 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mma_commit(&ctl->barS);
                 mma_commit(&ctl->empty[s]);
                 PT_MARK(2)
+                // the saved chunk state, straight from the operand copy of S' (this lane is idle until the next
+                // chunk's state is ready; in the lane that issues the outputs' products the wait for the store
+                // to have read 32 KB would hold those up)
+                mbar_wait(&ctl->m_done, c & 1, abort_flag);
+                if (want_saved) {
+                    tma_store_3d(&map_saved, sbuf, 0, 0, u * NC + c);
+                    tma_store_3d(&map_saved, sbuf + kStateSlab, 64, 0, u * NC + c);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                }
+                mbar_arrive(&ctl->barS2);                   // second arrival: the tcgen05.commit of Y = Qs S'
             }
             PT_DUMP(status, 12, 3, true)
+            if (want_saved) tma_store_wait_all();
         }
     } else if (warp == kWarpMmaY) {
         // ================= MY: outputs (+ saved-state stores) =================
@@ -348,11 +360,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 }
                 mbar_wait(&ctl->m_done, c & 1, abort_flag);
                 PT_MARK(1)
-                if (want_saved) {
-                    tma_store_3d(&map_saved, sbuf, 0, 0, u * NC + c);
-                    tma_store_3d(&map_saved, sbuf + kStateSlab, 64, 0, u * NC + c);
-                    tma_store_commit();
-                }
                 if (want_y) {
                     if (c >= 2) {
                         mbar_wait(&ctl->y_tfree[b], ((c - 2) >> 1) & 1, abort_flag);
@@ -363,7 +370,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                         mma_bf16_ss(ty, dq + kmaj(kk), dsm + (uint64_t)(kk * 128), idescY, kk > 0);
                 }
                 PT_MARK(2)
-                if (want_saved) tma_store_wait_read();      // the S' copy is rewritten once barS2 fires
                 mma_commit(&ctl->barS2);
                 if (want_y) {
                     mbar_wait(&ctl->p_ready[b], (c >> 1) & 1, abort_flag);
@@ -378,7 +384,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 PT_MARK(4)
             }
             PT_DUMP(status, 15, 5, true)
-            if (want_saved) tma_store_wait_all();
         }
     } else {
         // ================= ST: Y stores =================
