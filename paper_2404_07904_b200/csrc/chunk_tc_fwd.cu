@@ -50,8 +50,10 @@ constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024;             // + alignment
 constexpr uint32_t kColS = 0, kColY = 128, kColA = 384;
 
 struct Ctl {
-    uint64_t full[kStages];      // TMA -> T, MS, MY
-    uint64_t empty[kStages];     // tcgen05.commit (MS and MY) -> L: every MMA reading the stage has completed
+    uint64_t fullqf[kStages];    // TMA (o, f tiles) -> T
+    uint64_t full[kStages];      // TMA (i tile) -> MS, MY
+    uint64_t emptyqf[kStages];   // tcgen05.commit (MS and MY) -> L: every MMA reading Qs, Ks of the stage has completed
+    uint64_t emptyv[kStages];    // tcgen05.commit (MS and MY) -> L: every MMA reading V of the stage has completed
     uint64_t t_done[kStages];    // T -> MS, MY, E1 (Pm, E of the chunk)
     uint64_t m_tmem;             // E1 -> MS: the accumulator holds S' of the chunk
     uint64_t m_done;             // E1 -> MY: the bf16 copy of S' is in shared memory
@@ -95,8 +97,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->fullqf[s], 1);
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->empty[s], 2);
+            mbar_init(&ctl->emptyqf[s], 2);
+            mbar_init(&ctl->emptyv[s], 2);
             mbar_init(&ctl->t_done[s], kTransformThreads);
         }
         mbar_init(&ctl->m_tmem, kE1Threads);
@@ -134,7 +138,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         for (int c = warp >> 2; c < NC; c += kTGroups) {
             const int s = c % kStages;
             uint8_t *qbuf = smem + s * kStageBytes;
-            mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
+            mbar_wait(&ctl->fullqf[s], (c / kStages) & 1, abort_flag);
             PT_MARK(0)
             const int n_valid = kRagged ? N - c * kC : kC;
             float *tg = totals ? totals + ((size_t)u * NC + c) * 2 * kD : nullptr;     // Pm, E of the chunk for the backward
@@ -281,14 +285,20 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         if (lane == 0) {
             for (int c = 0; c < NC; ++c) {
                 const int s = c % kStages;
-                if (c >= kStages) mbar_wait(&ctl->empty[s], ((c / kStages) - 1) & 1, abort_flag);
                 uint8_t *st = smem + s * kStageBytes;
-                mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
+                // o and f have barriers of their own in both directions: the transform, which paces the kernel,
+                // needs only them, and their tiles are free as soon as Y = Qs S' of the chunk three back is done,
+                // well before its last product Y += P V has read V
+                if (c >= kStages) mbar_wait(&ctl->emptyqf[s], ((c / kStages) - 1) & 1, abort_flag);
+                mbar_arrive_expect_tx(&ctl->fullqf[s], 2 * kTile);
                 for (int b = 0; b < 2; ++b) {
-                    tma_load_3d(st + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + b * kSlab, &map_o, &ctl->fullqf[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->fullqf[s], 64 * b, c * kC, u);
                 }
+                if (c >= kStages) mbar_wait(&ctl->emptyv[s], ((c / kStages) - 1) & 1, abort_flag);
+                mbar_arrive_expect_tx(&ctl->full[s], kTile);
+                for (int b = 0; b < 2; ++b)
+                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
             }
         }
     } else if (warp == kWarpMmaS) {
@@ -314,7 +324,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     mma_bf16_ss(tmem + kColS, dfm0 + so + (uint64_t)(kk * 128), dvm0 + so + (uint64_t)(kk * 128),
                                 idescS, 1);
                 mma_commit(&ctl->barS);
-                mma_commit(&ctl->empty[s]);
+                mma_commit(&ctl->emptyqf[s]);
+                mma_commit(&ctl->emptyv[s]);
                 PT_MARK(2)
                 // the saved chunk state, straight from the operand copy of S' (this lane is idle until the next
                 // chunk's state is ready; in the lane that issues the outputs' products the wait for the store
@@ -371,6 +382,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 }
                 PT_MARK(2)
                 mma_commit(&ctl->barS2);
+                mma_commit(&ctl->emptyqf[s]);               // A and Y = Qs S' were the last readers of Qs, Ks here
                 if (want_y) {
                     mbar_wait(&ctl->p_ready[b], (c >> 1) & 1, abort_flag);
                     PT_MARK(3)
@@ -380,7 +392,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                         mma_bf16_ss(ty, dp + (uint64_t)(kk * 2), dvm + (uint64_t)(kk * 128), idescY, 1);
                     mma_commit(&ctl->barY[b]);
                 }
-                mma_commit(&ctl->empty[s]);
+                mma_commit(&ctl->emptyv[s]);
                 PT_MARK(4)
             }
             PT_DUMP(status, 15, 5, true)
@@ -406,7 +418,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         // a load may still be in flight towards this CTA's shared memory: give it time to land
         for (int s = 0; s < kStages; ++s) {
             const int last = ((NC - 1 - s) / kStages) * kStages + s;     // last chunk that used stage s
-            if (s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
+            if (s < NC) {
+                mbar_wait_drain(&ctl->fullqf[s], (last / kStages) & 1, 20000000ull);
+                mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
+            }
         }
     }
     __syncthreads();
