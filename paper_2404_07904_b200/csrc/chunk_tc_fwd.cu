@@ -11,9 +11,9 @@
 //       bf16 copy S' for Y = Qs S' and for the saved-state store;
 //   E2  4 output warps: causal mask of A into an operand slab, Y into a staging tile;
 //   L   1 warp: TMA loads of o, f, i;
-//   MS  1 warp: tcgen05.mma issue of the state update S' += Ks^T V, then the TMA store of S' (the saved
-//       chunk state) straight from the operand copy;
-//   MY  1 warp: tcgen05.mma issue of A = Qs Ks^T, Y = Qs S', Y += tril(A) V;
+//   MS  1 warp: tcgen05.mma issue of A = Qs Ks^T and of the state update S' += Ks^T V, then the TMA store of
+//       S' (the saved chunk state) straight from the operand copy;
+//   MY  1 warp: tcgen05.mma issue of Y = Qs S', Y += tril(A) V;
 //   ST  1 warp: TMA stores of the Y tiles.
 // Hand-offs are mbarriers; every wait is bounded (tc_common.cuh).
 //
@@ -309,6 +309,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             // start-address field (addresses are in 16-byte units and stay below 2^14).
             const uint64_t dfm0 = smem_desc_sw128(smem_u32(smem) + kTile, kSlab, 1024);      // Ks, MN-major
             const uint64_t dvm0 = smem_desc_sw128(smem_u32(smem) + 2 * kTile, kSlab, 1024);  // V, MN-major
+            constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
+            const uint64_t dq0 = smem_desc_sw128(smem_u32(smem), 16, 1024);                  // Qs, K-major
+            const uint64_t dfk0 = smem_desc_sw128(smem_u32(smem) + kTile, 16, 1024);         // Ks, K-major
+            auto kmaj = [](int kk) { return (uint64_t)(((kk >> 2) * kSlab + (kk & 3) * 32) >> 4); };
             PT_DECL
             for (int c = 0; c < NC; ++c) {
                 const int s = c % kStages;
@@ -316,6 +320,20 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (c / kStages) & 1, abort_flag);
                 PT_MARK(0)
+                // A = Qs Ks^T is issued here, not by the lane of the other output products: this lane has nothing
+                // to do until the state is rescaled, and every tcgen05.mma also costs the issuing lane's scheduler
+                // (shared with a transform warp) issue time, so the products are spread over two schedulers
+                if (want_y) {
+                    const int b = c & 1;
+                    if (c >= 2) {                                    // tril(A) of chunk c - 2 has left this buffer
+                        mbar_wait(&ctl->p_ready[b], ((c - 2) >> 1) & 1, abort_flag);
+                        tc_fence_after_sync();
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_bf16_ss(tmem + kColA + 64 * b, dq0 + so + kmaj(kk), dfk0 + so + kmaj(kk), idescA, kk > 0);
+                    mma_commit(&ctl->barA[b]);
+                }
                 mbar_wait(&ctl->m_tmem, c & 1, abort_flag);
                 PT_MARK(1)
                 tc_fence_after_sync();
@@ -345,10 +363,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     } else if (warp == kWarpMmaY) {
         // ================= MY: outputs (+ saved-state stores) =================
         if (lane == 0) {
-            constexpr uint32_t idescA = idesc_bf16(64, 64, 0, 0);      // Qs (K-major) x Ks (K-major)
             constexpr uint32_t idescY = idesc_bf16(64, 128, 0, 1);     // Qs or P (K-major) x S' or V (MN-major)
             const uint64_t dq0 = smem_desc_sw128(smem_u32(smem), 16, 1024);                  // Qs, K-major
-            const uint64_t dfk0 = smem_desc_sw128(smem_u32(smem) + kTile, 16, 1024);         // Ks, K-major
             const uint64_t dvm0 = smem_desc_sw128(smem_u32(smem) + 2 * kTile, kSlab, 1024);  // V, MN-major
             const uint64_t dsm = smem_desc_sw128(smem_u32(sbuf), kStateSlab, 1024);          // S', MN-major
             const uint64_t dp0 = smem_desc_sw128(smem_u32(pbuf), 16, 1024);                  // tril(A), K-major
@@ -357,18 +373,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             for (int c = 0; c < NC; ++c) {
                 const int s = c % kStages, b = c & 1;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
-                const uint64_t dq = dq0 + so, dfk = dfk0 + so, dvm = dvm0 + so;
+                const uint64_t dq = dq0 + so, dvm = dvm0 + so;
                 const uint64_t dp = dp0 + (uint64_t)b * (kSlab >> 4);
-                const uint32_t ty = tmem + kColY + 128 * b, ta = tmem + kColA + 64 * b;
+                const uint32_t ty = tmem + kColY + 128 * b;
                 mbar_wait(&ctl->full[s], (c / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (c / kStages) & 1, abort_flag);
                 PT_MARK(0)
-                if (want_y) {
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)          // A = Qs Ks^T
-                        mma_bf16_ss(ta, dq + kmaj(kk), dfk + kmaj(kk), idescA, kk > 0);
-                    mma_commit(&ctl->barA[b]);
-                }
                 mbar_wait(&ctl->m_done, c & 1, abort_flag);
                 PT_MARK(1)
                 if (want_y) {
