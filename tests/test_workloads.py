@@ -59,3 +59,22 @@ def test_shard_units_partition(total, ws):
         assert s == pos
         pos += n
     assert max(n for _, n in spans) - min(n for _, n in spans) <= 1
+
+
+def test_lm_workloads_have_the_papers_layer_shapes():
+    # the benchmark shapes come from the paper's table of model configurations (stored as a text fixture):
+    # hidden dim = H * d_k, expand ratio = head dim = 128, training sequence length 2048
+    import os
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "model_configurations.txt")) as fh:
+        for line in fh:
+            if line.strip() and not line.startswith("#"):
+                p = line.split()
+                rows.append((float(p[0]), int(p[1]), int(p[2]), int(p[3])))
+    by_hidden = {r[1]: r for r in rows}
+    w = W.CONFIGS["lm_2048"]
+    assert w.H * w.dk in by_hidden and w.dk == w.dv == by_hidden[w.H * w.dk][2] and w.N == by_hidden[w.H * w.dk][3]
+    w = W.CONFIGS["lm_2560"]
+    assert w.H * w.dk in by_hidden and w.dk == w.dv == by_hidden[w.H * w.dk][2]
+    for name in ("long_16k", "decode"):
+        assert W.CONFIGS[name].dk == W.CONFIGS[name].dv == 128
