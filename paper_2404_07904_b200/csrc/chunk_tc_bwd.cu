@@ -20,17 +20,19 @@
 //
 // Warp roles (hand-offs are mbarriers, every wait is bounded; loops stay rolled to keep the
 // instruction footprint of the concurrently running roles small):
-//   T   4 warps: raw o, f tiles -> Qs, Ks in place, one chunk ahead (two TMA stages);
-//   E1  4 warps: rescale the dS accumulator and publish its bf16 copy dS'' (the chain between
-//       chunks), causal masks of A and dA into operand slabs, R;
-//   E3  8 warps: d_o and most of d_f from dQs^T, dKs_intra^T, dKs_inter^T.  A thread owns (key dim,
-//       half of the chunk) and walks its 32 steps outwards from the middle, carrying the decay
-//       product and the running sums; what is still missing then is one constant per key dimension
-//       (R plus the two halves' sums), so the almost finished d_f and 1/f are parked in the TMEM
-//       columns just read;
+//   T   4 warps: raw o, f tiles -> Qs, Ks in place, one chunk ahead (two TMA stages); paced so that it does not
+//       run alongside the output phase and the final d_f pass two chunks back;
+//   E1  4 warps: rescale the dS accumulator and publish its bf16 copy dS'' (the chain between chunks), R;
+//   E3  8 warps: first the causal masks of A and dA into operand slabs (one 32 x 32 block per warp), then d_o
+//       and most of d_f from dQs^T, dKs_intra^T, dKs_inter^T.  A thread owns (key dim, half of the chunk)
+//       and walks its 32 steps outwards from the middle, carrying the decay product and the running sums;
+//       what is still missing then is one constant per key dimension (R plus the two halves' sums), so the
+//       almost finished d_f and 1/f are parked in the TMEM columns just read.  It works from a second,
+//       unswizzled copy of raw o and f and recomputes Qs, Ks with the transform's roundings, so the operand
+//       stage is free as soon as the chunk's products are done;
 //   O   4 warps: d_i from dV^T, and d_f completed from the parked values;
-//   L   1 warp: TMA loads (raw tiles, saved S');
-//   MX, MY1, MY2  1 warp each: tcgen05.mma issue of the three groups below (one lane issuing all 56
+//   L   1 warp: TMA loads (o, f, dy stage; v; saved S'; raw o, f), each refilled when its last reader is done;
+//   MX, MY1, MY2  1 warp each: tcgen05.mma issue of the three groups below (one lane issuing all 52
 //       products of a chunk is itself a bottleneck: its instruction stream is long and serial).
 // Per chunk the tensor pipe runs
 //   X : dS' += Qs^T dY | A | dA            (overlaps the outputs of the previous chunk)
@@ -38,7 +40,8 @@
 //   Y2: dQs^T | dKs_intra^T | dV^T += dY^T A   (needs tril(A), tril(dA), S', and the parked values consumed)
 //
 // Tensor-memory plan (512 columns, no spare): dS [0,128); A [128,192) in lanes 0..63 and dA [192,256) in
-// lanes 64..127 (products of the stacked operand (Qs; dY), M = 128); dQs^T [256,320); dKs_intra^T [320,384); dKs_inter^T [384,448); dV^T [448,512).
+// lanes 64..127 (products of the stacked operand (Qs; dY), M = 128); dQs^T [256,320); dKs_intra^T [320,384);
+// dKs_inter^T [384,448); dV^T [448,512).
 #include "tc_chunk.cuh"
 
 namespace hgrn2 {
