@@ -32,7 +32,7 @@
 //       stage is free as soon as the chunk's products are done;
 //   O   4 warps: d_i from dV^T, and d_f completed from the parked values;
 //   L   1 warp: TMA loads (o, f, dy stage; v; saved S'; raw o, f), each refilled when its last reader is done;
-//   MX, MY1, MY2  1 warp each: tcgen05.mma issue of the three groups below (one lane issuing all 52
+//   MX, MY1, MY2  1 warp each: tcgen05.mma issue of the three groups below (one lane issuing all 56
 //       products of a chunk is itself a bottleneck: its instruction stream is long and serial).
 // Per chunk the tensor pipe runs
 //   X : dS' += Qs^T dY | A | dA            (overlaps the outputs of the previous chunk)
