@@ -91,7 +91,8 @@ size_t hgrn2_workspace_bytes(const hgrn2_desc *desc);
  *   SN   [B][H][dk][dv] float32          out, NULL = not wanted
  *   saved  hgrn2_saved_bytes(desc) bytes out, NULL = inference (nothing kept for backward)
  *   ws     hgrn2_workspace_bytes(desc) bytes, scratch; its first word is the status word,
- *          which this call clears on the stream before the kernel. */
+ *          which every call resets to HGRN2_OK on the stream before any of its work can report into it
+ *          (a small asynchronous clear, or the first kernel of the call itself). */
 hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
                        const float *S0, void *y, float *SN, void *saved, void *ws,
                        void *cuda_stream);

@@ -140,7 +140,11 @@ hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, con
     a.o = o; a.f = f; a.i = i; a.S0 = S0; a.y = y; a.SN = SN;
     a.states = static_cast<float *>(saved);
     a.status = static_cast<StatusBlock *>(ws);
-    if (cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+    // The status word starts every call at zero.  On the tensor-core path the first kernel of the call does that
+    // itself (a separate clear between two kernels of a stream costs a microsecond of idle GPU each time);
+    // everywhere else, and when no kernel will run, it is a small asynchronous memset.
+    a.clear_status = use_tc(desc) && !empty;
+    if (!a.clear_status && cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
     if ((size_t)desc->B * desc->H == 0) return HGRN2_OK;
     if (desc->N == 0) {
         if (SN) {
@@ -173,7 +177,8 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
     a.o = o; a.f = f; a.i = i; a.S0 = S0; a.dy = dy; a.dSN = dSN;
     a.d_o = d_o; a.d_f = d_f; a.d_i = d_i; a.dS0 = dS0;
     a.status = static_cast<StatusBlock *>(ws);
-    if (cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+    a.clear_status = use_tc(desc) && !empty;                     // see hgrn2_fwd
+    if (!a.clear_status && cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
     if ((size_t)desc->B * desc->H == 0) return HGRN2_OK;
     if (desc->N == 0) {
         if (dS0) {
@@ -194,6 +199,7 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
         cudaError_t e = tc ? launch_tc_fwd(r) : launch_alu_fwd(r);
         if (e != cudaSuccess) return HGRN2_ERR_CUDA;
         a.states = r.states;
+        a.clear_status = false;                                  // the forward's first kernel has done it
     }
     cudaError_t e = tc ? launch_tc_bwd(a) : launch_alu_bwd(a);
     return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;

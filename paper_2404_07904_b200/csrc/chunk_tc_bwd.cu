@@ -201,8 +201,15 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
               const __grid_constant__ CUtensorMap map_saved, const __grid_constant__ CUtensorMap map_o_raw,
               const __grid_constant__ CUtensorMap map_f_raw, const float *__restrict__ totals,
               const float *__restrict__ dSN, __nv_bfloat16 *__restrict__ d_o, __nv_bfloat16 *__restrict__ d_f,
-              __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N, int NC, StatusBlock *status)
+              __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N, int NC, StatusBlock *status,
+              int clear_status)
 {
+    // the first kernel of a call zeroes the status word; the only early report, the alignment check below, is the
+    // same in every CTA, so CTA 0 repeats it after its own clear
+    if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) {
+        status->code = 0;
+        status->where = 0;
+    }
     extern __shared__ __align__(1024) uint8_t smem[];
     if (smem_u32(smem) & 1023u) {          // every byte is spoken for: the swizzled tiles need the base aligned
         if (threadIdx.x == 0) report_error(status, HGRN2_ERR_CUDA, 3);
@@ -714,7 +721,8 @@ __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const floa
 }
 
 
-static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly)
+static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly,
+                                   bool clear)
 {
     CUtensorMap mo, mf, mi, mg, ms, mor, mfr;
     if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
@@ -729,7 +737,7 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
         mo, mf, mi, mg, ms, mor, mfr,
         a.totals, dSN, static_cast<__nv_bfloat16 *>(a.d_o),
-        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status);
+        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status, clear ? 1 : 0);
     return cudaGetLastError();
 }
 
@@ -740,10 +748,12 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
     a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
     const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
     cudaError_t err = cudaSuccess;
+    bool clear = a.clear_status;                                  // for the first kernel launched only
     if (plan.main_units) {
         const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
-        err = launch_bwd_once(m, plan.main_units, a.N, a.NC, m.dSN, m.dS0, false);
+        err = launch_bwd_once(m, plan.main_units, a.N, a.NC, m.dSN, m.dS0, false, clear);
         if (err != cudaSuccess) return err;
+        clear = false;
     }
     if (plan.tail_units) {
         const SeqArgs t = tc_slice_units(a, plan.main_units, plan.tail_units);
@@ -753,12 +763,12 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         float *G_loc = static_cast<float *>(a.seg_scratch);
         float *dS_end = G_loc + Ut * G * kD * kD;
         float *lam = dS_end + Ut * G * kD * kD;
-        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, G_loc, true);     // state-gradient chains only
+        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, G_loc, true, clear);     // state-gradient chains only
         if (err != cudaSuccess) return err;
         seg_decay_kernel<<<(unsigned)(Ut * G), kD, 0, a.stream>>>(t.totals, lam, a.NC / G);
         seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false);
+        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false, false);
     }
     return err;
 }

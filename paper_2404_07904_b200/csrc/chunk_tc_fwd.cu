@@ -80,8 +80,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
               const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
               float *__restrict__ totals, float *__restrict__ seg_decay, int want_y, int want_saved, int N, int NC,
-              StatusBlock *status)
+              StatusBlock *status, int clear_status)
 {
+    // the first kernel of a call zeroes the status word (errors are reported seconds later, after a wait ran out)
+    if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) {
+        status->code = 0;
+        status->where = 0;
+    }
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *sbuf = smem + kOffS;
@@ -551,7 +556,7 @@ size_t tc_segment_scratch_bytes(const hgrn2_desc *d, int C)
 }
 
 static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *S0, float *SN, float *seg_decay,
-                                   bool want_y, bool want_saved)
+                                   bool want_y, bool want_saved, bool clear)
 {
     CUtensorMap mo, mf, mi, my, ms;
     // tensor maps need a valid base even for outputs that are not wanted: point those at an input
@@ -569,7 +574,7 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? a.totals : nullptr;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, seg_decay, want_y,
-                                                                   want_saved, N, NC, a.status);
+                                                                   want_saved, N, NC, a.status, clear ? 1 : 0);
     return cudaGetLastError();
 }
 
@@ -581,10 +586,12 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
     const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
     const bool want_y = a.y != nullptr, want_saved = a.states != nullptr;
     cudaError_t err = cudaSuccess;
+    bool clear = a.clear_status;                                  // for the first kernel launched only
     if (plan.main_units) {
         const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
-        err = launch_fwd_once(m, plan.main_units, a.N, a.NC, m.S0, m.SN, nullptr, want_y, want_saved);
+        err = launch_fwd_once(m, plan.main_units, a.N, a.NC, m.S0, m.SN, nullptr, want_y, want_saved, clear);
         if (err != cudaSuccess) return err;
+        clear = false;
     }
     if (plan.tail_units) {
         const SeqArgs t = tc_slice_units(a, plan.main_units, plan.tail_units);
@@ -594,11 +601,11 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         float *S_loc = static_cast<float *>(a.seg_scratch);
         float *S_start = S_loc + Ut * G * kD * kD;
         float *lam = S_start + Ut * G * kD * kD;
-        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false);
+        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false, clear);
         if (err != cudaSuccess) return err;
         seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, want_y, want_saved);
+        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, want_y, want_saved, false);
     }
     return err;
 }

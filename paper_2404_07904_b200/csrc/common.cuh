@@ -57,6 +57,7 @@ struct SeqArgs {
     StatusBlock *status;
     void *seg_scratch;            // tensor-core path: scratch for sequences split into segments (nullable)
     float *totals = nullptr;      // tensor-core path: per-chunk decay totals inside the saved data (set by its launchers)
+    bool clear_status = false;    // tensor-core path: the first kernel of the call zeroes the status word itself
     cudaStream_t stream;
 };
 

@@ -156,6 +156,27 @@ def test_empty_sequence_and_empty_batch():
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("io,N,H", [("bf16", 200, 2), ("bf16", 1024, 3), ("f32", 100, 2)])
+def test_every_call_starts_with_a_clean_status_word(io, N, H):
+    # a stale error code in the workspace must not survive the next call: forward, backward with the saved
+    # states, backward that recomputes them; whole units, segmented sequences (few units) and the fp32 path
+    w = W.scaled(W.CONFIGS["lm_2048"], B=1, H=H, N=N, io=io, dk=128 if io == "bf16" else 64,
+                 dv=128 if io == "bf16" else 64, seed=5)
+    t = G.to_dev(W.make_inputs(w), io)
+    y, SN, saved, ws, desc = binding.hgrn2_fwd(t["o"], t["f"], t["i"], None)
+    torch.cuda.synchronize()
+    stale = torch.tensor([6, 1], dtype=torch.int32, device="cuda").view(torch.uint8)
+    for use_saved in (True, False):
+        ws[:8] = stale
+        binding.hgrn2_fwd(t["o"], t["f"], t["i"], None, y=y, saved=saved, ws=ws)
+        torch.cuda.synchronize()
+        assert binding.hgrn2_poll(ws) == 0
+        ws[:8] = stale
+        binding.hgrn2_bwd(t["o"], t["f"], t["i"], None, t["dy"], None, saved if use_saved else None, ws=ws)
+        torch.cuda.synchronize()
+        assert binding.hgrn2_poll(ws) == 0
+
+
 def test_run_to_run_determinism():
     w = W.scaled(W.CONFIGS["lm_2048"], B=1, H=3, N=257, has_S0=True, has_dSN=True)
     inp = W.make_inputs(w)
