@@ -295,6 +295,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 // needs only them, and their tiles are free as soon as Y = Qs S' of the chunk three back is done,
                 // well before its last product Y += P V has read V
                 if (c >= kStages) mbar_wait(&ctl->emptyqf[s], ((c / kStages) - 1) & 1, abort_flag);
+                // the next chunk's o, f tiles are asked into L2 now: their load can be issued only when their stage
+                // frees, one chunk from now, and then finds them there (measured on the fwd + bwd step: -1 %; two
+                // chunks ahead, or including the v tile, gave nothing)
+                if (c + 1 < NC)
+                    for (int b = 0; b < 2; ++b) {
+                        tma_prefetch_3d(&map_o, 64 * b, (c + 1) * kC, u);
+                        tma_prefetch_3d(&map_f, 64 * b, (c + 1) * kC, u);
+                    }
                 mbar_arrive_expect_tx(&ctl->fullqf[s], 2 * kTile);
                 for (int b = 0; b < 2; ++b) {
                     tma_load_3d(st + b * kSlab, &map_o, &ctl->fullqf[s], 64 * b, c * kC, u);
