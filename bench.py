@@ -34,7 +34,7 @@ NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (captured on the same workloads the bench times: lm_2048 and the full decode batch).
-NCU_TRAFFIC_BYTES = {"fwd": 201.38e6 + 153.92e6, "bwd": 406.95e6 + 170.21e6, "step": 271.60e6 + 212.48e6}
+NCU_TRAFFIC_BYTES = {"fwd": 201.40e6 + 154.21e6, "bwd": 406.95e6 + 170.12e6, "step": 271.60e6 + 212.48e6}
 
 
 def load_peaks():
