@@ -21,9 +21,14 @@
  *   - Sequence tensors are [B][H][N][d] with d innermost; o and f have d = dk, i, y
  *     and dy have d = dv.  Their element type is desc->io (float or bf16).
  *   - State tensors S0, SN, dS0, dSN, S are [B][H][dk][dv] float32, dv innermost.
- *   - f must lie in [0, 1].  The chunked kernels work with in-chunk cumulative decay
- *     and treat f below 2^-100 as 2^-100; d_f divides by f and loses accuracy as
- *     f -> 0 (it stays finite).
+ *   - f must lie in [0, 1]; the whole closed interval is supported by every call.  The
+ *     tensor-core kernels rescale their operands by in-chunk cumulative decay, which they can
+ *     represent only while the decay across each half of a 64-token chunk stays above 2^-100
+ *     per key dimension (a gate that averages above ~0.12 over 32 steps).  A (batch, head) unit
+ *     that leaves this range is detected on the device and redone, inside the same call, by
+ *     pairwise-safe fp32 routines (exact, but two orders of magnitude slower for that unit);
+ *     hgrn2_exact_path_units reports how many units a call handled that way.  d_f divides by
+ *     f (f below 2^-100 is taken as 2^-100 there), so it loses accuracy as f -> 0.
  *   - Errors detected on the host (bad sizes, NULL or misaligned pointers, unsupported
  *     shapes, too small a workspace) are returned at once and nothing is launched.
  *     A failed launch returns HGRN2_ERR_CUDA.  Device-side problems (a bounded wait
@@ -79,9 +84,10 @@ typedef struct hgrn2_desc {
 size_t hgrn2_saved_bytes(const hgrn2_desc *desc);
 
 /* Bytes of the workspace `ws` every call takes: a 256-byte status block, room for the
- * saved data that hgrn2_bwd re-creates when it is given saved = NULL and, when the batch
- * has too few (batch, head) units to fill the GPU, scratch for running each sequence as
- * several segments (the size therefore depends on the current device).  0 on a bad desc. */
+ * saved data that hgrn2_bwd re-creates when it is given saved = NULL and, on the tensor-core
+ * path, scratch for running each sequence as several segments when the batch has too few
+ * (batch, head) units to fill the GPU (the size therefore depends on the current device) and
+ * one dk x dv float matrix per unit for units redone on the exact path.  0 on a bad desc. */
 size_t hgrn2_workspace_bytes(const hgrn2_desc *desc);
 
 /* Forward over a whole sequence (Eq. 3 unrolled chunk by chunk; training and prefill).
@@ -132,7 +138,7 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
  *               status word of the call is copied there on the stream, for hgrn2_poll.
  * Limits and caveats
  *   - hgrn2_workspace_bytes(desc) - 256 must not exceed HGRN2_STATIC_SCRATCH_BYTES (bf16 d = 128:
- *     B*H*ceil(N/64) <= 992 chunks of 33 KB each); larger problems return HGRN2_ERR_WORKSPACE and nothing
+ *     B*H*(33 KB * ceil(N/64) + 64 KB) <= 32 MiB); larger problems return HGRN2_ERR_WORKSPACE and nothing
  *     is launched.  Use hgrn2_bwd with a caller-owned workspace for those.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in
  *     it.  Each call clears the status block and overwrites every state it later reads, so stale
@@ -170,6 +176,13 @@ hgrn2_status hgrn2_step_multi(const hgrn2_desc *desc, const void *o, const void 
  * after synchronising the stream the work ran on.  Returns HGRN2_OK, HGRN2_ERR_TIMEOUT,
  * HGRN2_ERR_DOMAIN, or HGRN2_ERR_CUDA if the copy itself failed. */
 hgrn2_status hgrn2_poll(const void *ws);
+
+/* Number of (batch, head) unit passes that the last tensor-core call using `ws` (a device pointer) redid on
+ * the exact fp32 path because the unit's decay left the range described at the top of this file (Eq. 3 holds
+ * on all of [0, 1]; the rescaled-operand form of the chunkwise products does not).  A backward that re-creates
+ * its states (saved = NULL) counts a unit once for each of its two passes.  Blocking copy: synchronise the
+ * stream first.  0 on the fp32 kernels; -1 if `ws` is NULL or the copy failed. */
+int32_t hgrn2_exact_path_units(const void *ws);
 
 /* Static, human-readable name of a status code. */
 const char *hgrn2_status_string(hgrn2_status s);

@@ -27,6 +27,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "hgrn2_saved_bytes", "hgrn2_workspace_bytes", "hgrn2_fwd", "hgrn2_bwd", "hgrn2_step",
     "hgrn2_step_multi", "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path", "hgrn2_bwd_static_scratch",
+    "hgrn2_exact_path_units",
 )
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
@@ -69,6 +70,8 @@ def load() -> ctypes.CDLL:
     lib.hgrn2_status_string.argtypes = [ctypes.c_int]
     lib.hgrn2_poll.restype = ctypes.c_int
     lib.hgrn2_poll.argtypes = [vp]
+    lib.hgrn2_exact_path_units.restype = ctypes.c_int32
+    lib.hgrn2_exact_path_units.argtypes = [vp]
     lib.hgrn2_fwd.restype = ctypes.c_int
     lib.hgrn2_fwd.argtypes = [dp] + [vp] * 9
     lib.hgrn2_bwd.restype = ctypes.c_int
@@ -227,6 +230,11 @@ def hgrn2_step_multi(o, f, i, S, *, y=None, stream=None):
     code = load().hgrn2_step_multi(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S), _ptr(y), _stream(stream))
     _check(code, "hgrn2_step_multi")
     return y
+
+
+def exact_path_units(ws: torch.Tensor) -> int:
+    """Unit passes the last tensor-core call using `ws` redid on the exact fp32 path (synchronise first)."""
+    return int(load().hgrn2_exact_path_units(_ptr(ws)))
 
 
 def hgrn2_poll(ws: torch.Tensor) -> int:

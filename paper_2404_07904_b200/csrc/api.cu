@@ -1,5 +1,6 @@
 // C ABI of the HGRN2 library: argument checks and dispatch.  Every step of the path runs in
 // the kernels of this directory; nothing here computes on the host.
+#include <stddef.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -13,6 +14,7 @@ int         tc_default_chunk();
 bool        tc_chunk_supported(int C);
 size_t      tc_saved_bytes(const hgrn2_desc *d, int C);
 size_t      tc_segment_scratch_bytes(const hgrn2_desc *d, int C);
+size_t      tc_exact_scratch_bytes(const hgrn2_desc *d);
 cudaError_t launch_tc_fwd(const SeqArgs &a);
 cudaError_t launch_tc_bwd(const SeqArgs &a);
 }  // namespace hgrn2
@@ -72,9 +74,16 @@ size_t saved_bytes_for(const hgrn2_desc *d, int C)
 void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream, void *ws)
 {
     memset(&a, 0, sizeof(a));
-    // workspace layout: status block | room for re-created saved data | segment scratch (tensor-core path)
-    if (use_tc(d) && tc_segment_scratch_bytes(d, C) != 0)
-        a.seg_scratch = static_cast<char *>(ws) + sizeof(StatusBlock) + saved_bytes_for(d, C);
+    // workspace layout: status block | room for re-created saved data | tensor-core path: segment scratch, then one
+    // float matrix per unit for units redone on the exact path
+    a.seg_scratch = nullptr;
+    a.exact_scratch = nullptr;
+    if (use_tc(d)) {
+        char *p = static_cast<char *>(ws) + sizeof(StatusBlock) + saved_bytes_for(d, C);
+        const size_t seg = tc_segment_scratch_bytes(d, C);
+        if (seg != 0) a.seg_scratch = p;
+        a.exact_scratch = reinterpret_cast<float *>(p + seg);
+    }
     a.B = d->B; a.H = d->H; a.N = d->N; a.dk = d->dk; a.dv = d->dv; a.C = C;
     a.NC = (d->N + C - 1) / C;
     a.io = d->io;
@@ -104,7 +113,8 @@ size_t hgrn2_workspace_bytes(const hgrn2_desc *desc)
 {
     const int C = resolve_chunk(desc);
     if (C == 0) return 0;
-    return sizeof(StatusBlock) + saved_bytes_for(desc, C) + (use_tc(desc) ? tc_segment_scratch_bytes(desc, C) : 0);
+    return sizeof(StatusBlock) + saved_bytes_for(desc, C) +
+           (use_tc(desc) ? tc_segment_scratch_bytes(desc, C) + tc_exact_scratch_bytes(desc) : 0);
 }
 
 const char *hgrn2_status_string(hgrn2_status s)
@@ -244,6 +254,16 @@ hgrn2_status hgrn2_poll(const void *ws)
     if (cudaMemcpy(&code, ws, sizeof(code), cudaMemcpyDeviceToHost) != cudaSuccess) return HGRN2_ERR_CUDA;
     if (code < 0 || code > HGRN2_ERR_DOMAIN) return HGRN2_ERR_CUDA;
     return static_cast<hgrn2_status>(code);
+}
+
+int32_t hgrn2_exact_path_units(const void *ws)
+{
+    if (!ws) return -1;
+    int32_t n = 0;
+    if (cudaMemcpy(&n, static_cast<const char *>(ws) + offsetof(StatusBlock, exact_units), sizeof(n),
+                   cudaMemcpyDeviceToHost) != cudaSuccess)
+        return -1;
+    return n;
 }
 
 }  // extern "C"

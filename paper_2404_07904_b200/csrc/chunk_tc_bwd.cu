@@ -42,6 +42,7 @@
 // Tensor-memory plan (512 columns, no spare): dS [0,128); A [128,192) in lanes 0..63 and dA [192,256) in
 // lanes 64..127 (products of the stacked operand (Qs; dY), M = 128); dQs^T [256,320); dKs_intra^T [320,384);
 // dKs_inter^T [384,448); dV^T [448,512).
+#include "chunk_alu.cuh"
 #include "tc_chunk.cuh"
 
 namespace hgrn2 {
@@ -98,9 +99,13 @@ struct Ctl {
     uint32_t tmem_base;
     int abort_flag;
     int o_done;                   // O -> T: final passes finished so far, counted per warp (pacing only)
+    int exact_flag;               // E1: a decay of this CTA's tokens left the range of the rescaled operands
 };
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
+
+constexpr int kExactC = 32;       // chunk length of the exact fp32 routines at d = 128 (their shared-memory budget)
+static_assert(alu::bwd_smem_floats(kD, kD, kExactC) * sizeof(float) <= kSmemBytes, "exact path fits the CTA's shared memory");
 
 // d_o and the nearly finished d_f of one thread: key dimension k, local times [32 * kUp, 32 * kUp + 32),
 // walked outwards from the middle of the chunk in blocks of eight.  Returns this half's sums of a and e.
@@ -194,7 +199,8 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
 // into segments.  A template parameter, not a flag: the full kernel is sensitive to its instruction footprint.
 // kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens); when false,
 // every per-row validity test below folds away.
-template <bool kDsOnly, bool kRagged>
+// kMultiCta: a unit runs as several CTAs (segments) of this launch (see the forward kernel).
+template <bool kDsOnly, bool kRagged, bool kMultiCta>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
@@ -202,13 +208,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
               const __grid_constant__ CUtensorMap map_f_raw, const float *__restrict__ totals,
               const float *__restrict__ dSN, __nv_bfloat16 *__restrict__ d_o, __nv_bfloat16 *__restrict__ d_f,
               __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N, int NC, StatusBlock *status,
-              int clear_status)
+              int clear_status, const ExactArgs ex)
 {
     // the first kernel of a call zeroes the status word; the only early report, the alignment check below, is the
     // same in every CTA, so CTA 0 repeats it after its own clear
     if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) {
         status->code = 0;
         status->where = 0;
+        status->exact_units = 0;
     }
     extern __shared__ __align__(1024) uint8_t smem[];
     if (smem_u32(smem) & 1023u) {          // every byte is spoken for: the swizzled tiles need the base aligned
@@ -253,6 +260,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->acc_free2, kOThreads);
         ctl->abort_flag = 0;
         ctl->o_done = 0;
+        ctl->exact_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
         tma_prefetch_desc(&map_f);
@@ -312,6 +320,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         for (int it = 0; it < NC; ++it) {
             // ---- dS'' = (Pm_prev E) dS' (the accumulator, or dSN first) -> TMEM, bf16 copy -> dsbuf
             PT_MARK(0)
+            // a total on the floor: the decay across that half chunk is more than the rescaled operands can carry
+            if (fminf(pm_c, ee_c) <= kProdFloor) ctl->exact_flag = 1;
             const float factor = pm_prev * ee_c;
             pm_prev = pm_c;
             if (it + 1 < NC) {
@@ -687,6 +697,33 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     }
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+
+    // ---- exact path (see the forward kernel): the unit is redone from its inputs and its saved chunk states by the
+    // pairwise-safe fp32 routine; with several CTAs per unit the last one to finish does it.
+    if (ex.o == nullptr) return;
+    const int unit = kMultiCta ? u / ex.G : u;
+    if constexpr (kMultiCta) {
+        if (tid == 0) {
+            if (ctl->exact_flag) atomicOr(&ex.unit_flag[unit], 1);
+            __threadfence();
+            int go = 0;
+            if (atomicAdd(&ex.unit_count[unit], 1) == ex.G - 1) {
+                __threadfence();
+                go = atomicOr(&ex.unit_flag[unit], 0);
+            }
+            ctl->exact_flag = go;
+        }
+        __syncthreads();
+    }
+    if (!ctl->exact_flag || *abort_flag) return;
+    __syncthreads();                                               // every thread has read the flag: smem is reused now
+    if (tid == 0) atomicAdd(&status->exact_units, 1);
+    const size_t seq = (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
+    const int nc64 = (ex.N + kC - 1) / kC;
+    alu::bwd_unit<__nv_bfloat16, __nv_bfloat16>(
+        reinterpret_cast<float *>(smem), ex.o + seq, ex.f + seq, ex.i + seq, ex.dy + seq, ex.dSN ? ex.dSN + st : nullptr,
+        ex.states + (size_t)unit * nc64 * kD * kD, kC / kExactC, ex.scratch + st, ex.d_o + seq, ex.d_f + seq,
+        ex.d_i + seq, ex.dS0 ? ex.dS0 + st : nullptr, ex.N, kD, kD, kExactC, (ex.N + kExactC - 1) / kExactC);
 }
 
 }  // namespace
@@ -705,9 +742,14 @@ __global__ void seg_decay_kernel(const float *__restrict__ totals, float *__rest
 // Chains the segments in reverse: dS_end[r] = gradient w.r.t. the state at the end of segment r.
 __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const float *__restrict__ G_loc,
                                        const float *__restrict__ lam, float *__restrict__ dS_end,
-                                       float *__restrict__ dS0, int G)
+                                       float *__restrict__ dS0, int G, int *__restrict__ unit_flag,
+                                       int *__restrict__ unit_count, int units)
 {
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
+    if (e < (size_t)units) {             // exact-path bookkeeping of the full pass that follows starts at zero
+        unit_flag[e] = 0;
+        unit_count[e] = 0;
+    }
     const size_t u = e / (kD * kD);
     const int k = (int)((e / kD) % kD);
     const size_t kv = e % (kD * kD);
@@ -721,8 +763,29 @@ __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const floa
 }
 
 
+static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag, int *unit_count)
+{
+    ExactArgs ex;
+    ex.o = static_cast<const __nv_bfloat16 *>(a.o);
+    ex.f = static_cast<const __nv_bfloat16 *>(a.f);
+    ex.i = static_cast<const __nv_bfloat16 *>(a.i);
+    ex.dy = static_cast<const __nv_bfloat16 *>(a.dy);
+    ex.dSN = a.dSN;
+    ex.d_o = static_cast<__nv_bfloat16 *>(a.d_o);
+    ex.d_f = static_cast<__nv_bfloat16 *>(a.d_f);
+    ex.d_i = static_cast<__nv_bfloat16 *>(a.d_i);
+    ex.dS0 = a.dS0;
+    ex.states = reinterpret_cast<__nv_bfloat16 *>(a.states);
+    ex.scratch = a.exact_scratch;
+    ex.N = N_unit;
+    ex.G = G;
+    ex.unit_flag = unit_flag;
+    ex.unit_count = unit_count;
+    return ex;
+}
+
 static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly,
-                                   bool clear)
+                                   bool clear, const ExactArgs &ex)
 {
     CUtensorMap mo, mf, mi, mg, ms, mor, mfr;
     if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
@@ -730,14 +793,17 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
         !make_map_plain(&mor, a.o, U, N, kC) || !make_map_plain(&mfr, a.f, U, N, kC))
         return cudaErrorInvalidValue;
     const bool ragged = N % kC != 0;
-    auto kernel = kDsOnly ? (ragged ? tc_bwd_kernel<true, true> : tc_bwd_kernel<true, false>)
-                          : (ragged ? tc_bwd_kernel<false, true> : tc_bwd_kernel<false, false>);
+    if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
+    auto kernel = kDsOnly ? (ragged ? tc_bwd_kernel<true, true, false> : tc_bwd_kernel<true, false, false>)
+                          : (ragged ? tc_bwd_kernel<false, true, false>
+                                    : (ex.o != nullptr && ex.G > 1 ? tc_bwd_kernel<false, false, true>
+                                                                    : tc_bwd_kernel<false, false, false>));
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
         mo, mf, mi, mg, ms, mor, mfr,
         a.totals, dSN, static_cast<__nv_bfloat16 *>(a.d_o),
-        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status, clear ? 1 : 0);
+        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status, clear ? 1 : 0, ex);
     return cudaGetLastError();
 }
 
@@ -751,7 +817,8 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
     bool clear = a.clear_status;                                  // for the first kernel launched only
     if (plan.main_units) {
         const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
-        err = launch_bwd_once(m, plan.main_units, a.N, a.NC, m.dSN, m.dS0, false, clear);
+        err = launch_bwd_once(m, plan.main_units, a.N, a.NC, m.dSN, m.dS0, false, clear,
+                              exact_args(m, a.N, 1, nullptr, nullptr));
         if (err != cudaSuccess) return err;
         clear = false;
     }
@@ -763,12 +830,16 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         float *G_loc = static_cast<float *>(a.seg_scratch);
         float *dS_end = G_loc + Ut * G * kD * kD;
         float *lam = dS_end + Ut * G * kD * kD;
-        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, G_loc, true, clear);     // state-gradient chains only
+        int *unit_flag = reinterpret_cast<int *>(lam + Ut * G * kD), *unit_count = unit_flag + Ut;
+        // state-gradient chains only; no exact path of their own: the full pass below meets the same decays
+        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, G_loc, true, clear, ExactArgs{});
         if (err != cudaSuccess) return err;
         seg_decay_kernel<<<(unsigned)(Ut * G), kD, 0, a.stream>>>(t.totals, lam, a.NC / G);
-        seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G);
+        seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G,
+                                                                                    unit_flag, unit_count, (int)Ut);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false, false);
+        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false, false,
+                              exact_args(t, a.N, G, unit_flag, unit_count));
     }
     return err;
 }

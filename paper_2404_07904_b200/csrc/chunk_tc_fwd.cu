@@ -20,6 +20,7 @@
 // Tensor-memory plan (512 columns): S' at [0,128) (lane = key dim, column = value dim); Y, double
 // buffered, at [128,384) and A, double buffered, at [384,512) in the M = 64 accumulator layout
 // (row r -> lane 32 * (r / 16) + r % 16).
+#include "chunk_alu.cuh"
 #include "tc_chunk.cuh"
 
 namespace hgrn2 {
@@ -67,25 +68,32 @@ struct Ctl {
     uint64_t y_sfree;            // ST -> E2: the staging tile may be overwritten
     uint32_t tmem_base;
     int abort_flag;
+    int exact_flag;              // E1: a decay of this CTA's tokens left the range of the rescaled operands
 };
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
+constexpr int kExactC = 32;      // chunk length of the exact fp32 routines at d = 128 (their shared-memory budget)
+static_assert(alu::fwd_smem_floats(kD, kD, kExactC) * sizeof(float) <= kSmemBytes - 1024, "exact path fits the CTA's shared memory");
+
 // kSegDecay: also write the product of f over the whole (sub)sequence per key dimension to seg_decay (used when
 // sequences are split into segments).  A template parameter: the kernel is sensitive to its instruction footprint.
 // kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens).
-template <bool kSegDecay, bool kRagged>
+// kMultiCta: a unit runs as several CTAs (segments) of this launch; the bookkeeping that lets the last of them
+// take the unit's exact path is compiled in only then (its mere presence costs the one-CTA-per-unit launch 3 %).
+template <bool kSegDecay, bool kRagged, bool kMultiCta>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
               const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
               float *__restrict__ totals, float *__restrict__ seg_decay, int want_y, int want_saved, int N, int NC,
-              StatusBlock *status, int clear_status)
+              StatusBlock *status, int clear_status, const ExactArgs ex)
 {
     // the first kernel of a call zeroes the status word (errors are reported seconds later, after a wait ran out)
     if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) {
         status->code = 0;
         status->where = 0;
+        status->exact_units = 0;
     }
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -121,6 +129,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->y_staged, kE2Threads);
         mbar_init(&ctl->y_sfree, 1);
         ctl->abort_flag = 0;
+        ctl->exact_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
         tma_prefetch_desc(&map_f);
@@ -171,9 +180,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk) back into TMEM
             mbar_wait(&ctl->t_done[c % kStages], (c / kStages) & 1, abort_flag);
             PT_MARK(0)
-            const float factor = e_prev * pm[(c & 3) * 128 + krow];
+            const float pm_c = pm[(c & 3) * 128 + krow];
+            const float factor = e_prev * pm_c;
             e_prev = ee[(c & 3) * 128 + krow];
-            if (kSegDecay) lam *= pm[(c & 3) * 128 + krow] * e_prev;
+            // a total on the floor: the decay across that half chunk is more than the rescaled operands can carry
+            if (fminf(pm_c, e_prev) <= kProdFloor) ctl->exact_flag = 1;
+            if (kSegDecay) lam *= pm_c * e_prev;
             uint32_t r[64];
             if (c == 0) {
                 if (S0) {
@@ -449,6 +461,35 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     }
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+
+    // ---- exact path: the sweep met a decay its operands cannot represent, so the unit is redone, from its inputs,
+    // by the pairwise-safe fp32 routine (every output of the unit is overwritten).  With several CTAs per unit
+    // (segments) the last one to finish does it, once every other has written its part.
+    if (ex.o == nullptr) return;
+    const int unit = kMultiCta ? u / ex.G : u;
+    if constexpr (kMultiCta) {
+        if (tid == 0) {
+            if (ctl->exact_flag) atomicOr(&ex.unit_flag[unit], 1);
+            __threadfence();
+            int go = 0;
+            if (atomicAdd(&ex.unit_count[unit], 1) == ex.G - 1) {
+                __threadfence();
+                go = atomicOr(&ex.unit_flag[unit], 0);
+            }
+            ctl->exact_flag = go;
+        }
+        __syncthreads();
+    }
+    if (!ctl->exact_flag || *abort_flag) return;
+    __syncthreads();                                               // every thread has read the flag: smem is reused now
+    if (tid == 0) atomicAdd(&status->exact_units, 1);
+    const size_t seq = (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
+    const int nc64 = (ex.N + kC - 1) / kC;
+    alu::fwd_unit<__nv_bfloat16, __nv_bfloat16>(
+        reinterpret_cast<float *>(smem), ex.o + seq, ex.f + seq, ex.i + seq, ex.S0 ? ex.S0 + st : nullptr,
+        ex.y ? ex.y + seq : nullptr, ex.SN ? ex.SN + st : nullptr,
+        ex.states ? ex.states + (size_t)unit * nc64 * kD * kD : nullptr, kC / kExactC, ex.N, kD, kD, kExactC,
+        (ex.N + kExactC - 1) / kExactC);
 }
 
 }  // namespace
@@ -475,9 +516,13 @@ size_t tc_saved_bytes(const hgrn2_desc *d, int C)
 // [U * G][N / G][128] view of the same memory, so the kernel itself does not know about segments.
 __global__ void seg_combine_kernel(const float *__restrict__ S0, const float *__restrict__ S_loc,
                                    const float *__restrict__ lam, float *__restrict__ S_start, float *__restrict__ SN,
-                                   int G)
+                                   int G, int *__restrict__ unit_flag, int *__restrict__ unit_count, int units)
 {
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
+    if (e < (size_t)units) {             // exact-path bookkeeping of the full pass that follows starts at zero
+        unit_flag[e] = 0;
+        unit_count[e] = 0;
+    }
     const size_t u = e / (kD * kD);
     const int k = (int)((e / kD) % kD);
     const size_t kv = e % (kD * kD);
@@ -548,6 +593,7 @@ SeqArgs tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n)
     s.SN = a.SN ? a.SN + st : nullptr;
     s.dSN = a.dSN ? a.dSN + st : nullptr;
     s.dS0 = a.dS0 ? a.dS0 + st : nullptr;
+    s.exact_scratch = a.exact_scratch ? a.exact_scratch + st : nullptr;
     if (a.states) {
         s.states = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + (size_t)u0 * a.NC * kSavedStateBytes);
         s.totals = a.totals + (size_t)u0 * a.NC * 2 * kD;
@@ -555,16 +601,39 @@ SeqArgs tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n)
     return s;
 }
 
+// Per-unit flag and counter of the exact path when a unit runs as several CTAs, after the segment scratch proper.
+static size_t seg_flag_bytes(uint64_t units) { return ((size_t)units * 2 * sizeof(int) + 15) & ~(size_t)15; }
+
 size_t tc_segment_scratch_bytes(const hgrn2_desc *d, int C)
 {
     const uint64_t U = (uint64_t)d->B * d->H;
     const int NC = (d->N + C - 1) / C;
     const SegPlan p = tc_seg_plan(U, d->N, NC);
-    return p.tail_units ? (size_t)p.tail_units * p.G * (2 * kD * kD + kD) * sizeof(float) : 0;
+    return p.tail_units ? (size_t)p.tail_units * p.G * (2 * kD * kD + kD) * sizeof(float) + seg_flag_bytes(p.tail_units) : 0;
+}
+
+// One float matrix per unit for the exact path of the backward (chunk_alu.cuh, bwd_unit).
+size_t tc_exact_scratch_bytes(const hgrn2_desc *d) { return (size_t)d->B * d->H * kD * kD * sizeof(float); }
+
+static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag, int *unit_count)
+{
+    ExactArgs ex;
+    ex.o = static_cast<const __nv_bfloat16 *>(a.o);
+    ex.f = static_cast<const __nv_bfloat16 *>(a.f);
+    ex.i = static_cast<const __nv_bfloat16 *>(a.i);
+    ex.S0 = a.S0;
+    ex.y = static_cast<__nv_bfloat16 *>(a.y);
+    ex.SN = a.SN;
+    ex.states = reinterpret_cast<__nv_bfloat16 *>(a.states);
+    ex.N = N_unit;
+    ex.G = G;
+    ex.unit_flag = unit_flag;
+    ex.unit_count = unit_count;
+    return ex;
 }
 
 static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *S0, float *SN, float *seg_decay,
-                                   bool want_y, bool want_saved, bool clear)
+                                   bool want_y, bool want_saved, bool clear, const ExactArgs &ex)
 {
     CUtensorMap mo, mf, mi, my, ms;
     // tensor maps need a valid base even for outputs that are not wanted: point those at an input
@@ -576,13 +645,16 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
         !make_map(&my, ybase, U, N, kC) || !make_map(&ms, sbase, sunits, srows, want_saved ? kD : kC))
         return cudaErrorInvalidValue;
     const bool ragged = N % kC != 0;
-    auto kernel = seg_decay ? (ragged ? tc_fwd_kernel<true, true> : tc_fwd_kernel<true, false>)
-                            : (ragged ? tc_fwd_kernel<false, true> : tc_fwd_kernel<false, false>);
+    if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
+    auto kernel = seg_decay ? (ragged ? tc_fwd_kernel<true, true, false> : tc_fwd_kernel<true, false, false>)
+                            : (ragged ? tc_fwd_kernel<false, true, false>
+                                      : (ex.o != nullptr && ex.G > 1 ? tc_fwd_kernel<false, false, true>
+                                                                      : tc_fwd_kernel<false, false, false>));
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? a.totals : nullptr;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, seg_decay, want_y,
-                                                                   want_saved, N, NC, a.status, clear ? 1 : 0);
+                                                                   want_saved, N, NC, a.status, clear ? 1 : 0, ex);
     return cudaGetLastError();
 }
 
@@ -597,7 +669,8 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
     bool clear = a.clear_status;                                  // for the first kernel launched only
     if (plan.main_units) {
         const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
-        err = launch_fwd_once(m, plan.main_units, a.N, a.NC, m.S0, m.SN, nullptr, want_y, want_saved, clear);
+        err = launch_fwd_once(m, plan.main_units, a.N, a.NC, m.S0, m.SN, nullptr, want_y, want_saved, clear,
+                              exact_args(m, a.N, 1, nullptr, nullptr));
         if (err != cudaSuccess) return err;
         clear = false;
     }
@@ -609,11 +682,15 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         float *S_loc = static_cast<float *>(a.seg_scratch);
         float *S_start = S_loc + Ut * G * kD * kD;
         float *lam = S_start + Ut * G * kD * kD;
-        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false, clear);
+        int *unit_flag = reinterpret_cast<int *>(lam + Ut * G * kD), *unit_count = unit_flag + Ut;
+        // the state-only pass needs no exact path of its own: the full pass below meets the same decays
+        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false, clear, ExactArgs{});
         if (err != cudaSuccess) return err;
-        seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G);
+        seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G,
+                                                                                unit_flag, unit_count, (int)Ut);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, want_y, want_saved, false);
+        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, want_y, want_saved, false,
+                              exact_args(t, a.N, G, unit_flag, unit_count));
     }
     return err;
 }

@@ -17,7 +17,8 @@ constexpr float kFMin = 7.888609052210118e-31f;   // 2^-100
 struct StatusBlock {
     int32_t code;      // hgrn2_status, 0 = ok; first error wins
     int32_t where;     // kernel-specific location tag of the first error
-    int32_t pad[62];
+    int32_t exact_units;   // tensor-core path: units the call redid on the exact fp32 path (decay out of range)
+    int32_t pad[61];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
 
@@ -56,6 +57,7 @@ struct SeqArgs {
     float *dS0;                   // nullable
     StatusBlock *status;
     void *seg_scratch;            // tensor-core path: scratch for sequences split into segments (nullable)
+    float *exact_scratch = nullptr;   // tensor-core backward: [B*H][dk][dv] floats for units redone on the exact path
     float *totals = nullptr;      // tensor-core path: per-chunk decay totals inside the saved data (set by its launchers)
     bool clear_status = false;    // tensor-core path: the first kernel of the call zeroes the status word itself
     cudaStream_t stream;
@@ -68,6 +70,22 @@ struct StepArgs {
     float *S;
     void *y;
     cudaStream_t stream;
+};
+
+// Tensor-core path: what a CTA needs to redo a whole unit on the exact fp32 path (chunk_alu.cuh) after its
+// sweep has found a decay that the rescaled operands cannot represent.  Plain pointers to unit 0 of the launch
+// (the kernels proper work through tensor maps); o == nullptr switches the exact path off.
+struct ExactArgs {
+    const __nv_bfloat16 *o = nullptr, *f = nullptr, *i = nullptr, *dy = nullptr;
+    const float *S0 = nullptr, *dSN = nullptr;
+    __nv_bfloat16 *y = nullptr, *d_o = nullptr, *d_f = nullptr, *d_i = nullptr;
+    float *SN = nullptr, *dS0 = nullptr;
+    __nv_bfloat16 *states = nullptr;    // saved chunk states: [unit][chunk of 64][128][128] bf16
+    float *scratch = nullptr;           // backward: [unit][128][128] floats
+    int N = 0;                          // tokens of a whole unit
+    int G = 1;                          // CTAs (segments) per unit in this launch
+    int *unit_flag = nullptr;           // G > 1: per unit, set by any segment that left the range
+    int *unit_count = nullptr;          // G > 1: per unit, segments finished so far
 };
 
 // Tensor-core path, few or left-over units: which units run whole and which are split into G segments each.

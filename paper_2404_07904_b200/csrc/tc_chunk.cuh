@@ -15,8 +15,11 @@
 //
 // The factors exp(b_t - b_m) are in-chunk cumulative PRODUCTS of f taken outward from the middle
 // (the linear-space image of the log-space cumulative sum): rows after m multiply by prod f, rows
-// before m divide by it.  Products are floored at 2^-100, so extreme decay inside half a chunk
-// (more than 2^100 across 32 steps) loses accuracy but never produces Inf or NaN.
+// before m divide by it.  The two factors of a pair can be represented only while the decay across each
+// half of the chunk stays above 2^-100 per key dimension.  Products are floored there (so nothing becomes
+// Inf or NaN); a half whose total Pm or E sits on the floor has left the range, which the state warps of
+// both kernels see when they pick the totals up: they raise the CTA's exact-path flag and the kernels then
+// redo the whole unit with the pairwise-safe fp32 routines of chunk_alu.cuh, which hold on all of [0, 1].
 #pragma once
 
 #include "tc_common.cuh"
@@ -132,6 +135,7 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
             *reinterpret_cast<uint32_t *>(fbuf + off) = fma_bf16x2(fw[j], skp ^ 0x80008000u, skp);
         }
     }
+    // the products only shrink along the walk, so the last one tells whether any row met the floor
     const float2 t2 = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
     if (tot) *reinterpret_cast<float2 *>(tot + col) = t2;
     if (tot_g) *reinterpret_cast<float2 *>(tot_g + col) = t2;
