@@ -8,9 +8,17 @@ calls) is timed separately and reported in the same JSON line under "decode".
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-With N > 1 the script expects to be launched by torch.distributed.run, one rank per GPU; the
-(batch, head) units are independent, so every rank runs the same per-GPU workload (weak
-scaling) and no collective touches the data path.
+With N > 1 it runs one rank per GPU: either launched by torch.distributed.run, or - when started as a
+plain `python bench.py --gpus N` - it starts its own ranks by re-executing itself under
+torch.distributed.run on 127.0.0.1.  The (batch, head) units are independent, so every rank runs the
+same per-GPU workload (weak scaling) and no collective touches the data path.
+
+Timing.  The step loop is timed in batches of exactly K steps (CUDA events on the launching stream, a
+barrier and a device synchronise on both sides, max over ranks); batches are repeated until at least
+--min-seconds of device time have been spent, so that the SM clock is sampled under a sustained load, and
+the MEDIAN batch is reported (`value`, `ms_per_step`; the spread is in `timing`).  `roofline.kernels` and the
+dominant-kernel figures come from separate loops of one kernel alone (forward only, backward only); those
+find different data in L2 than the alternating step does, so their sum differs from the step by a few %.
 """
 from __future__ import annotations
 
@@ -32,9 +40,11 @@ if ROOT not in sys.path:
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (captured on the same workloads the bench times: lm_2048 and the full decode batch).
-NCU_TRAFFIC_BYTES = {"fwd": 201.40e6 + 154.21e6, "bwd": 406.95e6 + 170.12e6, "step": 271.60e6 + 212.48e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu captures summarised under
+# profiles/ (same workloads as timed here: lm_2048 and the full decode batch); nothing here measures traffic.
+# None = the kernel has changed since its counters were taken.
+NCU_TRAFFIC_BYTES = {"fwd": None, "bwd": None, "step": 271.60e6 + 212.48e6}
+NCU_TRAFFIC_SOURCE = {"fwd": None, "bwd": None, "step": "profiles/step_kernel_decode.md"}
 
 
 def load_peaks():
@@ -123,8 +133,11 @@ class ClockSampler:
                     reasons.add(name)
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        hist = {}
+        for v in sm:
+            hist[str(int(v))] = hist.get(str(int(v)), 0) + 1
+        return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": max(mx),
+                "reasons": sorted(reasons), "samples": len(sm), "sm_mhz_hist": hist}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -263,7 +276,7 @@ def run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf):
     out = []
     if rank != 0:
         return out
-    for name, gamma in (("long_16k", None), ("lm_2560", 0.9)):
+    for name, gamma in (("long_16k", None),) + tuple(("lm_2560", g) for g in W.LM_2560_GAMMAS):
         w = W.CONFIGS[name]
         inp = W.make_inputs(w, gamma=gamma)
         t = {k: (None if v is None else torch.from_numpy(v).to(dev)) for k, v in inp.items()}
@@ -293,12 +306,16 @@ def run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf):
         ms = timed(step, n) / n
         ms_f = timed(fwd, n) / n
         ms_b = timed(bwd, n) / n
+        torch.cuda.synchronize()
+        assert binding.hgrn2_poll(ws) == 0, f"device-side error on {name}"
         ab = train_bytes(w)
         state_bytes = 4 * w.B * w.H * w.dk * w.dv * 4 if w.has_S0 else 0
         t_hbm = (ab["fwd"] + ab["bwd"] + state_bytes) / (peaks["hbm_gbs"] * 1e9)
         out.append({"workload": name, "B": w.B, "H": w.H, "N": w.N, "gamma": w.gamma if gamma is None else gamma,
                     "units": w.B * w.H, "ms_per_step": ms, "fwd_ms": ms_f, "bwd_ms": ms_b,
-                    "tokens_per_s": w.tokens / (ms * 1e-3), "frac_of_hbm_roofline": t_hbm * 1e3 / ms})
+                    "tokens_per_s": w.tokens / (ms * 1e-3), "frac_of_hbm_roofline": t_hbm * 1e3 / ms,
+                    "frac_of_nominal_hbm_roofline": t_hbm * 1e3 / ms * peaks["hbm_gbs"] / NOMINAL["hbm_gbs"],
+                    "exact_path_units": binding.exact_path_units(ws)})
         del o, f, i, dy, saved, ws, y, d_o, d_f, d_i
         torch.cuda.empty_cache()
     return out
@@ -314,8 +331,7 @@ def run_cuda(args):
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if world != args.gpus:
-        if world == 1 and args.gpus > 1:
-            raise SystemExit("for --gpus N > 1 launch with: python -m torch.distributed.run --nproc-per-node N bench.py --gpus N ...")
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s)")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
     if rank == 0:
@@ -427,11 +443,21 @@ def run_cuda(args):
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
     if rank == 0:
         sampler.start()
-    ms_total = max_over_ranks(timed(step, K))
-    ms_fwd = max_over_ranks(timed(fwd, K))
-    ms_bwd = max_over_ranks(timed(bwd, K))
+    # batches of exactly K steps until at least --min-seconds of device time; every rank takes the same number of
+    # batches because the continue/stop decision is made on the max-over-ranks times
+    batch_ms, spent = [], 0.0
+    while True:
+        batch_ms.append(max_over_ranks(timed(step, K)))
+        spent += batch_ms[-1] * 1e-3
+        if spent >= args.min_seconds or len(batch_ms) >= 100000:
+            break
     if rank == 0:
         sampler.stop()
+    clocks = sampler.summary()
+    ms_total = statistics.median(batch_ms)
+    # isolated kernel loops (their own L2 state: see the module docstring)
+    ms_fwd = max_over_ranks(timed(fwd, K))
+    ms_bwd = max_over_ranks(timed(bwd, K))
     for _ in range(2):
         e2e_step()
     torch.cuda.synchronize()
@@ -445,6 +471,7 @@ def run_cuda(args):
     assert e2e_err < 1e-2, f"end-to-end path disagrees with the device-resident path: {e2e_err}"
     ms_e2e = max_over_ranks(timed(e2e_step, max(3, min(K, 10)))) / max(3, min(K, 10))
     assert binding.hgrn2_poll(ws) == 0, "device-side error during the timed region"
+    assert binding.exact_path_units(ws) == 0, "the benchmark workload must stay on the tensor-core kernels"
 
     ms_step = ms_total / K
     tokens_per_step = world * w.tokens
@@ -454,25 +481,44 @@ def run_cuda(args):
     fl = train_flops(w)
     kern = {}
     for name, ms in (("fwd", ms_fwd / K), ("bwd", ms_bwd / K)):
-        kern[name] = {"ms": ms, "GBps": ab[name] / (ms * 1e-3) / 1e9, "TFLOPs": fl[name] / (ms * 1e-3) / 1e12}
+        kern[name] = {"ms": ms, "GBps": ab[name] / (ms * 1e-3) / 1e9, "TFLOPs": fl[name] / (ms * 1e-3) / 1e12,
+                      "timed": "isolated loop of this kernel alone"}
     dom = "bwd" if kern["bwd"]["ms"] >= kern["fwd"]["ms"] else "fwd"
-    # roofline of the whole step: the slower of bytes at HBM bandwidth and FLOPs at dense bf16 peak
-    t_hbm = (ab["fwd"] + ab["bwd"]) / (peaks["hbm_gbs"] * 1e9)
-    t_tc = (fl["fwd"] + fl["bwd"]) / (peaks["bf16_tflops_sustained"] * 1e12)
-    roof_tokens = w.tokens / max(t_hbm, t_tc)
+    # Roofline of a pass = the slower of its bytes at HBM bandwidth and its FLOPs at the dense bf16 rate.  Measured
+    # peaks: the burst GEMM rate for a kernel timed alone, the sustained one for the seconds-long step loop.
+    def bound_of(nbytes, flops, tf_key):
+        t_h = nbytes / (peaks["hbm_gbs"] * 1e9)
+        t_t = flops / (peaks[tf_key] * 1e12)
+        t_hn = nbytes / (NOMINAL["hbm_gbs"] * 1e9)
+        t_tn = flops / (NOMINAL["bf16_tflops"] * 1e12)
+        return {"bound": "hbm" if t_h >= t_t else "tensor", "t_hbm_us": t_h * 1e6, "t_tensor_us": t_t * 1e6,
+                "t_roof_us": max(t_h, t_t) * 1e6, "t_roof_nominal_us": max(t_hn, t_tn) * 1e6}
+    rk = bound_of(ab[dom], fl[dom], "bf16_tflops")
+    rs = bound_of(ab["fwd"] + ab["bwd"], fl["fwd"] + fl["bwd"], "bf16_tflops_sustained")
+    sm_mhz = clocks.get("sm_mhz")
     roofline = {
-        "bound": "hbm", "kernel": f"hgrn2_{dom} ({path})", "achieved": kern[dom]["GBps"], "peak": peaks["hbm_gbs"],
+        "bound": rk["bound"], "kernel": f"hgrn2_{dom} ({path})", "achieved": kern[dom]["GBps"], "peak": peaks["hbm_gbs"],
         "unit": "GB/s", "frac": kern[dom]["GBps"] / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES[dom],
+        "traffic_source": NCU_TRAFFIC_SOURCE[dom],
         "peak_source": f"of {peak_kind}", "algorithmic_bytes_per_launch": ab[dom],
-        "frac_nominal": kern[dom]["GBps"] / NOMINAL["hbm_gbs"],
-        "step": {"roofline_tokens_per_s": roof_tokens, "frac": (value / world) / roof_tokens,
-                 "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6},
+        "frac_nominal": kern[dom]["GBps"] / NOMINAL["hbm_gbs"], "timed": "isolated loop of the dominant kernel",
+        "step": {"timed": "median batch of the fwd+bwd step loop (the line's value)", "bound": rs["bound"],
+                 "t_hbm_us": rs["t_hbm_us"], "t_tensor_us": rs["t_tensor_us"],
+                 "roofline_tokens_per_s": w.tokens / (rs["t_roof_us"] * 1e-6),
+                 "frac": rs["t_roof_us"] * 1e-3 / ms_step, "frac_source": f"of {peak_kind}",
+                 "frac_nominal": rs["t_roof_nominal_us"] * 1e-3 / ms_step,
+                 "nominal": dict(NOMINAL),
+                 "sm_mhz_median": sm_mhz,
+                 "sm_cycles_per_step": (ms_step * 1e-3 * sm_mhz * 1e6) if sm_mhz else None},
         "kernels": kern,
     }
+    timing = {"batches": len(batch_ms), "steps_per_batch": K, "seconds": spent,
+              "ms_per_step_median": ms_step, "ms_per_step_min": min(batch_ms) / K, "ms_per_step_max": max(batch_ms) / K}
 
     if args.only == "train":
         if rank == 0:
-            print(json.dumps({"only": "train", "ms_per_step": ms_step, "kernels": kern}), flush=True)
+            print(json.dumps({"only": "train", "ms_per_step": ms_step, "kernels": kern, "timing": timing,
+                              "clocks": clocks}), flush=True)
         return 0
     decode = run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks, peak_kind, bf)
     others = run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf) if not args.skip_others else []
@@ -506,11 +552,47 @@ def run_cuda(args):
                 "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in host.values()),
                 "d2h_bytes_per_step": sum(v.numel() * v.element_size() for v in host_out.values())},
         "gpu_launches": 2 * K,
-        "clocks": sampler.summary(),
+        "timing": timing,
+        "clocks": clocks,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+    return 0
+
+
+def self_launch(argv, n):
+    """Start n ranks of this script under torch.distributed.run on this node and return their exit code."""
+    import socket
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    return subprocess.call(cmd, env=env)
+
+
+def run_launch_check(args):
+    """Stub arm for the launcher path (no GPU): the ranks rendezvous over gloo, take the barrier and the
+    max-over-ranks reduction the CUDA arm uses for its timings, and rank 0 prints one JSON line."""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    t = torch.tensor([100.0 + rank], dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"impl": "launch-check", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                          "max_over_ranks": float(t.item())}), flush=True)
     return 0
 
 
@@ -519,14 +601,20 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference", "launch-check"])
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="repeat the timed K-step batch until this much device time has been spent (median batch reported)")
     ap.add_argument("--only", default="all", choices=["all", "train", "decode"],
                     help="restrict the run to one part (for profiling); the JSON line is printed for 'all' only")
     ap.add_argument("--decode-steps", type=int, default=0, help="decode calls to time (0 = the workload's 512)")
     ap.add_argument("--skip-others", action="store_true", help="do not time the long-context and larger-layer workloads")
     args = ap.parse_args()
     if args.impl == "reference":
-        return run_reference(args)
+        return run_reference(args)      # rank 0 alone works, with or without a launcher
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return self_launch(sys.argv[1:], args.gpus)
+    if args.impl == "launch-check":
+        return run_launch_check(args)
     return run_cuda(args)
 
 

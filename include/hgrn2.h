@@ -146,7 +146,10 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
  *     or different host threads without ordering) race on the array and must be serialised by
  *     the caller.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress,
- *     with that device current).  Make that first call outside any stream capture.
+ *     with that device current).  Make that first call outside any stream capture.  With CUDA's
+ *     lazy module loading this is also the moment the driver sets the array's memory aside, so
+ *     make it early - a warm-up call per device at start-up, e.g. with N = 0 - while the device
+ *     still has 32 MiB free: once a pool owns all memory the lookup fails with HGRN2_ERR_CUDA.
  * Errors: as hgrn2_bwd, plus HGRN2_ERR_WORKSPACE as above and HGRN2_ERR_CUDA if the address
  * lookup fails. */
 hgrn2_status hgrn2_bwd_static_scratch(const hgrn2_desc *desc, const void *o, const void *f,

@@ -220,6 +220,7 @@ hgrn2_status hgrn2_step(const hgrn2_desc *desc, const void *o, const void *f, co
 {
     if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
     if (!dim_ok(desc->dk) || !dim_ok(desc->dv)) return HGRN2_ERR_UNSUPPORTED;
+    if ((size_t)desc->B * desc->H == 0) return HGRN2_OK;         // no unit: nothing to update, pointers may be NULL
     const void *req[] = {o, f, i, S, y};
     hgrn2_status st = check_ptrs(req, 5, nullptr, 0);
     if (st != HGRN2_OK) return st;

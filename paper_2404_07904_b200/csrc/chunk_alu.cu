@@ -49,7 +49,7 @@ cudaError_t launch_fwd_t(const SeqArgs &a)
     const size_t smem = alu::fwd_smem_floats(a.dk, a.dv, a.C) * sizeof(float);
     cudaError_t err = cudaFuncSetAttribute(alu_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    alu_fwd_kernel<T><<<a.B * a.H, kAluThreads, smem, a.stream>>>(
+    alu_fwd_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i), a.S0,
         static_cast<T *>(a.y), a.SN, a.states, a.N, a.dk, a.dv, a.C, a.NC);
     return cudaGetLastError();
@@ -61,7 +61,7 @@ cudaError_t launch_bwd_t(const SeqArgs &a)
     const size_t smem = alu::bwd_smem_floats(a.dk, a.dv, a.C) * sizeof(float);
     cudaError_t err = cudaFuncSetAttribute(alu_bwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    alu_bwd_kernel<T><<<a.B * a.H, kAluThreads, smem, a.stream>>>(
+    alu_bwd_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i),
         static_cast<const T *>(a.dy), a.dSN, a.states, static_cast<T *>(a.d_o), static_cast<T *>(a.d_f),
         static_cast<T *>(a.d_i), a.dS0, a.N, a.dk, a.dv, a.C, a.NC);
@@ -84,15 +84,20 @@ int alu_default_chunk(int dk, int dv)
     return 0;
 }
 
+// one CTA per unit: the unit count must fit the grid's x dimension
+static bool grid_ok(const SeqArgs &a) { return (long long)a.B * a.H <= 0x7fffffffLL; }
+
 cudaError_t launch_alu_fwd(const SeqArgs &a)
 {
     if ((long long)a.B * a.H == 0 || a.N == 0) return cudaSuccess;
+    if (!grid_ok(a)) return cudaErrorInvalidConfiguration;
     return a.io == HGRN2_BF16 ? launch_fwd_t<__nv_bfloat16>(a) : launch_fwd_t<float>(a);
 }
 
 cudaError_t launch_alu_bwd(const SeqArgs &a)
 {
     if ((long long)a.B * a.H == 0 || a.N == 0) return cudaSuccess;
+    if (!grid_ok(a)) return cudaErrorInvalidConfiguration;
     return a.io == HGRN2_BF16 ? launch_bwd_t<__nv_bfloat16>(a) : launch_bwd_t<float>(a);
 }
 

@@ -62,3 +62,17 @@ def test_two_rank_unit_sharding_matches_single_process(tmp_path):
     got = np.load(tmp_path / "y.npy").reshape(y.shape)
     np.testing.assert_array_equal(got, y)
     assert float(np.load(tmp_path / "t.npy")[0]) == 11.0
+
+
+def test_bench_starts_its_own_ranks():
+    # `python bench.py --gpus 2` with no launcher around it must re-execute itself under torch.distributed.run
+    # and print one JSON line from rank 0; driven here with the CPU stub arm (gloo)
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "launch-check",
+                          "--steps", "3", "--warmup", "1"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["max_over_ranks"] == 101.0 and lines[0]["steps"] == 3

@@ -51,6 +51,25 @@ def test_two_calls_in_a_row_match_hgrn2_bwd(io):
             assert err <= G.TOL[io], (name, err)
 
 
+def test_matches_the_oracle_and_serves_segmented_sequences():
+    # few units: the sequences run as several segments, whose scratch also lives in the built-in array; outputs
+    # against hgrn2_bwd and, for two units, against the fp64 oracle
+    w = W.scaled(W.CONFIGS["long_16k"], B=1, H=4, N=2048, seed=33)
+    d = binding.make_desc(w.B, w.H, w.N, w.dk, w.dv, binding.HGRN2_BF16)
+    assert binding.workspace_bytes(d) - 256 <= binding.STATIC_SCRATCH_BYTES
+    assert binding.workspace_bytes(d) > 256 + binding.saved_bytes(d) + w.B * w.H * w.dk * w.dv * 4, "segment scratch expected"
+    inp = W.make_inputs(w)
+    t = G.to_dev(inp, "bf16")
+    want = _reference(t, w.chunk)
+    got = _static(t, w.chunk)
+    names = ("d_o", "d_f", "d_i", "dS0")
+    for name, g, r in zip(names, got, want):
+        assert G.rel_err(g.float().cpu().numpy(), r.float().cpu().numpy()) <= G.TOL["bf16"], name
+    for (b, h), wu in G.oracle_fwd_bwd(inp, [(0, 0), (0, 3)]).items():
+        gu = {name: g[b:b + 1, h:h + 1].float().cpu().numpy() for name, g in zip(names, got)}
+        G.assert_close(gu, {k: wu[k] for k in names}, G.TOL["bf16"], f"static scratch vs oracle, unit {(b, h)}")
+
+
 def test_rejects_problems_larger_than_the_array():
     # 8 x 16 heads x 32 chunks x 32 KB of bf16 states = 128 MB > 32 MB: refused on the host, nothing runs
     d = binding.make_desc(8, 16, 2048, 128, 128, binding.HGRN2_BF16)
