@@ -318,7 +318,71 @@ def run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf):
                     "exact_path_units": binding.exact_path_units(ws)})
         del o, f, i, dy, saved, ws, y, d_o, d_f, d_i
         torch.cuda.empty_cache()
+    out.append(run_packed_mix(binding, W, dev, timed, peaks, bf))
     return out
+
+
+# A ragged batch as a long-context fine-tuning step would see it: 24 sequences between 256 and 4096 tokens
+# (longest first), 16 heads of 128.  Timed packed (hgrn2_*_varlen) and padded to the longest (hgrn2_fwd/bwd).
+PACKED_MIX_LENGTHS = (4096, 3072, 2048, 2048, 1536, 1024, 1024, 1024, 1024, 768, 768, 768, 512, 512, 512, 512,
+                      384, 384, 256, 256, 256, 256, 256, 256)
+
+
+def run_packed_mix(binding, W, dev, timed, peaks, bf):
+    import torch
+    lengths = PACKED_MIX_LENGTHS
+    H, d, B, T, Nmax = 16, 128, len(lengths), int(sum(lengths)), max(lengths)
+    w = W.scaled(W.CONFIGS["lm_2048"], B=1, H=H, N=T, seed=9)
+    inp = W.make_inputs(w)
+    pk = {k: torch.from_numpy(inp[k][0]).to(dev).to(bf) for k in ("o", "f", "i", "dy")}
+    cu_h = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    cu = torch.from_numpy(cu_h).to(dev)
+    # the padded equivalent: [B, H, Nmax, d] with neutral tokens (f = 1, o = i = dy = 0) after each sequence's end
+    pad = {k: torch.zeros((B, H, Nmax, d), dtype=bf, device=dev) for k in pk}
+    pad["f"].fill_(1.0)
+    for b in range(B):
+        s, e = int(cu_h[b]), int(cu_h[b + 1])
+        for k in pk:
+            pad[k][b, :, :e - s] = pk[k][:, s:e]
+    res = {"workload": "packed_mix", "sequences": B, "H": H, "tokens": T, "longest": Nmax, "padded_tokens": B * Nmax}
+    y, SN, saved, ws, _ = binding.hgrn2_fwd_varlen(pk["o"], pk["f"], pk["i"], cu, None, want_final_state=False)
+    outs = [torch.empty_like(pk["o"]) for _ in range(3)]
+
+    def step_packed():
+        binding.hgrn2_fwd_varlen(pk["o"], pk["f"], pk["i"], cu, None, y=y, saved=saved, ws=ws, want_final_state=False)
+        binding.hgrn2_bwd_varlen(pk["o"], pk["f"], pk["i"], cu, None, pk["dy"], None, saved, d_o=outs[0], d_f=outs[1],
+                                 d_i=outs[2], ws=ws, want_dS0=False)
+
+    for _ in range(3):
+        step_packed()
+    n = 10
+    ms_p = timed(step_packed, n) / n
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws) == 0
+    y_packed = y.clone()
+    del saved, ws, outs
+    yp, _, saved2, ws2, _ = binding.hgrn2_fwd(pad["o"], pad["f"], pad["i"], None, want_final_state=False)
+    outs2 = [torch.empty_like(pad["o"]) for _ in range(3)]
+
+    def step_padded():
+        binding.hgrn2_fwd(pad["o"], pad["f"], pad["i"], None, y=yp, saved=saved2, ws=ws2, want_final_state=False)
+        binding.hgrn2_bwd(pad["o"], pad["f"], pad["i"], None, pad["dy"], None, saved2, d_o=outs2[0], d_f=outs2[1],
+                          d_i=outs2[2], ws=ws2, want_dS0=False)
+
+    for _ in range(3):
+        step_padded()
+    ms_d = timed(step_padded, n) / n
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws2) == 0
+    # both layouts must agree on the real tokens (padding with the neutral token is exact)
+    s, e = int(cu_h[3]), int(cu_h[4])
+    diff = (y_packed[:, s:e].float() - yp[3, :, :e - s].float()).abs().max() / yp[3, :, :e - s].float().abs().max()
+    assert float(diff) < 1e-2, f"packed and padded results differ: {float(diff)}"
+    bytes_real = 11 * H * T * d * 2
+    res.update({"ms_per_step_packed": ms_p, "ms_per_step_padded": ms_d, "tokens_per_s_packed": T / (ms_p * 1e-3),
+                "tokens_per_s_padded": T / (ms_d * 1e-3), "speedup_over_padded": ms_d / ms_p,
+                "frac_of_hbm_roofline_packed": bytes_real / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_p})
+    return res
 
 
 def run_cuda(args):

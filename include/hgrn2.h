@@ -118,6 +118,33 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
                        void *d_o, void *d_f, void *d_i, float *dS0, void *ws,
                        void *cuda_stream);
 
+/* Variable-length (packed) batches.  Eq. 3 runs over each sequence separately - the state is reset to the
+ * sequence's own initial state at every boundary - and a recurrent model's cost is linear in the tokens actually
+ * present (Section 1: linear-time inference with a constant-size state), so ragged batches are passed packed
+ * instead of padded to a common length:
+ *   desc->B = number of sequences, desc->N = T, the total number of token rows per head, desc->H heads;
+ *   o, f [H][T][dk], i, y, dy [H][T][dv] and the gradients likewise (desc->io), device memory, 16-byte aligned;
+ *   cu_seqlens  int32[B + 1] in DEVICE memory, 4-byte aligned: sequence b occupies rows [cu[b], cu[b+1]) of every
+ *               head; cu[0] = 0, non-decreasing, cu[B] <= T.  Empty sequences are allowed (their state passes
+ *               through).  The offsets are read on the device only; malformed ones make the affected units write
+ *               nothing and, on the tensor-core path, put HGRN2_ERR_INVALID_ARG into the status word.
+ *   S0, SN, dSN, dS0 [B][H][dk][dv] float32: one state per (sequence, head), NULL as in hgrn2_fwd / hgrn2_bwd;
+ *   saved  hgrn2_saved_bytes_varlen(desc) bytes (NULL as in hgrn2_fwd / hgrn2_bwd);
+ *   ws     hgrn2_workspace_bytes_varlen(desc) bytes.
+ * Everything else - ownership, streams, errors, the closed interval for f - is as for hgrn2_fwd / hgrn2_bwd.
+ * One CTA serves one (sequence, head) unit, dispatched in index order: with more units than SMs, put long
+ * sequences first.  Sequences are not split into segments here, so a batch of few long sequences is better
+ * served by hgrn2_fwd. */
+size_t hgrn2_saved_bytes_varlen(const hgrn2_desc *desc);
+size_t hgrn2_workspace_bytes_varlen(const hgrn2_desc *desc);
+hgrn2_status hgrn2_fwd_varlen(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                              const int32_t *cu_seqlens, const float *S0, void *y, float *SN,
+                              void *saved, void *ws, void *cuda_stream);
+hgrn2_status hgrn2_bwd_varlen(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                              const int32_t *cu_seqlens, const float *S0, const void *dy,
+                              const float *dSN, const void *saved, void *d_o, void *d_f, void *d_i,
+                              float *dS0, void *ws, void *cuda_stream);
+
 /* Largest chunk-state scratch, in bytes, that hgrn2_bwd_static_scratch can serve. */
 #define HGRN2_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
 

@@ -126,3 +126,45 @@ def hgrn2_step(o, f, i, S):
     rc = _load().ref_hgrn2_step(B, H, dk, dv, op, fp, ip, S.ctypes.data_as(_DP), yp)
     _check(rc, "ref_hgrn2_step")
     return y
+
+
+def hgrn2_fwd_varlen(o, f, i, cu, S0=None):
+    """Packed batch: o, f [H, T, d_k], i [H, T, d_v]; sequence b occupies rows cu[b]:cu[b+1] of every head and
+    starts from S0[b] ([B, H, d_k, d_v], or zero).  No arithmetic of its own: every sequence goes through
+    hgrn2_fwd (Eq. 3) separately.  Returns (y [H, T, d_v], S_N [B, H, d_k, d_v])."""
+    H, T, dk = o.shape
+    dv = i.shape[-1]
+    B = len(cu) - 1
+    y = np.zeros((H, T, dv), dtype=np.float64)
+    SN = np.zeros((B, H, dk, dv), dtype=np.float64)
+    for b in range(B):
+        s, e = int(cu[b]), int(cu[b + 1])
+        s0 = None if S0 is None else np.asarray(S0[b:b + 1], dtype=np.float64)
+        if e == s:
+            SN[b] = 0.0 if s0 is None else s0[0]
+            continue
+        yb, snb = hgrn2_fwd(o[None, :, s:e], f[None, :, s:e], i[None, :, s:e], s0)
+        y[:, s:e] = yb[0]
+        SN[b] = snb[0]
+    return y, SN
+
+
+def hgrn2_bwd_varlen(o, f, i, cu, S0, dy, dSN=None):
+    """VJP of hgrn2_fwd_varlen, sequence by sequence through hgrn2_bwd.  Returns (d_o, d_f, d_i, dS0)."""
+    H, T, dk = o.shape
+    dv = i.shape[-1]
+    B = len(cu) - 1
+    d_o = np.zeros((H, T, dk), dtype=np.float64)
+    d_f = np.zeros((H, T, dk), dtype=np.float64)
+    d_i = np.zeros((H, T, dv), dtype=np.float64)
+    dS0 = np.zeros((B, H, dk, dv), dtype=np.float64)
+    for b in range(B):
+        s, e = int(cu[b]), int(cu[b + 1])
+        s0 = None if S0 is None else np.asarray(S0[b:b + 1], dtype=np.float64)
+        dsn = None if dSN is None else np.asarray(dSN[b:b + 1], dtype=np.float64)
+        if e == s:
+            dS0[b] = 0.0 if dsn is None else dsn[0]
+            continue
+        a, c, d, g = hgrn2_bwd(o[None, :, s:e], f[None, :, s:e], i[None, :, s:e], s0, dy[None, :, s:e], dsn)
+        d_o[:, s:e], d_f[:, s:e], d_i[:, s:e], dS0[b] = a[0], c[0], d[0], g[0]
+    return d_o, d_f, d_i, dS0

@@ -27,7 +27,8 @@ STATUS_NAMES = {
 EXPORTS = (
     "hgrn2_saved_bytes", "hgrn2_workspace_bytes", "hgrn2_fwd", "hgrn2_bwd", "hgrn2_step",
     "hgrn2_step_multi", "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path", "hgrn2_bwd_static_scratch",
-    "hgrn2_exact_path_units",
+    "hgrn2_exact_path_units", "hgrn2_saved_bytes_varlen", "hgrn2_workspace_bytes_varlen", "hgrn2_fwd_varlen",
+    "hgrn2_bwd_varlen",
 )
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
@@ -76,6 +77,14 @@ def load() -> ctypes.CDLL:
     lib.hgrn2_fwd.argtypes = [dp] + [vp] * 9
     lib.hgrn2_bwd.restype = ctypes.c_int
     lib.hgrn2_bwd.argtypes = [dp] + [vp] * 13
+    lib.hgrn2_saved_bytes_varlen.restype = ctypes.c_size_t
+    lib.hgrn2_saved_bytes_varlen.argtypes = [dp]
+    lib.hgrn2_workspace_bytes_varlen.restype = ctypes.c_size_t
+    lib.hgrn2_workspace_bytes_varlen.argtypes = [dp]
+    lib.hgrn2_fwd_varlen.restype = ctypes.c_int
+    lib.hgrn2_fwd_varlen.argtypes = [dp] + [vp] * 10
+    lib.hgrn2_bwd_varlen.restype = ctypes.c_int
+    lib.hgrn2_bwd_varlen.argtypes = [dp] + [vp] * 14
     lib.hgrn2_bwd_static_scratch.restype = ctypes.c_int
     lib.hgrn2_bwd_static_scratch.argtypes = [dp] + [vp] * 12
     lib.hgrn2_step.restype = ctypes.c_int
@@ -188,6 +197,55 @@ def hgrn2_bwd(o, f, i, S0, dy, dSN=None, saved=None, *, d_o=None, d_f=None, d_i=
     code = load().hgrn2_bwd(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(S0), _ptr(dy), _ptr(dSN),
                             _ptr(saved), _ptr(d_o), _ptr(d_f), _ptr(d_i), _ptr(dS0), _ptr(ws), _stream(stream))
     _check(code, "hgrn2_bwd")
+    return d_o, d_f, d_i, dS0, ws
+
+
+def hgrn2_fwd_varlen(o, f, i, cu_seqlens, S0=None, *, y=None, SN=None, saved=None, ws=None, want_final_state=True,
+                     save_for_backward=True, chunk=0, flags=0, stream=None):
+    """Forward over a packed batch: o, f [H, T, dk], i [H, T, dv]; cu_seqlens int32 [B + 1] on the device; states
+    [B, H, dk, dv].  Returns (y, SN, saved, ws, desc)."""
+    H, T, dk = o.shape
+    dv = i.shape[-1]
+    B = cu_seqlens.numel() - 1
+    if cu_seqlens.dtype != torch.int32:
+        raise TypeError("cu_seqlens must be int32")
+    desc = make_desc(B, H, T, dk, dv, _io_code(o), chunk, flags)
+    dev = o.device
+    if y is None:
+        y = torch.empty((H, T, dv), dtype=o.dtype, device=dev)
+    if SN is None and want_final_state:
+        SN = torch.empty((B, H, dk, dv), dtype=torch.float32, device=dev)
+    lib = load()
+    if saved is None and save_for_backward:
+        saved = torch.empty(max(int(lib.hgrn2_saved_bytes_varlen(ctypes.byref(desc))), 16), dtype=torch.uint8, device=dev)
+    if ws is None:
+        ws = torch.empty(int(lib.hgrn2_workspace_bytes_varlen(ctypes.byref(desc))), dtype=torch.uint8, device=dev)
+    code = lib.hgrn2_fwd_varlen(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(cu_seqlens), _ptr(S0), _ptr(y),
+                                _ptr(SN), _ptr(saved), _ptr(ws), _stream(stream))
+    _check(code, "hgrn2_fwd_varlen")
+    return y, SN, saved, ws, desc
+
+
+def hgrn2_bwd_varlen(o, f, i, cu_seqlens, S0, dy, dSN=None, saved=None, *, d_o=None, d_f=None, d_i=None, dS0=None,
+                     ws=None, want_dS0=True, chunk=0, flags=0, stream=None):
+    """Backward of hgrn2_fwd_varlen.  Returns (d_o, d_f, d_i, dS0, ws)."""
+    H, T, dk = o.shape
+    dv = i.shape[-1]
+    B = cu_seqlens.numel() - 1
+    desc = make_desc(B, H, T, dk, dv, _io_code(o), chunk, flags)
+    dev = o.device
+    d_o = torch.empty_like(o) if d_o is None else d_o
+    d_f = torch.empty_like(f) if d_f is None else d_f
+    d_i = torch.empty_like(i) if d_i is None else d_i
+    if dS0 is None and want_dS0:
+        dS0 = torch.empty((B, H, dk, dv), dtype=torch.float32, device=dev)
+    lib = load()
+    if ws is None:
+        ws = torch.empty(int(lib.hgrn2_workspace_bytes_varlen(ctypes.byref(desc))), dtype=torch.uint8, device=dev)
+    code = lib.hgrn2_bwd_varlen(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(i), _ptr(cu_seqlens), _ptr(S0), _ptr(dy),
+                                _ptr(dSN), _ptr(saved), _ptr(d_o), _ptr(d_f), _ptr(d_i), _ptr(dS0), _ptr(ws),
+                                _stream(stream))
+    _check(code, "hgrn2_bwd_varlen")
     return d_o, d_f, d_i, dS0, ws
 
 

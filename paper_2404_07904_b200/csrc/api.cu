@@ -15,6 +15,7 @@ bool        tc_chunk_supported(int C);
 size_t      tc_saved_bytes(const hgrn2_desc *d, int C);
 size_t      tc_segment_scratch_bytes(const hgrn2_desc *d, int C);
 size_t      tc_exact_scratch_bytes(const hgrn2_desc *d);
+size_t      tc_saved_bytes_packed(const hgrn2_desc *d);
 cudaError_t launch_tc_fwd(const SeqArgs &a);
 cudaError_t launch_tc_bwd(const SeqArgs &a);
 }  // namespace hgrn2
@@ -64,23 +65,32 @@ hgrn2_status check_ptrs(const void *const *req, int nreq, const void *const *opt
 
 size_t state_bytes(const hgrn2_desc *d) { return (size_t)d->B * d->H * d->dk * d->dv * sizeof(float); }
 
-size_t saved_bytes_for(const hgrn2_desc *d, int C)
+// packed = a variable-length batch: d->B sequences share d->N token rows per head (state slots: see PackedArgs)
+size_t saved_bytes_for(const hgrn2_desc *d, int C, bool packed = false)
 {
-    if (use_tc(d)) return tc_saved_bytes(d, C);
+    if (use_tc(d)) return packed ? tc_saved_bytes_packed(d) : tc_saved_bytes(d, C);
     const size_t NC = ((size_t)d->N + C - 1) / C;
-    return (size_t)d->B * d->H * NC * d->dk * d->dv * sizeof(float);
+    const size_t slots = packed ? (size_t)d->H * ((size_t)d->N / C + d->B + 1) : (size_t)d->B * d->H * NC;
+    return slots * d->dk * d->dv * sizeof(float);
 }
 
-void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream, void *ws)
+size_t workspace_bytes_for(const hgrn2_desc *d, int C, bool packed)
+{
+    return sizeof(StatusBlock) + saved_bytes_for(d, C, packed) +
+           (use_tc(d) ? (packed ? 0 : tc_segment_scratch_bytes(d, C)) + tc_exact_scratch_bytes(d) : 0);
+}
+
+void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream, void *ws, const int32_t *cu = nullptr)
 {
     memset(&a, 0, sizeof(a));
+    a.cu = cu;
     // workspace layout: status block | room for re-created saved data | tensor-core path: segment scratch, then one
     // float matrix per unit for units redone on the exact path
     a.seg_scratch = nullptr;
     a.exact_scratch = nullptr;
     if (use_tc(d)) {
-        char *p = static_cast<char *>(ws) + sizeof(StatusBlock) + saved_bytes_for(d, C);
-        const size_t seg = tc_segment_scratch_bytes(d, C);
+        char *p = static_cast<char *>(ws) + sizeof(StatusBlock) + saved_bytes_for(d, C, cu != nullptr);
+        const size_t seg = cu ? 0 : tc_segment_scratch_bytes(d, C);
         if (seg != 0) a.seg_scratch = p;
         a.exact_scratch = reinterpret_cast<float *>(p + seg);
     }
@@ -113,8 +123,21 @@ size_t hgrn2_workspace_bytes(const hgrn2_desc *desc)
 {
     const int C = resolve_chunk(desc);
     if (C == 0) return 0;
-    return sizeof(StatusBlock) + saved_bytes_for(desc, C) +
-           (use_tc(desc) ? tc_segment_scratch_bytes(desc, C) + tc_exact_scratch_bytes(desc) : 0);
+    return workspace_bytes_for(desc, C, false);
+}
+
+size_t hgrn2_saved_bytes_varlen(const hgrn2_desc *desc)
+{
+    const int C = resolve_chunk(desc);
+    if (C == 0) return 0;
+    return saved_bytes_for(desc, C, true);
+}
+
+size_t hgrn2_workspace_bytes_varlen(const hgrn2_desc *desc)
+{
+    const int C = resolve_chunk(desc);
+    if (C == 0) return 0;
+    return workspace_bytes_for(desc, C, true);
 }
 
 const char *hgrn2_status_string(hgrn2_status s)
@@ -132,8 +155,13 @@ const char *hgrn2_status_string(hgrn2_status s)
     return "unknown status";
 }
 
-hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
-                       const float *S0, void *y, float *SN, void *saved, void *ws, void *cuda_stream)
+}  // extern "C"
+
+namespace {
+
+// cu == nullptr: [B][H][N][d] tensors; otherwise a packed batch of desc->B sequences in [H][N][d] tensors
+hgrn2_status fwd_impl(const hgrn2_desc *desc, const void *o, const void *f, const void *i, const int32_t *cu,
+                      const float *S0, void *y, float *SN, void *saved, void *ws, void *cuda_stream)
 {
     if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
     const int C = resolve_chunk(desc);
@@ -146,7 +174,7 @@ hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, con
     if (st != HGRN2_OK) return st;
 
     SeqArgs a;
-    fill_args(a, desc, C, cuda_stream, ws);
+    fill_args(a, desc, C, cuda_stream, ws, cu);
     a.o = o; a.f = f; a.i = i; a.S0 = S0; a.y = y; a.SN = SN;
     a.states = static_cast<float *>(saved);
     a.status = static_cast<StatusBlock *>(ws);
@@ -168,9 +196,9 @@ hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, con
     return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
 }
 
-hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
-                       const float *S0, const void *dy, const float *dSN, const void *saved,
-                       void *d_o, void *d_f, void *d_i, float *dS0, void *ws, void *cuda_stream)
+hgrn2_status bwd_impl(const hgrn2_desc *desc, const void *o, const void *f, const void *i, const int32_t *cu,
+                      const float *S0, const void *dy, const float *dSN, const void *saved,
+                      void *d_o, void *d_f, void *d_i, float *dS0, void *ws, void *cuda_stream)
 {
     if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
     const int C = resolve_chunk(desc);
@@ -183,7 +211,7 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
     if (st != HGRN2_OK) return st;
 
     SeqArgs a;
-    fill_args(a, desc, C, cuda_stream, ws);
+    fill_args(a, desc, C, cuda_stream, ws, cu);
     a.o = o; a.f = f; a.i = i; a.S0 = S0; a.dy = dy; a.dSN = dSN;
     a.d_o = d_o; a.d_f = d_f; a.d_i = d_i; a.dS0 = dS0;
     a.status = static_cast<StatusBlock *>(ws);
@@ -213,6 +241,42 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
     }
     cudaError_t e = tc ? launch_tc_bwd(a) : launch_alu_bwd(a);
     return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+hgrn2_status hgrn2_fwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                       const float *S0, void *y, float *SN, void *saved, void *ws, void *cuda_stream)
+{
+    return fwd_impl(desc, o, f, i, nullptr, S0, y, SN, saved, ws, cuda_stream);
+}
+
+hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                       const float *S0, const void *dy, const float *dSN, const void *saved,
+                       void *d_o, void *d_f, void *d_i, float *dS0, void *ws, void *cuda_stream)
+{
+    return bwd_impl(desc, o, f, i, nullptr, S0, dy, dSN, saved, d_o, d_f, d_i, dS0, ws, cuda_stream);
+}
+
+hgrn2_status hgrn2_fwd_varlen(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                              const int32_t *cu_seqlens, const float *S0, void *y, float *SN, void *saved, void *ws,
+                              void *cuda_stream)
+{
+    if (!cu_seqlens) return HGRN2_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(cu_seqlens) & 3u) return HGRN2_ERR_ALIGNMENT;
+    return fwd_impl(desc, o, f, i, cu_seqlens, S0, y, SN, saved, ws, cuda_stream);
+}
+
+hgrn2_status hgrn2_bwd_varlen(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
+                              const int32_t *cu_seqlens, const float *S0, const void *dy, const float *dSN,
+                              const void *saved, void *d_o, void *d_f, void *d_i, float *dS0, void *ws,
+                              void *cuda_stream)
+{
+    if (!cu_seqlens) return HGRN2_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(cu_seqlens) & 3u) return HGRN2_ERR_ALIGNMENT;
+    return bwd_impl(desc, o, f, i, cu_seqlens, S0, dy, dSN, saved, d_o, d_f, d_i, dS0, ws, cuda_stream);
 }
 
 hgrn2_status hgrn2_step(const hgrn2_desc *desc, const void *o, const void *f, const void *i,

@@ -14,17 +14,33 @@ namespace {
 
 constexpr int kAluThreads = 256;
 
+// Where unit u lives: first token row in the [rows][d] view, tokens, chunks, first chunk-state slot.  Ordinary
+// layout: unit u owns rows [u N, u N + N).  Packed batch (cu set; unit = sequence b, head h; N rows per head):
+// rows [h N + cu[b], h N + cu[b + 1]), state slots from h (N / C + B + 1) + cu[b] / C + b.
+struct Geom { long long row; int n; int nc; long long slot; };
+__device__ inline Geom unit_geom(long long u, int N, int C, int NC, const int *cu, int H)
+{
+    if (cu == nullptr) return Geom{u * N, N, NC, u * NC};
+    const int B = gridDim.x / H;
+    const int b = (int)(u / H), h = (int)(u - (long long)b * H);
+    const int start = cu[b];
+    int n = cu[b + 1] - start;
+    if (start < 0 || n < 0 || start + n > N) n = 0;          // malformed offsets: touch nothing
+    return Geom{(long long)h * N + start, n, (n + C - 1) / C, (long long)h * (N / C + B + 1) + start / C + b};
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kAluThreads)
 alu_fwd_kernel(const T *__restrict__ o, const T *__restrict__ f, const T *__restrict__ i,
                const float *__restrict__ S0, T *__restrict__ y, float *__restrict__ SN,
-               float *__restrict__ states, int N, int dk, int dv, int C, int NC)
+               float *__restrict__ states, int N, int dk, int dv, int C, int NC, const int *__restrict__ cu, int H)
 {
     extern __shared__ float smem[];
     const long long u = blockIdx.x, ss = (long long)dk * dv;
-    alu::fwd_unit<T, float>(smem, o + u * N * dk, f + u * N * dk, i + u * N * dv, S0 ? S0 + u * ss : nullptr,
-                            y ? y + u * N * dv : nullptr, SN ? SN + u * ss : nullptr,
-                            states ? states + u * NC * ss : nullptr, 1, N, dk, dv, C, NC);
+    const Geom g = unit_geom(u, N, C, NC, cu, H);
+    alu::fwd_unit<T, float>(smem, o + g.row * dk, f + g.row * dk, i + g.row * dv, S0 ? S0 + u * ss : nullptr,
+                            y ? y + g.row * dv : nullptr, SN ? SN + u * ss : nullptr,
+                            states ? states + g.slot * ss : nullptr, 1, g.n, dk, dv, C, g.nc);
 }
 
 template <typename T>
@@ -32,13 +48,15 @@ __global__ void __launch_bounds__(kAluThreads)
 alu_bwd_kernel(const T *__restrict__ o, const T *__restrict__ f, const T *__restrict__ i,
                const T *__restrict__ dy, const float *__restrict__ dSN,
                const float *__restrict__ states, T *__restrict__ d_o, T *__restrict__ d_f,
-               T *__restrict__ d_i, float *__restrict__ dS0, int N, int dk, int dv, int C, int NC)
+               T *__restrict__ d_i, float *__restrict__ dS0, int N, int dk, int dv, int C, int NC,
+               const int *__restrict__ cu, int H)
 {
     extern __shared__ float smem[];
     const long long u = blockIdx.x, ss = (long long)dk * dv;
-    alu::bwd_unit<T, float>(smem, o + u * N * dk, f + u * N * dk, i + u * N * dv, dy + u * N * dv,
-                            dSN ? dSN + u * ss : nullptr, states + u * NC * ss, 1, nullptr, d_o + u * N * dk,
-                            d_f + u * N * dk, d_i + u * N * dv, dS0 ? dS0 + u * ss : nullptr, N, dk, dv, C, NC);
+    const Geom g = unit_geom(u, N, C, NC, cu, H);
+    alu::bwd_unit<T, float>(smem, o + g.row * dk, f + g.row * dk, i + g.row * dv, dy + g.row * dv,
+                            dSN ? dSN + u * ss : nullptr, states + g.slot * ss, 1, nullptr, d_o + g.row * dk,
+                            d_f + g.row * dk, d_i + g.row * dv, dS0 ? dS0 + u * ss : nullptr, g.n, dk, dv, C, g.nc);
 }
 
 constexpr size_t kMaxSmem = 227 * 1024;
@@ -51,7 +69,7 @@ cudaError_t launch_fwd_t(const SeqArgs &a)
     if (err != cudaSuccess) return err;
     alu_fwd_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i), a.S0,
-        static_cast<T *>(a.y), a.SN, a.states, a.N, a.dk, a.dv, a.C, a.NC);
+        static_cast<T *>(a.y), a.SN, a.states, a.N, a.dk, a.dv, a.C, a.NC, a.cu, a.H);
     return cudaGetLastError();
 }
 
@@ -64,7 +82,7 @@ cudaError_t launch_bwd_t(const SeqArgs &a)
     alu_bwd_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i),
         static_cast<const T *>(a.dy), a.dSN, a.states, static_cast<T *>(a.d_o), static_cast<T *>(a.d_f),
-        static_cast<T *>(a.d_i), a.dS0, a.N, a.dk, a.dv, a.C, a.NC);
+        static_cast<T *>(a.d_i), a.dS0, a.N, a.dk, a.dv, a.C, a.NC, a.cu, a.H);
     return cudaGetLastError();
 }
 

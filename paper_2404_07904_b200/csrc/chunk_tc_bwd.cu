@@ -110,8 +110,8 @@ static_assert(alu::bwd_smem_floats(kD, kD, kExactC) * sizeof(float) <= kSmemByte
 // d_o and the nearly finished d_f of one thread: key dimension k, local times [32 * kUp, 32 * kUp + 32),
 // walked outwards from the middle of the chunk in blocks of eight.  Returns this half's sums of a and e.
 // do_g points at element (row 0 of the chunk, column k) of d_o in global memory.  oraw, fraw: the chunk's raw
-// o and f as plain [64][128] bf16 tiles (rows beyond the end of the sequence read as zero there, so f is
-// patched to the neutral 1).  Qs and Ks are recomputed from them with the transform's own roundings, so the
+// o and f as plain [64][128] bf16 tiles (rows beyond the end of the sequence hold zeros, or in a packed batch the
+// next sequence's tokens: they are patched to the neutral f = 1, o = 0).  Qs and Ks are recomputed from them with the transform's own roundings, so the
 // operand stage does not have to be held until the outputs are done.
 template <bool kUp, bool kRagged>
 __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat16 *oraw, const __nv_bfloat16 *fraw,
@@ -133,7 +133,7 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
             const int t = t0 + j;
             fw[j] = reinterpret_cast<const unsigned short *>(fraw)[t * kD + k];
             qw[j] = reinterpret_cast<const unsigned short *>(oraw)[t * kD + k];
-            if (kRagged && t >= n_valid) fw[j] = 0x3F80u;
+            if (kRagged && t >= n_valid) { fw[j] = 0x3F80u; qw[j] = 0u; }
             fv[j] = __uint_as_float(fw[j] << 16);
         }
         tmem_wait_ld();
@@ -207,8 +207,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
               const __grid_constant__ CUtensorMap map_saved, const __grid_constant__ CUtensorMap map_o_raw,
               const __grid_constant__ CUtensorMap map_f_raw, const float *__restrict__ totals,
               const float *__restrict__ dSN, __nv_bfloat16 *__restrict__ d_o, __nv_bfloat16 *__restrict__ d_f,
-              __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N, int NC, StatusBlock *status,
-              int clear_status, const ExactArgs ex)
+              __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N_all, int NC_all, StatusBlock *status,
+              int clear_status, const ExactArgs ex, const PackedArgs pk)
 {
     // the first kernel of a call zeroes the status word; the only early report, the alignment check below, is the
     // same in every CTA, so CTA 0 repeats it after its own clear
@@ -237,6 +237,31 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int u = blockIdx.x;
+    // This CTA's sequence: rows [row0, row0 + N) of plane zu of the [planes][rows][128] tensors, NC chunks, chunk-start
+    // state c in slot slot0 + c.  Packed batches (ragged instantiations only) read theirs from the offsets array.
+    int row0 = 0, zu = u, N = N_all, NC = NC_all;
+    size_t slot0 = (size_t)u * NC_all;
+    if constexpr (kRagged) {
+        if (pk.cu != nullptr) {
+            const int b = u / pk.H;
+            zu = u - b * pk.H;
+            row0 = __ldg(pk.cu + b);
+            N = __ldg(pk.cu + b + 1) - row0;
+            NC = (N + kC - 1) / kC;
+            slot0 = (size_t)zu * pk.slots_per_head + row0 / kC + b;
+            if (row0 < 0 || N < 0 || row0 + N > N_all) {          // malformed offsets: report, touch nothing
+                if (tid == 0) report_error(status, HGRN2_ERR_INVALID_ARG, 4);
+                return;
+            }
+            if (N <= 0) {                // empty sequence: the state gradient passes through
+                if (dS0 != nullptr)
+                    for (int x = tid; x < kD * kD; x += kThreads)
+                        dS0[(size_t)u * kD * kD + x] = dSN ? dSN[(size_t)u * kD * kD + x] : 0.f;
+                return;
+            }
+        }
+    }
+    const size_t grow0 = (size_t)zu * N_all + row0;                 // first row of the sequence in the [planes * rows][128] view
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -314,7 +339,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         // ================= E1: state-gradient warps =================
         // Pm, E of every chunk come from the forward's saved totals, so this chain does not wait for T
         float pm_prev = 1.f;
-        const float *tot_u = totals + (size_t)u * NC * 2 * kD + krow;
+        const float *tot_u = totals + slot0 * 2 * kD + krow;
         float pm_c = __ldg(tot_u + (size_t)(NC - 1) * 2 * kD), ee_c = __ldg(tot_u + (size_t)(NC - 1) * 2 * kD + kD);
         PT_DECL
         for (int it = 0; it < NC; ++it) {
@@ -419,7 +444,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
             const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
-            const size_t row0 = (size_t)u * N + (size_t)c * kC;
+            const size_t crow0 = grow0 + (size_t)c * kC;
             // ---- tril(A), tril(dA) -> operand slabs, one 32 x 32 block per warp.  The
             // previous chunk's products have read the slabs: this role waited for them before its outputs.
             mbar_wait(&ctl->barX, it & 1, abort_flag);
@@ -440,8 +465,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             tc_fence_after_sync();
             float asum, esum;
             PT_STAMP(status, 14, tid == kWarpE3 * 32 && it == 16)
-            if (half) phase_main<true, kRagged>(tl, oraw, fraw, krow, d_o + row0 * kD + krow, n_valid, asum, esum);
-            else      phase_main<false, kRagged>(tl, oraw, fraw, krow, d_o + row0 * kD + krow, n_valid, asum, esum);
+            if (half) phase_main<true, kRagged>(tl, oraw, fraw, krow, d_o + crow0 * kD + krow, n_valid, asum, esum);
+            else      phase_main<false, kRagged>(tl, oraw, fraw, krow, d_o + crow0 * kD + krow, n_valid, asum, esum);
             mbar_arrive(&ctl->raw_read);
             if (half) xa[krow] = asum; else xe[krow] = esum;
             tmem_wait_st();
@@ -459,7 +484,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
             const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
-            const size_t row0 = (size_t)u * N + (size_t)c * kC;
+            const size_t crow0 = grow0 + (size_t)c * kC;
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
             PT_MARK(0)
             PT_STAMP(status, 16, tid == kWarpO * 32 && it == 16)
@@ -473,7 +498,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (8 * b + j < n_valid)
-                        d_i[(row0 + 8 * b + j) * kD + krow] = __float2bfloat16_rn(__uint_as_float(r[j]));
+                        d_i[(crow0 + 8 * b + j) * kD + krow] = __float2bfloat16_rn(__uint_as_float(r[j]));
             }
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_freeV);
@@ -494,7 +519,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (8 * b + j < n_valid)
-                        d_f[(row0 + 8 * b + j) * kD + krow] =
+                        d_f[(crow0 + 8 * b + j) * kD + krow] =
                             __float2bfloat16_rn(fmaf(K, __uint_as_float(rf[j]), __uint_as_float(uu[j])));
             }
             tc_fence_before_sync();
@@ -513,28 +538,28 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 uint8_t *st = smem + s * kStageBytes;
                 mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
                 for (int b = 0; b < 2; ++b) {
-                    tma_load_3d(st + kOffQ + b * kSS, &map_o, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + kOffK + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kOffQ + b * kSS, &map_o, &ctl->full[s], 64 * b, row0 + c * kC, zu);
+                    tma_load_3d(st + kOffK + b * kSlab, &map_f, &ctl->full[s], 64 * b, row0 + c * kC, zu);
                 }
                 for (int b = 0; b < 2; ++b)
-                    tma_load_3d(st + kOffG + b * kSS, &map_dy, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + kOffG + b * kSS, &map_dy, &ctl->full[s], 64 * b, row0 + c * kC, zu);
             };
             auto issue_v = [&](int it) {
                 const int c = NC - 1 - it;
                 mbar_arrive_expect_tx(&ctl->vfull, kTile);
-                for (int b = 0; b < 2; ++b) tma_load_3d(vbuf + b * kSlab, &map_i, &ctl->vfull, 64 * b, c * kC, u);
+                for (int b = 0; b < 2; ++b) tma_load_3d(vbuf + b * kSlab, &map_i, &ctl->vfull, 64 * b, row0 + c * kC, zu);
             };
             auto issue_raw = [&](int it) {
                 const int c = NC - 1 - it;
                 mbar_arrive_expect_tx(&ctl->rawfull, 2 * kTile);
-                tma_load_3d(smem + kOffRawO, &map_o_raw, &ctl->rawfull, 0, c * kC, u);
-                tma_load_3d(smem + kOffRawF, &map_f_raw, &ctl->rawfull, 0, c * kC, u);
+                tma_load_3d(smem + kOffRawO, &map_o_raw, &ctl->rawfull, 0, row0 + c * kC, zu);
+                tma_load_3d(smem + kOffRawF, &map_f_raw, &ctl->rawfull, 0, row0 + c * kC, zu);
             };
             auto issue_state = [&](int it) {
                 const int c = NC - 1 - it;
                 mbar_arrive_expect_tx(&ctl->sfull, kStateTile);
                 for (int b = 0; b < 2; ++b)
-                    tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, u * NC + c);
+                    tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, (int)(slot0 + c));
             };
             issue_stage(0);
             if (!kDsOnly) {
@@ -718,12 +743,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     if (!ctl->exact_flag || *abort_flag) return;
     __syncthreads();                                               // every thread has read the flag: smem is reused now
     if (tid == 0) atomicAdd(&status->exact_units, 1);
-    const size_t seq = (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
-    const int nc64 = (ex.N + kC - 1) / kC;
+    const bool packed = kRagged && pk.cu != nullptr;
+    const int n_unit = packed ? N : ex.N;                          // tokens of the whole unit
+    const size_t seq = packed ? grow0 * kD : (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
+    const size_t slot_u = packed ? slot0 : (size_t)unit * ((ex.N + kC - 1) / kC);
     alu::bwd_unit<__nv_bfloat16, __nv_bfloat16>(
         reinterpret_cast<float *>(smem), ex.o + seq, ex.f + seq, ex.i + seq, ex.dy + seq, ex.dSN ? ex.dSN + st : nullptr,
-        ex.states + (size_t)unit * nc64 * kD * kD, kC / kExactC, ex.scratch + st, ex.d_o + seq, ex.d_f + seq,
-        ex.d_i + seq, ex.dS0 ? ex.dS0 + st : nullptr, ex.N, kD, kD, kExactC, (ex.N + kExactC - 1) / kExactC);
+        ex.states + slot_u * kD * kD, kC / kExactC, ex.scratch + st, ex.d_o + seq, ex.d_f + seq,
+        ex.d_i + seq, ex.dS0 ? ex.dS0 + st : nullptr, n_unit, kD, kD, kExactC, (n_unit + kExactC - 1) / kExactC);
 }
 
 }  // namespace
@@ -784,15 +811,20 @@ static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag,
     return ex;
 }
 
+PackedArgs tc_packed_args(const SeqArgs &a);
+
+// U CTAs; ordinary layout: U planes of N rows; packed batch (pk.cu set): pk.H planes of N rows shared by the U units.
 static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly,
-                                   bool clear, const ExactArgs &ex)
+                                   bool clear, const ExactArgs &ex, const PackedArgs &pk = PackedArgs{})
 {
     CUtensorMap mo, mf, mi, mg, ms, mor, mfr;
-    if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
-        !make_map(&mg, a.dy, U, N, kC) || !make_map(&ms, a.states, U * NC, kD, kD) ||
-        !make_map_plain(&mor, a.o, U, N, kC) || !make_map_plain(&mfr, a.f, U, N, kC))
+    const uint64_t planes = pk.cu ? (uint64_t)pk.H : U;
+    const uint64_t slots = pk.cu ? (uint64_t)pk.H * pk.slots_per_head : U * NC;
+    if (!make_map(&mo, a.o, planes, N, kC) || !make_map(&mf, a.f, planes, N, kC) || !make_map(&mi, a.i, planes, N, kC) ||
+        !make_map(&mg, a.dy, planes, N, kC) || !make_map(&ms, a.states, slots, kD, kD) ||
+        !make_map_plain(&mor, a.o, planes, N, kC) || !make_map_plain(&mfr, a.f, planes, N, kC))
         return cudaErrorInvalidValue;
-    const bool ragged = N % kC != 0;
+    const bool ragged = N % kC != 0 || pk.cu != nullptr;
     if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
     auto kernel = kDsOnly ? (ragged ? tc_bwd_kernel<true, true, false> : tc_bwd_kernel<true, false, false>)
                           : (ragged ? tc_bwd_kernel<false, true, false>
@@ -803,7 +835,7 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
         mo, mf, mi, mg, ms, mor, mfr,
         a.totals, dSN, static_cast<__nv_bfloat16 *>(a.d_o),
-        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status, clear ? 1 : 0, ex);
+        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status, clear ? 1 : 0, ex, pk);
     return cudaGetLastError();
 }
 
@@ -811,6 +843,14 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
 {
     const uint64_t U = (uint64_t)a0.B * a0.H;
     SeqArgs a = a0;
+    if (a.cu) {
+        // packed batch: one CTA per (sequence, head), every CTA reads its own rows from the offsets array
+        const PackedArgs pk = tc_packed_args(a);
+        a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
+                                             (size_t)pk.H * pk.slots_per_head * kSavedStateBytes);
+        return launch_bwd_once(a, U, a.N, 0, a.dSN, a.dS0, false, a.clear_status, exact_args(a, a.N, 1, nullptr, nullptr),
+                               pk);
+    }
     a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
     const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
     cudaError_t err = cudaSuccess;

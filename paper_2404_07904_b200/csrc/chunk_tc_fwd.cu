@@ -86,8 +86,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
               const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
-              float *__restrict__ totals, float *__restrict__ seg_decay, int want_y, int want_saved, int N, int NC,
-              StatusBlock *status, int clear_status, const ExactArgs ex)
+              float *__restrict__ totals, float *__restrict__ seg_decay, int want_y, int want_saved, int N_all, int NC_all,
+              StatusBlock *status, int clear_status, const ExactArgs ex, const PackedArgs pk)
 {
     // the first kernel of a call zeroes the status word (errors are reported seconds later, after a wait ran out)
     if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -107,6 +107,30 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int u = blockIdx.x;
+    // This CTA's sequence: rows [row0, row0 + N) of plane zu of the [planes][rows][128] tensors, NC chunks, chunk-start
+    // state c in slot slot0 + c.  Packed batches (ragged instantiations only) read theirs from the offsets array.
+    int row0 = 0, zu = u, N = N_all, NC = NC_all;
+    size_t slot0 = (size_t)u * NC_all;
+    if constexpr (kRagged) {
+        if (pk.cu != nullptr) {
+            const int b = u / pk.H;
+            zu = u - b * pk.H;
+            row0 = __ldg(pk.cu + b);
+            N = __ldg(pk.cu + b + 1) - row0;
+            NC = (N + kC - 1) / kC;
+            slot0 = (size_t)zu * pk.slots_per_head + row0 / kC + b;
+            if (row0 < 0 || N < 0 || row0 + N > N_all) {          // malformed offsets: report, touch nothing
+                if (tid == 0) report_error(status, HGRN2_ERR_INVALID_ARG, 4);
+                return;
+            }
+            if (N <= 0) {                // empty sequence: the state passes through
+                if (SN != nullptr)
+                    for (int x = tid; x < kD * kD; x += kThreads)
+                        SN[(size_t)u * kD * kD + x] = S0 ? S0[(size_t)u * kD * kD + x] : 0.f;
+                return;
+            }
+        }
+    }
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -155,7 +179,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_wait(&ctl->fullqf[s], (c / kStages) & 1, abort_flag);
             PT_MARK(0)
             const int n_valid = kRagged ? N - c * kC : kC;
-            float *tg = totals ? totals + ((size_t)u * NC + c) * 2 * kD : nullptr;     // Pm, E of the chunk for the backward
+            float *tg = totals ? totals + (slot0 + c) * 2 * kD : nullptr;       // Pm, E of the chunk for the backward
             if (n_valid >= kC) {
                 transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
                                        kC, tt);
@@ -312,18 +336,18 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 // chunks ahead, or including the v tile, gave nothing)
                 if (c + 1 < NC)
                     for (int b = 0; b < 2; ++b) {
-                        tma_prefetch_3d(&map_o, 64 * b, (c + 1) * kC, u);
-                        tma_prefetch_3d(&map_f, 64 * b, (c + 1) * kC, u);
+                        tma_prefetch_3d(&map_o, 64 * b, row0 + (c + 1) * kC, zu);
+                        tma_prefetch_3d(&map_f, 64 * b, row0 + (c + 1) * kC, zu);
                     }
                 mbar_arrive_expect_tx(&ctl->fullqf[s], 2 * kTile);
                 for (int b = 0; b < 2; ++b) {
-                    tma_load_3d(st + b * kSlab, &map_o, &ctl->fullqf[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->fullqf[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + b * kSlab, &map_o, &ctl->fullqf[s], 64 * b, row0 + c * kC, zu);
+                    tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->fullqf[s], 64 * b, row0 + c * kC, zu);
                 }
                 if (c >= kStages) mbar_wait(&ctl->emptyv[s], ((c / kStages) - 1) & 1, abort_flag);
                 mbar_arrive_expect_tx(&ctl->full[s], kTile);
                 for (int b = 0; b < 2; ++b)
-                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, c * kC, u);
+                    tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, row0 + c * kC, zu);
             }
         }
     } else if (warp == kWarpMmaS) {
@@ -375,8 +399,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 // to have read 32 KB would hold those up)
                 mbar_wait(&ctl->m_done, c & 1, abort_flag);
                 if (want_saved) {
-                    tma_store_3d(&map_saved, sbuf, 0, 0, u * NC + c);
-                    tma_store_3d(&map_saved, sbuf + kStateSlab, 64, 0, u * NC + c);
+                    tma_store_3d(&map_saved, sbuf, 0, 0, (int)(slot0 + c));
+                    tma_store_3d(&map_saved, sbuf + kStateSlab, 64, 0, (int)(slot0 + c));
                     tma_store_commit();
                     tma_store_wait_read();
                 }
@@ -434,16 +458,43 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         }
     } else {
         // ================= ST: Y stores =================
-        if (lane == 0 && want_y) {
+        if constexpr (!kRagged) {
+            if (lane == 0 && want_y) {
+                for (int c = 0; c < NC; ++c) {
+                    mbar_wait(&ctl->y_staged, c & 1, abort_flag);
+                    tma_store_3d(&map_y, ybuf, 0, c * kC, u);
+                    tma_store_3d(&map_y, ybuf + kSlab, 64, c * kC, u);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                    mbar_arrive(&ctl->y_sfree);
+                }
+                tma_store_wait_all();
+            }
+        } else if (want_y) {
+            // In a packed batch the rows after a sequence's last token belong to the next sequence (a tile store
+            // would overwrite them; past the end of an ordinary tensor it simply drops them), so the partial last
+            // chunk of a packed sequence is stored row by row, by the whole warp.
             for (int c = 0; c < NC; ++c) {
                 mbar_wait(&ctl->y_staged, c & 1, abort_flag);
-                tma_store_3d(&map_y, ybuf, 0, c * kC, u);
-                tma_store_3d(&map_y, ybuf + kSlab, 64, c * kC, u);
-                tma_store_commit();
-                tma_store_wait_read();
-                mbar_arrive(&ctl->y_sfree);
+                const int n_valid = min(kC, N - c * kC);
+                if (pk.cu == nullptr || n_valid == kC) {
+                    if (lane == 0) {
+                        tma_store_3d(&map_y, ybuf, 0, row0 + c * kC, zu);
+                        tma_store_3d(&map_y, ybuf + kSlab, 64, row0 + c * kC, zu);
+                        tma_store_commit();
+                        tma_store_wait_read();
+                    }
+                } else {
+                    uint4 *dst = reinterpret_cast<uint4 *>(ex.y + ((size_t)zu * N_all + row0 + (size_t)c * kC) * kD);
+                    for (int x = lane; x < n_valid * 16; x += 32) {          // 16-byte pieces: row, slab, chunk
+                        const int r = x >> 4, h = (x >> 3) & 1, j = x & 7;
+                        dst[(size_t)r * 16 + h * 8 + j] = *reinterpret_cast<const uint4 *>(ybuf + h * kSlab + slab_chunk_off(r, j));
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->y_sfree);
             }
-            tma_store_wait_all();
+            if (lane == 0) tma_store_wait_all();
         }
     }
     tc_fence_before_sync();
@@ -483,13 +534,15 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     if (!ctl->exact_flag || *abort_flag) return;
     __syncthreads();                                               // every thread has read the flag: smem is reused now
     if (tid == 0) atomicAdd(&status->exact_units, 1);
-    const size_t seq = (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
-    const int nc64 = (ex.N + kC - 1) / kC;
+    const bool packed = kRagged && pk.cu != nullptr;
+    const int n_unit = packed ? N : ex.N;                          // tokens of the whole unit
+    const size_t seq = packed ? ((size_t)zu * N_all + row0) * kD : (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
+    const size_t slot_u = packed ? slot0 : (size_t)unit * ((ex.N + kC - 1) / kC);
     alu::fwd_unit<__nv_bfloat16, __nv_bfloat16>(
         reinterpret_cast<float *>(smem), ex.o + seq, ex.f + seq, ex.i + seq, ex.S0 ? ex.S0 + st : nullptr,
         ex.y ? ex.y + seq : nullptr, ex.SN ? ex.SN + st : nullptr,
-        ex.states ? ex.states + (size_t)unit * nc64 * kD * kD : nullptr, kC / kExactC, ex.N, kD, kD, kExactC,
-        (ex.N + kExactC - 1) / kExactC);
+        ex.states ? ex.states + slot_u * kD * kD : nullptr, kC / kExactC, n_unit, kD, kD, kExactC,
+        (n_unit + kExactC - 1) / kExactC);
 }
 
 }  // namespace
@@ -632,19 +685,23 @@ static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag,
     return ex;
 }
 
+// U CTAs; ordinary layout: U planes of N rows; packed batch (pk.cu set): pk.H planes of N rows shared by the U units.
 static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *S0, float *SN, float *seg_decay,
-                                   bool want_y, bool want_saved, bool clear, const ExactArgs &ex)
+                                   bool want_y, bool want_saved, bool clear, const ExactArgs &ex,
+                                   const PackedArgs &pk = PackedArgs{})
 {
     CUtensorMap mo, mf, mi, my, ms;
+    const uint64_t planes = pk.cu ? (uint64_t)pk.H : U;
+    const uint64_t slots = pk.cu ? (uint64_t)pk.H * pk.slots_per_head : U * NC;
     // tensor maps need a valid base even for outputs that are not wanted: point those at an input
     const void *ybase = want_y ? a.y : a.i;
     const void *sbase = want_saved ? static_cast<const void *>(a.states) : a.i;
     const uint64_t srows = want_saved ? (uint64_t)kD : (uint64_t)N;
-    const uint64_t sunits = want_saved ? U * NC : U;
-    if (!make_map(&mo, a.o, U, N, kC) || !make_map(&mf, a.f, U, N, kC) || !make_map(&mi, a.i, U, N, kC) ||
-        !make_map(&my, ybase, U, N, kC) || !make_map(&ms, sbase, sunits, srows, want_saved ? kD : kC))
+    const uint64_t sunits = want_saved ? slots : planes;
+    if (!make_map(&mo, a.o, planes, N, kC) || !make_map(&mf, a.f, planes, N, kC) || !make_map(&mi, a.i, planes, N, kC) ||
+        !make_map(&my, ybase, planes, N, kC) || !make_map(&ms, sbase, sunits, srows, want_saved ? kD : kC))
         return cudaErrorInvalidValue;
-    const bool ragged = N % kC != 0;
+    const bool ragged = N % kC != 0 || pk.cu != nullptr;
     if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
     auto kernel = seg_decay ? (ragged ? tc_fwd_kernel<true, true, false> : tc_fwd_kernel<true, false, false>)
                             : (ragged ? tc_fwd_kernel<false, true, false>
@@ -654,14 +711,37 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? a.totals : nullptr;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, seg_decay, want_y,
-                                                                   want_saved, N, NC, a.status, clear ? 1 : 0, ex);
+                                                                   want_saved, N, NC, a.status, clear ? 1 : 0, ex, pk);
     return cudaGetLastError();
+}
+
+PackedArgs tc_packed_args(const SeqArgs &a)
+{
+    PackedArgs pk;
+    pk.cu = a.cu;
+    pk.H = a.H;
+    pk.slots_per_head = a.N / kC + a.B + 1;
+    return pk;
+}
+
+size_t tc_saved_bytes_packed(const hgrn2_desc *d)
+{
+    return (size_t)d->H * ((size_t)d->N / kC + d->B + 1) * (kSavedStateBytes + kSavedTotalsBytes);
 }
 
 cudaError_t launch_tc_fwd(const SeqArgs &a0)
 {
     const uint64_t U = (uint64_t)a0.B * a0.H;
     SeqArgs a = a0;
+    if (a.cu) {
+        // packed batch: one CTA per (sequence, head), every CTA reads its own rows from the offsets array
+        const PackedArgs pk = tc_packed_args(a);
+        if (a.states)
+            a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
+                                                 (size_t)pk.H * pk.slots_per_head * kSavedStateBytes);
+        return launch_fwd_once(a, U, a.N, 0, a.S0, a.SN, nullptr, a.y != nullptr, a.states != nullptr, a.clear_status,
+                               exact_args(a, a.N, 1, nullptr, nullptr), pk);
+    }
     if (a.states) a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
     const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
     const bool want_y = a.y != nullptr, want_saved = a.states != nullptr;

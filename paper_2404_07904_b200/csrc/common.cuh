@@ -60,6 +60,7 @@ struct SeqArgs {
     float *exact_scratch = nullptr;   // tensor-core backward: [B*H][dk][dv] floats for units redone on the exact path
     float *totals = nullptr;      // tensor-core path: per-chunk decay totals inside the saved data (set by its launchers)
     bool clear_status = false;    // tensor-core path: the first kernel of the call zeroes the status word itself
+    const int *cu = nullptr;      // packed batch: device array of B + 1 row offsets (B = sequences, N = total rows per head)
     cudaStream_t stream;
 };
 
@@ -82,10 +83,20 @@ struct ExactArgs {
     float *SN = nullptr, *dS0 = nullptr;
     __nv_bfloat16 *states = nullptr;    // saved chunk states: [unit][chunk of 64][128][128] bf16
     float *scratch = nullptr;           // backward: [unit][128][128] floats
-    int N = 0;                          // tokens of a whole unit
+    int N = 0;                          // tokens of a whole unit (rows per head of a packed batch)
     int G = 1;                          // CTAs (segments) per unit in this launch
     int *unit_flag = nullptr;           // G > 1: per unit, set by any segment that left the range
     int *unit_count = nullptr;          // G > 1: per unit, segments finished so far
+};
+
+// Packed (variable-length) batches: the sequence tensors are [H][T][d] and sequence b occupies the token rows
+// [cu[b], cu[b + 1]) of every head; unit u = b * H + h.  cu == nullptr: the ordinary [B][H][N][d] layout.
+// Chunk-start states of a packed batch live in slots: sequence b owns slots floor(cu[b] / C) + b ... of its head
+// (never overlapping the next sequence's), slots_per_head = floor(T / C) + B + 1.
+struct PackedArgs {
+    const int *cu = nullptr;
+    int H = 0;
+    int slots_per_head = 0;
 };
 
 // Tensor-core path, few or left-over units: which units run whole and which are split into G segments each.

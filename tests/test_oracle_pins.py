@@ -301,3 +301,27 @@ def test_batch_head_units_are_independent():
         yb, Sb = ref.hgrn2_fwd(o[b:b + 1], f[b:b + 1], i[b:b + 1], S0[b:b + 1])
         np.testing.assert_array_equal(yb, y[b:b + 1])
         np.testing.assert_array_equal(Sb, SN[b:b + 1])
+
+
+def test_packed_batch_equals_the_same_sequences_as_an_ordinary_batch():
+    # the packed-batch wrappers add no arithmetic: B sequences of equal length laid end to end must reproduce the
+    # [B, H, N, d] result exactly, forward and backward, states included (this pins their indexing)
+    rng = np.random.default_rng(5)
+    B, H, N, dk, dv = 3, 2, 7, 4, 3
+    o = rng.standard_normal((B, H, N, dk)); f = rng.uniform(0.05, 1.0, (B, H, N, dk))
+    i = rng.standard_normal((B, H, N, dv)); dy = rng.standard_normal((B, H, N, dv))
+    S0 = rng.standard_normal((B, H, dk, dv)); dSN = rng.standard_normal((B, H, dk, dv))
+    pack = lambda x: np.ascontiguousarray(np.moveaxis(x, 0, 1).reshape(H, B * N, x.shape[-1]))
+    cu = np.arange(B + 1) * N
+    y, SN = ref.hgrn2_fwd(o, f, i, S0)
+    yp, SNp = ref.hgrn2_fwd_varlen(pack(o), pack(f), pack(i), cu, S0)
+    np.testing.assert_array_equal(yp, pack(y)); np.testing.assert_array_equal(SNp, SN)
+    g = ref.hgrn2_bwd(o, f, i, S0, dy, dSN)
+    gp = ref.hgrn2_bwd_varlen(pack(o), pack(f), pack(i), cu, S0, pack(dy), dSN)
+    for a, b in zip(g[:3], gp[:3]):
+        np.testing.assert_array_equal(b, pack(a))
+    np.testing.assert_array_equal(gp[3], g[3])
+    # an empty sequence passes its state (and its state gradient) through
+    cu2 = np.array([0, 0, N])
+    _, SN2 = ref.hgrn2_fwd_varlen(pack(o)[:, :N], pack(f)[:, :N], pack(i)[:, :N], cu2, S0[:2])
+    np.testing.assert_array_equal(SN2[0], S0[0])
