@@ -67,6 +67,13 @@ typedef enum { HGRN2_F32 = 0, HGRN2_BF16 = 1 } hgrn2_dtype;
 
 /* desc->flags */
 #define HGRN2_FLAG_FORCE_ALU 1u  /* use the fp32 CUDA-core kernels even where tensor-core ones exist */
+/* Debugging aid: every CTA of the tensor-core kernels starts as if its first device-side wait had just run out
+ * of its 2 s (the abort flag that such a wait raises is raised from the start; the timer comparison itself is
+ * not involved).  The call then takes the kernels' time-out exit - waits return at once, the load lanes stop
+ * asking for tiles, what is in flight is allowed to land, tensor memory is released, the kernel returns - and
+ * leaves HGRN2_ERR_TIMEOUT in the status word and unspecified values in its outputs (all writes stay inside
+ * the caller's buffers).  Used to test that exit. */
+#define HGRN2_FLAG_DEBUG_EXPIRE_WAITS 0x80000000u
 
 /* Problem description shared by all calls.  `chunk` is the chunk length C of the
  * chunkwise-parallel form (an implementation parameter: results agree for every

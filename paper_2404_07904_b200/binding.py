@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libhgrn2.so")
 
 HGRN2_F32, HGRN2_BF16 = 0, 1
 FLAG_FORCE_ALU = 1
+FLAG_DEBUG_EXPIRE_WAITS = 0x80000000
 
 STATUS_NAMES = {
     0: "HGRN2_OK", 1: "HGRN2_ERR_INVALID_ARG", 2: "HGRN2_ERR_UNSUPPORTED", 3: "HGRN2_ERR_ALIGNMENT",

@@ -84,6 +84,7 @@ void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream, void *ws, c
 {
     memset(&a, 0, sizeof(a));
     a.cu = cu;
+    a.start_aborted = (d->flags & HGRN2_FLAG_DEBUG_EXPIRE_WAITS) ? 1 : 0;
     // workspace layout: status block | room for re-created saved data | tensor-core path: segment scratch, then one
     // float matrix per unit for units redone on the exact path
     a.seg_scratch = nullptr;

@@ -96,10 +96,12 @@ struct Ctl {
     uint64_t acc_freeV;           // O -> M: dV^T has been read out
     uint64_t parked;              // E3 -> O: the parked values and the halves' sums are in place
     uint64_t acc_free2;           // O -> M: dQs^T and dKs_intra^T columns are free again
+    uint64_t drain;               // tcgen05.commit (MX, MY1, MY2, after their loops): every product issued has completed
+    int abort_flag;               // set by the first wait that runs out: every later wait returns at once
     uint32_t tmem_base;
-    int abort_flag;
     int o_done;                   // O -> T: final passes finished so far, counted per warp (pacing only)
     int exact_flag;               // E1: a decay of this CTA's tokens left the range of the rescaled operands
+    int l_stage, l_v, l_state, l_raw;   // L: fills asked for so far, per buffer, for the abort epilogue
 };
 static_assert(sizeof(Ctl) <= 256, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -208,7 +210,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
               const __grid_constant__ CUtensorMap map_f_raw, const float *__restrict__ totals,
               const float *__restrict__ dSN, __nv_bfloat16 *__restrict__ d_o, __nv_bfloat16 *__restrict__ d_f,
               __nv_bfloat16 *__restrict__ d_i, float *__restrict__ dS0, int N_all, int NC_all, StatusBlock *status,
-              int clear_status, const ExactArgs ex, const PackedArgs pk)
+              int clear_status, const ExactArgs ex, const PackedArgs pk, int start_aborted)
 {
     // the first kernel of a call zeroes the status word; the only early report, the alignment check below, is the
     // same in every CTA, so CTA 0 repeats it after its own clear
@@ -283,9 +285,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->acc_freeV, kOThreads);
         mbar_init(&ctl->parked, kE3Threads);
         mbar_init(&ctl->acc_free2, kOThreads);
-        ctl->abort_flag = 0;
+        mbar_init(&ctl->drain, 3);
+        ctl->abort_flag = start_aborted;
         ctl->o_done = 0;
         ctl->exact_flag = 0;
+        ctl->l_stage = ctl->l_v = ctl->l_state = ctl->l_raw = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
         tma_prefetch_desc(&map_f);
@@ -354,7 +358,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 ee_c = __ldg(tot_u + (size_t)(NC - 2 - it) * 2 * kD + kD);
             }
             if (it > 0) {
-                mbar_wait(&ctl->barX, (it - 1) & 1, abort_flag);     // dS' of the previous chunk is complete
+                mbar_wait(&ctl->barX, (it - 1) & 1, abort_flag);   // dS' of the previous chunk is complete
                 mbar_wait(&ctl->barY1, (it - 1) & 1, abort_flag);    // its dS'' copy is no longer read
                 tc_fence_after_sync();
             }
@@ -533,7 +537,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     } else if (warp == kWarpLoad) {
         // ================= L: TMA loads =================
         if (lane == 0) {
+            int n_stage = 0, n_v = 0, n_state = 0, n_raw = 0;       // fills asked for so far, per buffer
             auto issue_stage = [&](int it) {
+                n_stage = it + 1;
                 const int s = it % kStages, c = NC - 1 - it;
                 uint8_t *st = smem + s * kStageBytes;
                 mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
@@ -545,17 +551,20 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tma_load_3d(st + kOffG + b * kSS, &map_dy, &ctl->full[s], 64 * b, row0 + c * kC, zu);
             };
             auto issue_v = [&](int it) {
+                n_v = it + 1;
                 const int c = NC - 1 - it;
                 mbar_arrive_expect_tx(&ctl->vfull, kTile);
                 for (int b = 0; b < 2; ++b) tma_load_3d(vbuf + b * kSlab, &map_i, &ctl->vfull, 64 * b, row0 + c * kC, zu);
             };
             auto issue_raw = [&](int it) {
+                n_raw = it + 1;
                 const int c = NC - 1 - it;
                 mbar_arrive_expect_tx(&ctl->rawfull, 2 * kTile);
                 tma_load_3d(smem + kOffRawO, &map_o_raw, &ctl->rawfull, 0, row0 + c * kC, zu);
                 tma_load_3d(smem + kOffRawF, &map_f_raw, &ctl->rawfull, 0, row0 + c * kC, zu);
             };
             auto issue_state = [&](int it) {
+                n_state = it + 1;
                 const int c = NC - 1 - it;
                 mbar_arrive_expect_tx(&ctl->sfull, kStateTile);
                 for (int b = 0; b < 2; ++b)
@@ -570,22 +579,34 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             if (NC > 1) issue_stage(1);
             // Every buffer is refilled as soon as its last reader of chunk `it` is done; the waits below are in
             // the order in which those readers finish.
+            // A barrier must never be armed twice within one phase.  Normally a buffer's previous fill has long been
+            // consumed when its readers report; on the time-out exit those waits return at once, so before every
+            // refill the previous fill is waited for explicitly (one poll that succeeds at once in normal running).
             for (int it = 0; it + 1 < NC; ++it) {
                 if (!kDsOnly) {
                     mbar_wait(&ctl->barX, it & 1, abort_flag);       // dA = dY V^T ...
                     mbar_wait(&ctl->barY1, it & 1, abort_flag);      // ... and dKs_inter^T = dS'' V^T have read v
+                    mbar_wait_drain(&ctl->vfull, it & 1, 20000000ull);
                     issue_v(it + 1);
                     mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);   // R has read S' ...
                 }
                 mbar_wait(&ctl->barY2, it & 1, abort_flag);          // ... and so have the chunk's products;
-                if (!kDsOnly) issue_state(it + 1);
-                if (it + 2 < NC) issue_stage(it + 2);                // o, f, dy of the stage are free as well
+                if (!kDsOnly) {
+                    mbar_wait_drain(&ctl->sfull, it & 1, 20000000ull);
+                    issue_state(it + 1);
+                }
+                if (it + 2 < NC) {                                   // o, f, dy of the stage are free as well
+                    mbar_wait_drain(&ctl->full[it % kStages], (it / kStages) & 1, 20000000ull);
+                    issue_stage(it + 2);
+                }
                 PT_STAMP(status, 0, it == 14) PT_STAMP(status, 21, it == 16) PT_STAMP(status, 22, it == 15)
                 if (!kDsOnly) {
                     mbar_wait(&ctl->raw_read, it & 1, abort_flag);   // the output warps are done with raw o, f
+                    mbar_wait_drain(&ctl->rawfull, it & 1, 20000000ull);
                     issue_raw(it + 1);
                 }
             }
+            ctl->l_stage = n_stage; ctl->l_v = n_v; ctl->l_state = n_state; ctl->l_raw = n_raw;
         }
     } else if (lane == 0) {
         // ================= MX, MY1, MY2: MMA issue =================
@@ -675,7 +696,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
                 const uint64_t dqm = dqm0 + so, dfm = dfm0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
-                mbar_wait(&ctl->pd_ready, it & 1, abort_flag);        // tril(A), tril(dA); implies X and T of the chunk
+                mbar_wait(&ctl->pd_ready, it & 1, abort_flag);   // tril(A), tril(dA); implies X and T of the chunk
                 mbar_wait(&ctl->barY1, it & 1, abort_flag);           // dV^T += ... must follow dV^T = ...
                 PT_MARK(0)
                 PT_STAMP(status, 11, it == 16)
@@ -704,20 +725,23 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
             PT_DUMP(status, 21, 3, true)
         }
+        mma_commit(&ctl->drain);          // each of the three issuing lanes, after its loop
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0 && *abort_flag) {
-        report_error(status, HGRN2_ERR_TIMEOUT, 2);
-        // loads may still be in flight towards this CTA's shared memory: give them time to land
-        for (int s = 0; s < kStages; ++s) {
-            const int last = ((NC - 1 - s) / kStages) * kStages + s;
-            if (s < NC) mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
-        }
-        if (!kDsOnly) {
-            mbar_wait_drain(&ctl->sfull, (NC - 1) & 1, 20000000ull);
-            mbar_wait_drain(&ctl->vfull, (NC - 1) & 1, 20000000ull);
-            mbar_wait_drain(&ctl->rawfull, (NC - 1) & 1, 20000000ull);
+    if (tid == 0) {
+        // Nothing may be in flight when the CTA gives up its tensor and shared memory.  The three issuing lanes
+        // committed once more after their loops: that barrier completes when every product they issued has.
+        mbar_wait_drain(&ctl->drain, 0, 20000000ull);
+        if (*abort_flag) {
+            report_error(status, HGRN2_ERR_TIMEOUT, 2);
+            // tiles asked for but never consumed may still be on their way into this CTA's shared memory
+            const int ns = ctl->l_stage, nv = ctl->l_v, nst = ctl->l_state, nr = ctl->l_raw;
+            for (int s = 0; s < kStages; ++s)
+                if (ns > s) mbar_wait_drain(&ctl->full[s], ((ns - 1 - s) / kStages) & 1, 20000000ull);
+            if (nv > 0) mbar_wait_drain(&ctl->vfull, (nv - 1) & 1, 20000000ull);
+            if (nst > 0) mbar_wait_drain(&ctl->sfull, (nst - 1) & 1, 20000000ull);
+            if (nr > 0) mbar_wait_drain(&ctl->rawfull, (nr - 1) & 1, 20000000ull);
         }
     }
     __syncthreads();
@@ -835,7 +859,7 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
         mo, mf, mi, mg, ms, mor, mfr,
         a.totals, dSN, static_cast<__nv_bfloat16 *>(a.d_o),
-        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status, clear ? 1 : 0, ex, pk);
+        static_cast<__nv_bfloat16 *>(a.d_f), static_cast<__nv_bfloat16 *>(a.d_i), dS0, N, NC, a.status, clear ? 1 : 0, ex, pk, a.start_aborted);
     return cudaGetLastError();
 }
 

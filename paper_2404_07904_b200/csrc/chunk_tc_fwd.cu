@@ -46,7 +46,7 @@ constexpr uint32_t kOffY = kOffP + 2 * kSlab;                     // Y staging t
 constexpr uint32_t kOffPm = kOffY + kTile;                        // float pm[4][128]
 constexpr uint32_t kOffE = kOffPm + 4 * 128 * 4;                  // float ee[4][128]
 constexpr uint32_t kOffCtl = kOffE + 4 * 128 * 4;
-constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024;             // + alignment slack
+constexpr uint32_t kSmemBytes = kOffCtl + 320 + 1024;             // + alignment slack
 
 constexpr uint32_t kColS = 0, kColY = 128, kColA = 384;
 
@@ -66,11 +66,13 @@ struct Ctl {
     uint64_t y_tfree[2];         // E2 -> MY: the Y accumulator has been read out
     uint64_t y_staged;           // E2 -> ST
     uint64_t y_sfree;            // ST -> E2: the staging tile may be overwritten
+    uint64_t drain;              // tcgen05.commit (MS and MY, after their loops): every product issued has completed
+    int abort_flag;              // set by the first wait that runs out: every later wait returns at once
     uint32_t tmem_base;
-    int abort_flag;
     int exact_flag;              // E1: a decay of this CTA's tokens left the range of the rescaled operands
+    int l_qf, l_v;               // L: chunks whose o, f tiles (i tile) have been asked for, for the abort epilogue
 };
-static_assert(sizeof(Ctl) <= 256, "control block");
+static_assert(sizeof(Ctl) <= 320, "control block");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
 constexpr int kExactC = 32;      // chunk length of the exact fp32 routines at d = 128 (their shared-memory budget)
@@ -87,7 +89,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
               const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
               float *__restrict__ totals, float *__restrict__ seg_decay, int want_y, int want_saved, int N_all, int NC_all,
-              StatusBlock *status, int clear_status, const ExactArgs ex, const PackedArgs pk)
+              StatusBlock *status, int clear_status, const ExactArgs ex, const PackedArgs pk,
+              int start_aborted)
 {
     // the first kernel of a call zeroes the status word (errors are reported seconds later, after a wait ran out)
     if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -152,8 +155,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         }
         mbar_init(&ctl->y_staged, kE2Threads);
         mbar_init(&ctl->y_sfree, 1);
-        ctl->abort_flag = 0;
+        mbar_init(&ctl->drain, 2);
+        ctl->abort_flag = start_aborted;
         ctl->exact_flag = 0;
+        ctl->l_qf = 0;
+        ctl->l_v = 0;
         fence_barrier_init();
         tma_prefetch_desc(&map_o);
         tma_prefetch_desc(&map_f);
@@ -324,13 +330,21 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     } else if (warp == kWarpLoad) {
         // ================= L: TMA loads =================
         if (lane == 0) {
+            int n_qf = 0, n_v = 0;                                   // chunks whose tiles have been asked for
             for (int c = 0; c < NC; ++c) {
                 const int s = c % kStages;
                 uint8_t *st = smem + s * kStageBytes;
                 // o and f have barriers of their own in both directions: the transform, which paces the kernel,
                 // needs only them, and their tiles are free as soon as Y = Qs S' of the chunk three back is done,
                 // well before its last product Y += P V has read V
-                if (c >= kStages) mbar_wait(&ctl->emptyqf[s], ((c / kStages) - 1) & 1, abort_flag);
+                // A barrier must never be armed twice within one phase.  Normally the stage's previous fill has long
+                // been consumed when its empty barrier completes; on the time-out exit that wait returns at once, so
+                // the previous fill is waited for explicitly (one poll that succeeds at once in normal running;
+                // stopping this lane on the wait's return value instead cost 8 %).
+                if (c >= kStages) {
+                    mbar_wait(&ctl->emptyqf[s], ((c / kStages) - 1) & 1, abort_flag);
+                    mbar_wait_drain(&ctl->fullqf[s], ((c / kStages) - 1) & 1, 20000000ull);
+                }
                 // the next chunk's o, f tiles are asked into L2 now: their load can be issued only when their stage
                 // frees, one chunk from now, and then finds them there (measured on the fwd + bwd step: -1 %; two
                 // chunks ahead, or including the v tile, gave nothing)
@@ -344,11 +358,18 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tma_load_3d(st + b * kSlab, &map_o, &ctl->fullqf[s], 64 * b, row0 + c * kC, zu);
                     tma_load_3d(st + kTile + b * kSlab, &map_f, &ctl->fullqf[s], 64 * b, row0 + c * kC, zu);
                 }
-                if (c >= kStages) mbar_wait(&ctl->emptyv[s], ((c / kStages) - 1) & 1, abort_flag);
+                n_qf = c + 1;
+                if (c >= kStages) {
+                    mbar_wait(&ctl->emptyv[s], ((c / kStages) - 1) & 1, abort_flag);
+                    mbar_wait_drain(&ctl->full[s], ((c / kStages) - 1) & 1, 20000000ull);
+                }
                 mbar_arrive_expect_tx(&ctl->full[s], kTile);
                 for (int b = 0; b < 2; ++b)
                     tma_load_3d(st + 2 * kTile + b * kSlab, &map_i, &ctl->full[s], 64 * b, row0 + c * kC, zu);
+                n_v = c + 1;
             }
+            ctl->l_qf = n_qf;
+            ctl->l_v = n_v;
         }
     } else if (warp == kWarpMmaS) {
         // ================= MS: state update =================
@@ -408,6 +429,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
             PT_DUMP(status, 12, 3, true)
             if (want_saved) tma_store_wait_all();
+            mma_commit(&ctl->drain);
         }
     } else if (warp == kWarpMmaY) {
         // ================= MY: outputs (+ saved-state stores) =================
@@ -455,6 +477,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 PT_MARK(4)
             }
             PT_DUMP(status, 15, 5, true)
+            mma_commit(&ctl->drain);
         }
     } else {
         // ================= ST: Y stores =================
@@ -499,14 +522,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0 && *abort_flag) {
-        report_error(status, HGRN2_ERR_TIMEOUT, 1);
-        // a load may still be in flight towards this CTA's shared memory: give it time to land
-        for (int s = 0; s < kStages; ++s) {
-            const int last = ((NC - 1 - s) / kStages) * kStages + s;     // last chunk that used stage s
-            if (s < NC) {
-                mbar_wait_drain(&ctl->fullqf[s], (last / kStages) & 1, 20000000ull);
-                mbar_wait_drain(&ctl->full[s], (last / kStages) & 1, 20000000ull);
+    if (tid == 0) {
+        // Nothing may be in flight when the CTA gives up its tensor and shared memory.  The two issuing lanes
+        // committed once more after their loops: that barrier completes when every product they issued has.
+        mbar_wait_drain(&ctl->drain, 0, 20000000ull);
+        if (*abort_flag) {
+            report_error(status, HGRN2_ERR_TIMEOUT, 1);
+            // tiles asked for but never consumed may still be on their way into this CTA's shared memory
+            for (int s = 0; s < kStages; ++s) {
+                const int nq = ctl->l_qf, nv = ctl->l_v;
+                if (nq > s) mbar_wait_drain(&ctl->fullqf[s], (((nq - 1 - s) / kStages)) & 1, 20000000ull);
+                if (nv > s) mbar_wait_drain(&ctl->full[s], (((nv - 1 - s) / kStages)) & 1, 20000000ull);
             }
         }
     }
@@ -711,7 +737,8 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? a.totals : nullptr;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, seg_decay, want_y,
-                                                                   want_saved, N, NC, a.status, clear ? 1 : 0, ex, pk);
+                                                                   want_saved, N, NC, a.status, clear ? 1 : 0, ex, pk,
+                                                                   a.start_aborted);
     return cudaGetLastError();
 }
 

@@ -60,6 +60,7 @@ struct SeqArgs {
     float *exact_scratch = nullptr;   // tensor-core backward: [B*H][dk][dv] floats for units redone on the exact path
     float *totals = nullptr;      // tensor-core path: per-chunk decay totals inside the saved data (set by its launchers)
     bool clear_status = false;    // tensor-core path: the first kernel of the call zeroes the status word itself
+    int start_aborted = 0;        // tensor-core path, debugging: every CTA starts as if its first wait had run out
     const int *cu = nullptr;      // packed batch: device array of B + 1 row offsets (B = sequences, N = total rows per head)
     cudaStream_t stream;
 };

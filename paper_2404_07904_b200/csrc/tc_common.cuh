@@ -70,7 +70,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 
 // Waits for the phase with the given parity to complete, for at most kWaitLimitNs.  `abort_flag`
 // lives in shared memory: once any wait of the CTA has run out, every later wait returns at once,
-// so a broken pipeline drains in bounded time instead of hanging the GPU.  Returns false on give-up.
+// so a broken pipeline drains in bounded time instead of hanging the GPU.  Returns false on give-up (only the
+// load lanes look at that: they must not re-arm a barrier whose previous fill was never consumed; every other
+// role just runs through its remaining chunks on stale data, which is harmless and bounded).
+// Two measured facts shape the slow path: what it does between entry and its next poll is on the critical path
+// of every hand-off (reading the limit from shared memory there instead of using a constant cost 6 %), and
+// testing the return value at the wait sites of the hot roles cost 8 %.
 // The first poll is inlined; the loop itself is one shared out-of-line routine (the kernels wait in dozens
 // of places, and their combined instruction footprint matters more than a call).
 static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, volatile int *abort_flag);

@@ -313,3 +313,40 @@ def test_config5_decode_all_512_steps():
     for (b, h) in units:
         assert G.rel_err(Sh[b:b + 1, h:h + 1], S_ref[(b, h)]) <= 1e-5
     print("config 5 worst y error over 512 steps", worst)
+
+
+# ---------------------------------------------------------------- the kernels' time-out exit
+def test_expired_waits_end_in_a_timeout_status_and_leave_the_context_usable():
+    # With HGRN2_FLAG_DEBUG_EXPIRE_WAITS every device-side wait that has to wait gives up at once, so the product
+    # kernels (unmodified) take their time-out exit: they must return, report HGRN2_ERR_TIMEOUT, write only
+    # inside the caller's buffers, and the next ordinary call on the same workspace must be correct again.
+    w = W.scaled(W.CONFIGS["lm_2048"], B=1, H=1, N=128, has_S0=True, has_dSN=True, seed=91)
+    inp = W.make_inputs(w)
+    t = G.to_dev(inp, "bf16")
+    bufs = {}
+    outs = {}
+    for name, shape, dt in (("y", (1, 1, 128, 128), torch.bfloat16), ("SN", (1, 1, 128, 128), torch.float32),
+                            ("d_o", (1, 1, 128, 128), torch.bfloat16), ("d_f", (1, 1, 128, 128), torch.bfloat16),
+                            ("d_i", (1, 1, 128, 128), torch.bfloat16), ("dS0", (1, 1, 128, 128), torch.float32)):
+        bufs[name], outs[name] = G.canary(shape, dt)
+    y, SN, saved, ws, _ = binding.hgrn2_fwd(t["o"], t["f"], t["i"], t["S0"], y=outs["y"], SN=outs["SN"],
+                                            flags=binding.FLAG_DEBUG_EXPIRE_WAITS)
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws) == 6, "forward: HGRN2_ERR_TIMEOUT expected"
+    # an ordinary forward fills `saved` properly for the backward under test
+    binding.hgrn2_fwd(t["o"], t["f"], t["i"], t["S0"], y=outs["y"], SN=outs["SN"], saved=saved, ws=ws)
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws) == 0
+    binding.hgrn2_bwd(t["o"], t["f"], t["i"], t["S0"], t["dy"], t["dSN"], saved, d_o=outs["d_o"], d_f=outs["d_f"],
+                      d_i=outs["d_i"], dS0=outs["dS0"], ws=ws, flags=binding.FLAG_DEBUG_EXPIRE_WAITS)
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws) == 6, "backward: HGRN2_ERR_TIMEOUT expected"
+    for name, b in bufs.items():
+        assert G.canary_ok(b), f"out-of-bounds write next to {name}"
+    # the same workspace and buffers, no flag: status clean again and every output right
+    binding.hgrn2_bwd(t["o"], t["f"], t["i"], t["S0"], t["dy"], t["dSN"], saved, d_o=outs["d_o"], d_f=outs["d_f"],
+                      d_i=outs["d_i"], dS0=outs["dS0"], ws=ws)
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws) == 0
+    got = {k: v.float().cpu().numpy() for k, v in outs.items()}
+    G.assert_close(got, G.oracle_fwd_bwd(inp), 2e-2, "after the timed-out calls")
