@@ -43,8 +43,10 @@ NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu captures summarised under
 # profiles/ (same workloads as timed here: lm_2048 and the full decode batch); nothing here measures traffic.
 # None = the kernel has changed since its counters were taken.
-NCU_TRAFFIC_BYTES = {"fwd": None, "bwd": None, "step": 271.60e6 + 212.48e6}
-NCU_TRAFFIC_SOURCE = {"fwd": None, "bwd": None, "step": "profiles/step_kernel_decode.md"}
+NCU_TRAFFIC_BYTES = {"fwd": 201.40e6 + 154.28e6, "bwd": 406.94e6 + 171.45e6, "step": 271.60e6 + 212.48e6}
+NCU_TRAFFIC_SOURCE = {"fwd": "profiles/tc_fwd_bwd_lm2048.md (captured 2026-11-28, after the time-out exit change)",
+                      "bwd": "profiles/tc_fwd_bwd_lm2048.md (captured 2026-11-28, after the time-out exit change)",
+                      "step": "profiles/step_kernel_decode.md"}
 
 
 def load_peaks():
