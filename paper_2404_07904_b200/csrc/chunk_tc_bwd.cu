@@ -197,12 +197,10 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
     esum = H;
 }
 
-// kDsOnly: run the state-gradient chain alone (dS_0 from dS_N and dy; no other output), for sequences split
-// into segments.  A template parameter, not a flag: the full kernel is sensitive to its instruction footprint.
 // kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens); when false,
 // every per-row validity test below folds away.
 // kMultiCta: a unit runs as several CTAs (segments) of this launch (see the forward kernel).
-template <bool kDsOnly, bool kRagged, bool kMultiCta>
+template <bool kRagged, bool kMultiCta>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
@@ -320,7 +318,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             // chunk it - 2 is over.  Its tiles are there well before, but run earlier it shares the issue slots
             // with the output phase and that final pass, the longest stretch of the per-chunk loop (measured:
             // starting as soon as the tiles land costs 2 %, starting even earlier, via an L2 prefetch, 15 %).
-            if (!kDsOnly && it >= 2) {
+            if (it >= 2) {
                 if (lane == 0) count_wait(&ctl->o_done, kOWarps * (it - 1), abort_flag);   // one poller per warp
                 __syncwarp();
             }
@@ -398,7 +396,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_arrive(&ctl->m_done);
             PT_MARK(2)
             PT_STAMP(status, 6, tid == kWarpE1 * 32 && it == 16)
-            if (kDsOnly) continue;                                   // state-gradient chain only
 
             // ---- R_k = sum_v dS''[k,v] S'[k,v] from the two bf16 copies
             mbar_wait(&ctl->sfull, it & 1, abort_flag);
@@ -445,7 +442,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         const int half = (warp - kWarpE3) >> 2;                      // half of the chunk: local times [32 * half, +32)
         const uint32_t tl = tmem + lane_base;
         PT_DECL
-        for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
+        for (int it = 0; it < NC; ++it) {
             const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
             const size_t crow0 = grow0 + (size_t)c * kC;
@@ -485,7 +482,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         // ================= O: d_i, and d_f completed from the parked values =================
         const uint32_t tl = tmem + lane_base;
         PT_DECL
-        for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
+        for (int it = 0; it < NC; ++it) {
             const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
             const size_t crow0 = grow0 + (size_t)c * kC;
@@ -571,11 +568,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tma_load_3d(sbuf + b * kStateSlab, &map_saved, &ctl->sfull, 64 * b, 0, (int)(slot0 + c));
             };
             issue_stage(0);
-            if (!kDsOnly) {
-                issue_v(0);
-                issue_state(0);
-                issue_raw(0);
-            }
+            issue_v(0);
+            issue_state(0);
+            issue_raw(0);
             if (NC > 1) issue_stage(1);
             // Every buffer is refilled as soon as its last reader of chunk `it` is done; the waits below are in
             // the order in which those readers finish.
@@ -583,28 +578,22 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             // consumed when its readers report; on the time-out exit those waits return at once, so before every
             // refill the previous fill is waited for explicitly (one poll that succeeds at once in normal running).
             for (int it = 0; it + 1 < NC; ++it) {
-                if (!kDsOnly) {
-                    mbar_wait(&ctl->barX, it & 1, abort_flag);       // dA = dY V^T ...
-                    mbar_wait(&ctl->barY1, it & 1, abort_flag);      // ... and dKs_inter^T = dS'' V^T have read v
-                    mbar_wait_drain(&ctl->vfull, it & 1, 20000000ull);
-                    issue_v(it + 1);
-                    mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);   // R has read S' ...
-                }
+                mbar_wait(&ctl->barX, it & 1, abort_flag);           // dA = dY V^T ...
+                mbar_wait(&ctl->barY1, it & 1, abort_flag);          // ... and dKs_inter^T = dS'' V^T have read v
+                mbar_wait_drain(&ctl->vfull, it & 1, 20000000ull);
+                issue_v(it + 1);
+                mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);   // R has read S' ...
                 mbar_wait(&ctl->barY2, it & 1, abort_flag);          // ... and so have the chunk's products;
-                if (!kDsOnly) {
-                    mbar_wait_drain(&ctl->sfull, it & 1, 20000000ull);
-                    issue_state(it + 1);
-                }
+                mbar_wait_drain(&ctl->sfull, it & 1, 20000000ull);
+                issue_state(it + 1);
                 if (it + 2 < NC) {                                   // o, f, dy of the stage are free as well
                     mbar_wait_drain(&ctl->full[it % kStages], (it / kStages) & 1, 20000000ull);
                     issue_stage(it + 2);
                 }
                 PT_STAMP(status, 0, it == 14) PT_STAMP(status, 21, it == 16) PT_STAMP(status, 22, it == 15)
-                if (!kDsOnly) {
-                    mbar_wait(&ctl->raw_read, it & 1, abort_flag);   // the output warps are done with raw o, f
-                    mbar_wait_drain(&ctl->rawfull, it & 1, 20000000ull);
-                    issue_raw(it + 1);
-                }
+                mbar_wait(&ctl->raw_read, it & 1, abort_flag);       // the output warps are done with raw o, f
+                mbar_wait_drain(&ctl->rawfull, it & 1, 20000000ull);
+                issue_raw(it + 1);
             }
             ctl->l_stage = n_stage; ctl->l_v = n_v; ctl->l_state = n_state; ctl->l_raw = n_raw;
         }
@@ -637,19 +626,15 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
                 PT_MARK(0)
                 mbar_wait(&ctl->m_done, it & 1, abort_flag);          // dS'' in TMEM
-                if (it > 0 && !kDsOnly) mbar_wait(&ctl->pd_ready, (it - 1) & 1, abort_flag);   // A, dA of the previous chunk read out
-                if (!kDsOnly) mbar_wait(&ctl->vfull, it & 1, abort_flag);
+                if (it > 0) mbar_wait(&ctl->pd_ready, (it - 1) & 1, abort_flag);   // A, dA of the previous chunk read out
+                mbar_wait(&ctl->vfull, it & 1, abort_flag);
                 PT_MARK(1)
                 PT_STAMP(status, 3, it == 16)
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dS' = dS'' + Qs^T dY
                     mma_bf16_ss(tmem + kColDS, dqm + (uint64_t)(kk * 128), dgm + (uint64_t)(kk * 128), idDS, 1);
-                if constexpr (kDsOnly) {                    // state-gradient chain only: stand in for the other groups
-                    mma_commit(&ctl->barX);
-                    mma_commit(&ctl->barY1);
-                    mma_commit(&ctl->barY2);
-                } else {
+                {
                     // (Qs; dY) as one 128-row operand: (Qs; dY) Ks^T has A in lanes 0..63 and (Qs; dY) V^T has dA
                     // in lanes 64..127 (the other halves are not used), so every lane carries a row to mask
 #pragma unroll
@@ -665,7 +650,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
             PT_DUMP(status, 15, 3, true)
         } else if (warp == kWarpMmaY1) {
-            for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
+            for (int it = 0; it < NC; ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
                 const uint64_t dfk = dfk0 + so;
@@ -692,7 +677,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
             PT_DUMP(status, 18, 3, true)
         } else {
-            for (int it = 0; it < (kDsOnly ? 0 : NC); ++it) {
+            for (int it = 0; it < NC; ++it) {
                 const int s = it % kStages;
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
                 const uint64_t dqm = dqm0 + so, dfm = dfm0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
@@ -780,16 +765,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 }  // namespace
 
 // ---- sequences split into segments (see chunk_tc_fwd.cu) ----------------------------------------------
-// Total decay of every segment from the forward's saved per-chunk totals: lam[ur][k] = prod_c Pm E.
-__global__ void seg_decay_kernel(const float *__restrict__ totals, float *__restrict__ lam, int chunks_per_seg)
-{
-    const size_t ur = blockIdx.x;
-    const int k = threadIdx.x;
-    const float *t = totals + ur * chunks_per_seg * 2 * kD + k;
-    float p = 1.f;
-    for (int c = 0; c < chunks_per_seg; ++c) p *= t[(size_t)c * 2 * kD] * t[(size_t)c * 2 * kD + kD];
-    lam[ur * kD + k] = p;
-}
 // Chains the segments in reverse: dS_end[r] = gradient w.r.t. the state at the end of segment r.
 __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const float *__restrict__ G_loc,
                                        const float *__restrict__ lam, float *__restrict__ dS_end,
@@ -838,7 +813,7 @@ static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag,
 PackedArgs tc_packed_args(const SeqArgs &a);
 
 // U CTAs; ordinary layout: U planes of N rows; packed batch (pk.cu set): pk.H planes of N rows shared by the U units.
-static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0, bool kDsOnly,
+static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0,
                                    bool clear, const ExactArgs &ex, const PackedArgs &pk = PackedArgs{})
 {
     CUtensorMap mo, mf, mi, mg, ms, mor, mfr;
@@ -850,10 +825,8 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
         return cudaErrorInvalidValue;
     const bool ragged = N % kC != 0 || pk.cu != nullptr;
     if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
-    auto kernel = kDsOnly ? (ragged ? tc_bwd_kernel<true, true, false> : tc_bwd_kernel<true, false, false>)
-                          : (ragged ? tc_bwd_kernel<false, true, false>
-                                    : (ex.o != nullptr && ex.G > 1 ? tc_bwd_kernel<false, false, true>
-                                                                    : tc_bwd_kernel<false, false, false>));
+    auto kernel = ragged ? tc_bwd_kernel<true, false>
+                         : (ex.o != nullptr && ex.G > 1 ? tc_bwd_kernel<false, true> : tc_bwd_kernel<false, false>);
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
@@ -872,7 +845,7 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         const PackedArgs pk = tc_packed_args(a);
         a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
                                              (size_t)pk.H * pk.slots_per_head * kSavedStateBytes);
-        return launch_bwd_once(a, U, a.N, 0, a.dSN, a.dS0, false, a.clear_status, exact_args(a, a.N, 1, nullptr, nullptr),
+        return launch_bwd_once(a, U, a.N, 0, a.dSN, a.dS0, a.clear_status, exact_args(a, a.N, 1, nullptr, nullptr),
                                pk);
     }
     a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
@@ -881,7 +854,7 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
     bool clear = a.clear_status;                                  // for the first kernel launched only
     if (plan.main_units) {
         const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
-        err = launch_bwd_once(m, plan.main_units, a.N, a.NC, m.dSN, m.dS0, false, clear,
+        err = launch_bwd_once(m, plan.main_units, a.N, a.NC, m.dSN, m.dS0, clear,
                               exact_args(m, a.N, 1, nullptr, nullptr));
         if (err != cudaSuccess) return err;
         clear = false;
@@ -895,14 +868,13 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         float *dS_end = G_loc + Ut * G * kD * kD;
         float *lam = dS_end + Ut * G * kD * kD;
         int *unit_flag = reinterpret_cast<int *>(lam + Ut * G * kD), *unit_count = unit_flag + Ut;
-        // state-gradient chains only; no exact path of their own: the full pass below meets the same decays
-        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, G_loc, true, clear, ExactArgs{});
+        // state-gradient contributions of the segments (chunk_tc_state.cu): they hold for every f
+        err = launch_tc_state_bwd(t.o, t.f, t.dy, Ut * G, a.N / G, G_loc, lam, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
-        seg_decay_kernel<<<(unsigned)(Ut * G), kD, 0, a.stream>>>(t.totals, lam, a.NC / G);
         seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G,
                                                                                     unit_flag, unit_count, (int)Ut);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false, false,
+        err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false,
                               exact_args(t, a.N, G, unit_flag, unit_count));
     }
     return err;

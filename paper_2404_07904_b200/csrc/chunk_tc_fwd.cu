@@ -78,17 +78,15 @@ static_assert(kSmemBytes <= 232448, "shared memory budget");
 constexpr int kExactC = 32;      // chunk length of the exact fp32 routines at d = 128 (their shared-memory budget)
 static_assert(alu::fwd_smem_floats(kD, kD, kExactC) * sizeof(float) <= kSmemBytes - 1024, "exact path fits the CTA's shared memory");
 
-// kSegDecay: also write the product of f over the whole (sub)sequence per key dimension to seg_decay (used when
-// sequences are split into segments).  A template parameter: the kernel is sensitive to its instruction footprint.
 // kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens).
 // kMultiCta: a unit runs as several CTAs (segments) of this launch; the bookkeeping that lets the last of them
 // take the unit's exact path is compiled in only then (its mere presence costs the one-CTA-per-unit launch 3 %).
-template <bool kSegDecay, bool kRagged, bool kMultiCta>
+template <bool kRagged, bool kMultiCta>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
               const __grid_constant__ CUtensorMap map_saved, const float *__restrict__ S0, float *__restrict__ SN,
-              float *__restrict__ totals, float *__restrict__ seg_decay, int want_y, int want_saved, int N_all, int NC_all,
+              float *__restrict__ totals, int want_y, int want_saved, int N_all, int NC_all,
               StatusBlock *status, int clear_status, const ExactArgs ex, const PackedArgs pk,
               int start_aborted)
 {
@@ -204,7 +202,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         const int krow = 32 * sub + lane;
         const int v0 = 64 * half;
         float e_prev = 1.f;
-        float lam = 1.f;                                             // product of f over the whole sequence, this key dim
         PT_DECL
         for (int c = 0; c < NC; ++c) {
             // S' = (E_prev Pm) S'' (S'' = the accumulator, or S0 for the first chunk) back into TMEM
@@ -215,7 +212,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             e_prev = ee[(c & 3) * 128 + krow];
             // a total on the floor: the decay across that half chunk is more than the rescaled operands can carry
             if (fminf(pm_c, e_prev) <= kProdFloor) ctl->exact_flag = 1;
-            if (kSegDecay) lam *= pm_c * e_prev;
             uint32_t r[64];
             if (c == 0) {
                 if (S0) {
@@ -261,7 +257,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         }
         PT_DUMP(status, 2, 5, tid == kWarpE1 * 32)
 
-        if (kSegDecay && half == 0) seg_decay[(size_t)u * kD + krow] = lam;
 
         // S_N = Diag(E_last) S''
         mbar_wait(&ctl->barS, (NC - 1) & 1, abort_flag);
@@ -589,8 +584,8 @@ size_t tc_saved_bytes(const hgrn2_desc *d, int C)
 // ---- sequences split into segments ----------------------------------------------------------------------
 // One CTA per unit leaves most SMs idle when there are few units (a 16K-token batch of two sequences has
 // 32).  The recurrence is linear in the state, so a sequence can be cut into G segments that run as separate
-// CTAs: (1) every segment runs state-only from a zero state, giving its local end state and its total decay
-// Lambda = prod f; (2) a small kernel chains them, S_start[r+1] = Diag(Lambda[r]) S_start[r] + S_local[r];
+// CTAs: (1) every segment runs state-only from a zero state (chunk_tc_state.cu), giving its local end state and
+// its total decay Lambda = prod f; (2) a small kernel chains them, S_start[r+1] = Diag(Lambda[r]) S_start[r] + S_local[r];
 // (3) every segment runs in full from its S_start.  Token (r, t) of unit u is token t of "unit" u * G + r of a
 // [U * G][N / G][128] view of the same memory, so the kernel itself does not know about segments.
 __global__ void seg_combine_kernel(const float *__restrict__ S0, const float *__restrict__ S_loc,
@@ -712,7 +707,7 @@ static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag,
 }
 
 // U CTAs; ordinary layout: U planes of N rows; packed batch (pk.cu set): pk.H planes of N rows shared by the U units.
-static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *S0, float *SN, float *seg_decay,
+static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *S0, float *SN,
                                    bool want_y, bool want_saved, bool clear, const ExactArgs &ex,
                                    const PackedArgs &pk = PackedArgs{})
 {
@@ -729,14 +724,12 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
         return cudaErrorInvalidValue;
     const bool ragged = N % kC != 0 || pk.cu != nullptr;
     if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
-    auto kernel = seg_decay ? (ragged ? tc_fwd_kernel<true, true, false> : tc_fwd_kernel<true, false, false>)
-                            : (ragged ? tc_fwd_kernel<false, true, false>
-                                      : (ex.o != nullptr && ex.G > 1 ? tc_fwd_kernel<false, false, true>
-                                                                      : tc_fwd_kernel<false, false, false>));
+    auto kernel = ragged ? tc_fwd_kernel<true, false>
+                         : (ex.o != nullptr && ex.G > 1 ? tc_fwd_kernel<false, true> : tc_fwd_kernel<false, false>);
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? a.totals : nullptr;
-    kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, seg_decay, want_y,
+    kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, want_y,
                                                                    want_saved, N, NC, a.status, clear ? 1 : 0, ex, pk,
                                                                    a.start_aborted);
     return cudaGetLastError();
@@ -766,7 +759,7 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         if (a.states)
             a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
                                                  (size_t)pk.H * pk.slots_per_head * kSavedStateBytes);
-        return launch_fwd_once(a, U, a.N, 0, a.S0, a.SN, nullptr, a.y != nullptr, a.states != nullptr, a.clear_status,
+        return launch_fwd_once(a, U, a.N, 0, a.S0, a.SN, a.y != nullptr, a.states != nullptr, a.clear_status,
                                exact_args(a, a.N, 1, nullptr, nullptr), pk);
     }
     if (a.states) a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
@@ -776,7 +769,7 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
     bool clear = a.clear_status;                                  // for the first kernel launched only
     if (plan.main_units) {
         const SeqArgs m = tc_slice_units(a, 0, plan.main_units);
-        err = launch_fwd_once(m, plan.main_units, a.N, a.NC, m.S0, m.SN, nullptr, want_y, want_saved, clear,
+        err = launch_fwd_once(m, plan.main_units, a.N, a.NC, m.S0, m.SN, want_y, want_saved, clear,
                               exact_args(m, a.N, 1, nullptr, nullptr));
         if (err != cudaSuccess) return err;
         clear = false;
@@ -790,13 +783,13 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         float *S_start = S_loc + Ut * G * kD * kD;
         float *lam = S_start + Ut * G * kD * kD;
         int *unit_flag = reinterpret_cast<int *>(lam + Ut * G * kD), *unit_count = unit_flag + Ut;
-        // the state-only pass needs no exact path of its own: the full pass below meets the same decays
-        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, nullptr, S_loc, lam, false, false, clear, ExactArgs{});
+        // the state-only pass (chunk_tc_state.cu) holds for every f: it needs no exact path of its own
+        err = launch_tc_state_fwd(t.f, t.i, Ut * G, a.N / G, S_loc, lam, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
         seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G,
                                                                                 unit_flag, unit_count, (int)Ut);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, nullptr, want_y, want_saved, false,
+        err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, want_y, want_saved, false,
                               exact_args(t, a.N, G, unit_flag, unit_count));
     }
     return err;

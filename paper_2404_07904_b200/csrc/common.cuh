@@ -109,6 +109,10 @@ struct SegPlan {
 SegPlan     tc_seg_plan(uint64_t U, int N, int NC);
 SeqArgs     tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n);
 
+cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam,
+                                StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream);
+cudaError_t launch_tc_state_bwd(const void *o, const void *f, const void *dy, uint64_t U, int N, float *G_loc,
+                                float *lam, StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream);
 cudaError_t launch_step(const StepArgs &a);
 bool        step_multi_supported(int dk, int dv);
 cudaError_t launch_step_multi(const StepArgs &a);
