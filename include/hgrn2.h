@@ -152,6 +152,39 @@ hgrn2_status hgrn2_bwd_varlen(const hgrn2_desc *desc, const void *o, const void 
                               const float *dSN, const void *saved, void *d_o, void *d_f, void *d_i,
                               float *dS0, void *ws, void *cuda_stream);
 
+/* The layer's gate activations fused in front of the recurrence.  Eq. 1 forms the gates from dense projections,
+ * o = sigmoid(.), i = SiLU(.), and Eq. 2 gives the forget gate a per-channel lower bound beta in [0, 1):
+ *
+ *     o = sigmoid(zo),      f = beta + (1 - beta) * sigmoid(zf),      i = silu(zi)
+ *
+ * These calls take the pre-activations and return y (forward) and the gradients with respect to the
+ * pre-activations and to beta (backward), so the three gate tensors and their three gradients never make a round
+ * trip through a framework's element-wise kernels, and f is never rounded to the I/O type (a bf16 f near 1 would
+ * distort every decay product by 2^-9 / (1 - f)).
+ *   zo, zf [B][H][N][dk], zi [B][H][N][dv]   in  (desc->io), device memory, 16-byte aligned
+ *   beta   [H][dk] float32                   in, device memory, 16-byte aligned, values in [0, 1)
+ *   S0, y, SN, dy, dSN, dS0                  as in hgrn2_fwd / hgrn2_bwd
+ *   d_zo, d_zf [B][H][N][dk], d_zi [B][H][N][dv] out (desc->io)
+ *   d_beta [H][dk] float32                   out, NULL = not wanted (summed over batch and time in a fixed order)
+ *   saved  hgrn2_saved_bytes_gated(desc) bytes out of the forward / into the backward, NULL as in hgrn2_fwd /
+ *          hgrn2_bwd (inference; re-created inside the workspace)
+ *   ws     hgrn2_workspace_bytes_gated(desc) bytes
+ * On the fp32 kernels the activations are applied in the load stage and their derivatives in the store stage.
+ * On the tensor-core kernels (bf16, dk = dv = 128) one element-wise kernel in front writes o, i and the gate as
+ * bf16 (kept in `saved`) - the gate as the smaller of f and 1 - f with a sign that says which, so that it is
+ * resolved to 2^-9 of min(f, 1 - f) at both ends of [0, 1] - the recurrence kernels decode that, and one
+ * element-wise kernel behind applies the chain rule in place and sums d_beta.
+ * Ownership, streams and errors as for hgrn2_fwd / hgrn2_bwd. */
+size_t hgrn2_saved_bytes_gated(const hgrn2_desc *desc);
+size_t hgrn2_workspace_bytes_gated(const hgrn2_desc *desc);
+hgrn2_status hgrn2_fwd_gated(const hgrn2_desc *desc, const void *zo, const void *zf, const void *zi,
+                             const float *beta, const float *S0, void *y, float *SN, void *saved,
+                             void *ws, void *cuda_stream);
+hgrn2_status hgrn2_bwd_gated(const hgrn2_desc *desc, const void *zo, const void *zf, const void *zi,
+                             const float *beta, const float *S0, const void *dy, const float *dSN,
+                             const void *saved, void *d_zo, void *d_zf, void *d_zi, float *d_beta,
+                             float *dS0, void *ws, void *cuda_stream);
+
 /* Largest chunk-state scratch, in bytes, that hgrn2_bwd_static_scratch can serve. */
 #define HGRN2_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
 

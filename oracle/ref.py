@@ -168,3 +168,37 @@ def hgrn2_bwd_varlen(o, f, i, cu, S0, dy, dSN=None):
         a, c, d, g = hgrn2_bwd(o[None, :, s:e], f[None, :, s:e], i[None, :, s:e], s0, dy[None, :, s:e], dsn)
         d_o[:, s:e], d_f[:, s:e], d_i[:, s:e], dS0[b] = a[0], c[0], d[0], g[0]
     return d_o, d_f, d_i, dS0
+
+
+def _sigmoid(x):
+    return 1.0 / (1.0 + np.exp(-np.asarray(x, dtype=np.float64)))
+
+
+def gates(zo, zf, zi, beta):
+    """Eq. 1 / Eq. 2: o = sigmoid(zo), f = beta + (1 - beta) sigmoid(zf), i = zi sigmoid(zi) (SiLU).
+    z* [B, H, N, d]; beta [H, d_k], broadcast over batch and time."""
+    b = np.asarray(beta, dtype=np.float64)[None, :, None, :]
+    zi = np.asarray(zi, dtype=np.float64)
+    return _sigmoid(zo), b + (1.0 - b) * _sigmoid(zf), zi * _sigmoid(zi)
+
+
+def hgrn2_fwd_gated(zo, zf, zi, beta, S0=None):
+    """The gate activations followed by Eq. 3.  Returns (y, S_N)."""
+    o, f, i = gates(zo, zf, zi, beta)
+    return hgrn2_fwd(o, f, i, S0)
+
+
+def hgrn2_bwd_gated(zo, zf, zi, beta, S0, dy, dSN=None):
+    """VJP of hgrn2_fwd_gated: hgrn2_bwd, then the chain rule through the three activations.
+    Returns (d_zo, d_zf, d_zi, d_beta [H, d_k], dS0)."""
+    o, f, i = gates(zo, zf, zi, beta)
+    d_o, d_f, d_i, dS0 = hgrn2_bwd(o, f, i, S0, dy, dSN)
+    b = np.asarray(beta, dtype=np.float64)[None, :, None, :]
+    g = _sigmoid(zf)
+    zi = np.asarray(zi, dtype=np.float64)
+    si = _sigmoid(zi)
+    d_zo = d_o * o * (1.0 - o)
+    d_zf = d_f * (1.0 - b) * g * (1.0 - g)
+    d_zi = d_i * si * (1.0 + zi * (1.0 - si))
+    d_beta = (d_f * (1.0 - g)).sum(axis=(0, 2))
+    return d_zo, d_zf, d_zi, d_beta, dS0

@@ -29,7 +29,7 @@ EXPORTS = (
     "hgrn2_saved_bytes", "hgrn2_workspace_bytes", "hgrn2_fwd", "hgrn2_bwd", "hgrn2_step",
     "hgrn2_step_multi", "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path", "hgrn2_bwd_static_scratch",
     "hgrn2_exact_path_units", "hgrn2_saved_bytes_varlen", "hgrn2_workspace_bytes_varlen", "hgrn2_fwd_varlen",
-    "hgrn2_bwd_varlen",
+    "hgrn2_bwd_varlen", "hgrn2_saved_bytes_gated", "hgrn2_workspace_bytes_gated", "hgrn2_fwd_gated", "hgrn2_bwd_gated",
 )
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
@@ -86,6 +86,14 @@ def load() -> ctypes.CDLL:
     lib.hgrn2_fwd_varlen.argtypes = [dp] + [vp] * 10
     lib.hgrn2_bwd_varlen.restype = ctypes.c_int
     lib.hgrn2_bwd_varlen.argtypes = [dp] + [vp] * 14
+    lib.hgrn2_saved_bytes_gated.restype = ctypes.c_size_t
+    lib.hgrn2_saved_bytes_gated.argtypes = [dp]
+    lib.hgrn2_workspace_bytes_gated.restype = ctypes.c_size_t
+    lib.hgrn2_workspace_bytes_gated.argtypes = [dp]
+    lib.hgrn2_fwd_gated.restype = ctypes.c_int
+    lib.hgrn2_fwd_gated.argtypes = [dp] + [vp] * 10
+    lib.hgrn2_bwd_gated.restype = ctypes.c_int
+    lib.hgrn2_bwd_gated.argtypes = [dp] + [vp] * 15
     lib.hgrn2_bwd_static_scratch.restype = ctypes.c_int
     lib.hgrn2_bwd_static_scratch.argtypes = [dp] + [vp] * 12
     lib.hgrn2_step.restype = ctypes.c_int
@@ -248,6 +256,53 @@ def hgrn2_bwd_varlen(o, f, i, cu_seqlens, S0, dy, dSN=None, saved=None, *, d_o=N
                                 _stream(stream))
     _check(code, "hgrn2_bwd_varlen")
     return d_o, d_f, d_i, dS0, ws
+
+
+def hgrn2_fwd_gated(zo, zf, zi, beta, S0=None, *, y=None, SN=None, saved=None, ws=None, want_final_state=True,
+                    save_for_backward=True, chunk=0, flags=0, stream=None):
+    """Forward from the pre-activations: o = sigmoid(zo), f = beta + (1 - beta) sigmoid(zf), i = silu(zi), then the
+    recurrence.  zo, zf [B, H, N, dk], zi [B, H, N, dv], beta [H, dk] float32.  Returns (y, SN, saved, ws, desc)."""
+    B, H, N, dk = zo.shape
+    dv = zi.shape[-1]
+    desc = make_desc(B, H, N, dk, dv, _io_code(zo), chunk, flags)
+    dev = zo.device
+    lib = load()
+    if y is None:
+        y = torch.empty((B, H, N, dv), dtype=zo.dtype, device=dev)
+    if SN is None and want_final_state:
+        SN = torch.empty((B, H, dk, dv), dtype=torch.float32, device=dev)
+    if saved is None and save_for_backward:
+        saved = torch.empty(max(int(lib.hgrn2_saved_bytes_gated(ctypes.byref(desc))), 16), dtype=torch.uint8, device=dev)
+    if ws is None:
+        ws = torch.empty(int(lib.hgrn2_workspace_bytes_gated(ctypes.byref(desc))), dtype=torch.uint8, device=dev)
+    code = lib.hgrn2_fwd_gated(ctypes.byref(desc), _ptr(zo), _ptr(zf), _ptr(zi), _ptr(beta), _ptr(S0), _ptr(y), _ptr(SN),
+                               _ptr(saved), _ptr(ws), _stream(stream))
+    _check(code, "hgrn2_fwd_gated")
+    return y, SN, saved, ws, desc
+
+
+def hgrn2_bwd_gated(zo, zf, zi, beta, S0, dy, dSN=None, saved=None, *, d_zo=None, d_zf=None, d_zi=None, d_beta=None,
+                    dS0=None, ws=None, want_dS0=True, want_d_beta=True, chunk=0, flags=0, stream=None):
+    """Backward of hgrn2_fwd_gated.  Returns (d_zo, d_zf, d_zi, d_beta, dS0, ws)."""
+    B, H, N, dk = zo.shape
+    dv = zi.shape[-1]
+    desc = make_desc(B, H, N, dk, dv, _io_code(zo), chunk, flags)
+    dev = zo.device
+    lib = load()
+    d_zo = torch.empty_like(zo) if d_zo is None else d_zo
+    d_zf = torch.empty_like(zf) if d_zf is None else d_zf
+    d_zi = torch.empty_like(zi) if d_zi is None else d_zi
+    if d_beta is None and want_d_beta:
+        d_beta = torch.empty((H, dk), dtype=torch.float32, device=dev)
+    if dS0 is None and want_dS0:
+        dS0 = torch.empty((B, H, dk, dv), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = torch.empty(int(lib.hgrn2_workspace_bytes_gated(ctypes.byref(desc))), dtype=torch.uint8, device=dev)
+    code = lib.hgrn2_bwd_gated(ctypes.byref(desc), _ptr(zo), _ptr(zf), _ptr(zi), _ptr(beta), _ptr(S0), _ptr(dy),
+                               _ptr(dSN), _ptr(saved), _ptr(d_zo), _ptr(d_zf), _ptr(d_zi), _ptr(d_beta), _ptr(dS0),
+                               _ptr(ws), _stream(stream))
+    _check(code, "hgrn2_bwd_gated")
+    return d_zo, d_zf, d_zi, d_beta, dS0, ws
 
 
 def hgrn2_bwd_static_scratch(o, f, i, S0, dy, dSN, d_o, d_f, d_i, dS0=None, status_out=None, *, chunk=0, flags=0,

@@ -16,6 +16,12 @@ size_t      tc_saved_bytes(const hgrn2_desc *d, int C);
 size_t      tc_segment_scratch_bytes(const hgrn2_desc *d, int C);
 size_t      tc_exact_scratch_bytes(const hgrn2_desc *d);
 size_t      tc_saved_bytes_packed(const hgrn2_desc *d);
+// gate activations (gates.cu)
+int         gate_bwd_slices(long long U, int N);
+cudaError_t launch_gate_fwd(const SeqArgs &a, const float *beta, void *o_out, void *k_out, void *i_out);
+cudaError_t launch_gate_bwd(const SeqArgs &a, const float *beta, float *partial, float *d_beta);
+cudaError_t launch_alu_fwd_gated(const SeqArgs &a, const float *beta);
+cudaError_t launch_alu_bwd_gated(const SeqArgs &a, const float *beta, float *partial, float *d_beta);
 cudaError_t launch_tc_fwd(const SeqArgs &a);
 cudaError_t launch_tc_bwd(const SeqArgs &a);
 }  // namespace hgrn2
@@ -259,6 +265,179 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
                        void *d_o, void *d_f, void *d_i, float *dS0, void *ws, void *cuda_stream)
 {
     return bwd_impl(desc, o, f, i, nullptr, S0, dy, dSN, saved, d_o, d_f, d_i, dS0, ws, cuda_stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+// Gated entry points.  Tensor-core path: `saved` = [o | encoded gate | i] (bf16, what the element-wise kernel in front wrote)
+// followed by the ordinary saved data; the workspace = status block | room for all of that when saved is NULL |
+// segment scratch | exact-path scratch | partial sums of d_beta.  fp32 path: the ordinary saved data and workspace
+// plus one row of partial sums per unit.
+size_t gate_tensor_bytes(const hgrn2_desc *d) { return (size_t)d->B * d->H * d->N * d->dk * 2; }
+
+size_t saved_bytes_gated(const hgrn2_desc *d, int C)
+{
+    return (use_tc(d) ? 3 * gate_tensor_bytes(d) : 0) + saved_bytes_for(d, C);
+}
+
+size_t beta_partial_bytes(const hgrn2_desc *d)
+{
+    const long long U = (long long)d->B * d->H;
+    const int P = use_tc(d) ? gate_bwd_slices(U, d->N) : 1;
+    return (((size_t)U * P * d->dk * sizeof(float)) + 255) & ~(size_t)255;
+}
+
+size_t workspace_bytes_gated(const hgrn2_desc *d, int C)
+{
+    return sizeof(StatusBlock) + saved_bytes_gated(d, C) +
+           (use_tc(d) ? tc_segment_scratch_bytes(d, C) + tc_exact_scratch_bytes(d) : 0) + beta_partial_bytes(d);
+}
+
+// Pointers into the workspace behind the saved-data room.
+void gated_ws_layout(SeqArgs &a, const hgrn2_desc *d, int C, void *ws, float **partial)
+{
+    char *p = static_cast<char *>(ws) + sizeof(StatusBlock) + saved_bytes_gated(d, C);
+    a.seg_scratch = nullptr;
+    a.exact_scratch = nullptr;
+    if (use_tc(d)) {
+        const size_t seg = tc_segment_scratch_bytes(d, C);
+        if (seg != 0) a.seg_scratch = p;
+        a.exact_scratch = reinterpret_cast<float *>(p + seg);
+        p += seg + tc_exact_scratch_bytes(d);
+    }
+    *partial = reinterpret_cast<float *>(p);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t hgrn2_saved_bytes_gated(const hgrn2_desc *desc)
+{
+    const int C = resolve_chunk(desc);
+    return C == 0 ? 0 : saved_bytes_gated(desc, C);
+}
+
+size_t hgrn2_workspace_bytes_gated(const hgrn2_desc *desc)
+{
+    const int C = resolve_chunk(desc);
+    return C == 0 ? 0 : workspace_bytes_gated(desc, C);
+}
+
+hgrn2_status hgrn2_fwd_gated(const hgrn2_desc *desc, const void *zo, const void *zf, const void *zi, const float *beta,
+                             const float *S0, void *y, float *SN, void *saved, void *ws, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    const int C = resolve_chunk(desc);
+    if (C == 0) return HGRN2_ERR_UNSUPPORTED;
+    if (!ws) return HGRN2_ERR_WORKSPACE;
+    const bool empty = (size_t)desc->B * desc->H * desc->N == 0;
+    const void *req[] = {ws, zo, zf, zi, y, beta};
+    const void *opt[] = {S0, SN, saved, zo, zf, zi, y, beta};
+    hgrn2_status st = check_ptrs(req, empty ? 1 : 6, opt, empty ? 8 : 3);
+    if (st != HGRN2_OK) return st;
+
+    SeqArgs a;
+    fill_args(a, desc, C, cuda_stream, ws);
+    float *partial = nullptr;
+    gated_ws_layout(a, desc, C, ws, &partial);
+    a.o = zo; a.f = zf; a.i = zi; a.S0 = S0; a.y = y; a.SN = SN;
+    a.status = static_cast<StatusBlock *>(ws);
+    const bool tc = use_tc(desc);
+    a.clear_status = tc && !empty;
+    if (!a.clear_status && cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+    if ((size_t)desc->B * desc->H == 0) return HGRN2_OK;
+    if (desc->N == 0) {
+        if (SN) {
+            cudaError_t e = S0 ? cudaMemcpyAsync(SN, S0, state_bytes(desc), cudaMemcpyDeviceToDevice, a.stream)
+                               : cudaMemsetAsync(SN, 0, state_bytes(desc), a.stream);
+            if (e != cudaSuccess) return HGRN2_ERR_CUDA;
+        }
+        return HGRN2_OK;
+    }
+    if (!tc) {
+        a.states = static_cast<float *>(saved);
+        return launch_alu_fwd_gated(a, beta) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+    }
+    // the gates go to the head of `saved` (kept for the backward) or, for inference, of the workspace's room for it
+    char *gates = saved ? static_cast<char *>(saved) : static_cast<char *>(ws) + sizeof(StatusBlock);
+    const size_t gb = gate_tensor_bytes(desc);
+    if (launch_gate_fwd(a, beta, gates, gates + gb, gates + 2 * gb) != cudaSuccess) return HGRN2_ERR_CUDA;
+    a.o = gates; a.f = gates + gb; a.i = gates + 2 * gb;
+    a.gate_enc = true;
+    a.states = saved ? reinterpret_cast<float *>(gates + 3 * gb) : nullptr;
+    return launch_tc_fwd(a) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+hgrn2_status hgrn2_bwd_gated(const hgrn2_desc *desc, const void *zo, const void *zf, const void *zi, const float *beta,
+                             const float *S0, const void *dy, const float *dSN, const void *saved, void *d_zo,
+                             void *d_zf, void *d_zi, float *d_beta, float *dS0, void *ws, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    const int C = resolve_chunk(desc);
+    if (C == 0) return HGRN2_ERR_UNSUPPORTED;
+    if (!ws) return HGRN2_ERR_WORKSPACE;
+    const bool empty = (size_t)desc->B * desc->H * desc->N == 0;
+    const void *req[] = {ws, zo, zf, zi, dy, d_zo, d_zf, d_zi, beta};
+    const void *opt[] = {S0, dSN, saved, dS0, d_beta, zo, zf, zi, dy, d_zo, d_zf, d_zi, beta};
+    hgrn2_status st = check_ptrs(req, empty ? 1 : 9, opt, empty ? 13 : 5);
+    if (st != HGRN2_OK) return st;
+
+    SeqArgs a;
+    fill_args(a, desc, C, cuda_stream, ws);
+    float *partial = nullptr;
+    gated_ws_layout(a, desc, C, ws, &partial);
+    a.o = zo; a.f = zf; a.i = zi; a.S0 = S0; a.dy = dy; a.dSN = dSN;
+    a.d_o = d_zo; a.d_f = d_zf; a.d_i = d_zi; a.dS0 = dS0;
+    a.status = static_cast<StatusBlock *>(ws);
+    const bool tc = use_tc(desc);
+    a.clear_status = tc && !empty;
+    if (!a.clear_status && cudaMemsetAsync(ws, 0, sizeof(StatusBlock), a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+    const size_t beta_bytes = (size_t)desc->H * desc->dk * sizeof(float);
+    if (empty) {                                 // no token: nothing depends on beta; the state gradient passes through
+        if (d_beta && cudaMemsetAsync(d_beta, 0, beta_bytes, a.stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+        if ((size_t)desc->B * desc->H != 0 && dS0) {
+            cudaError_t e = dSN ? cudaMemcpyAsync(dS0, dSN, state_bytes(desc), cudaMemcpyDeviceToDevice, a.stream)
+                                : cudaMemsetAsync(dS0, 0, state_bytes(desc), a.stream);
+            if (e != cudaSuccess) return HGRN2_ERR_CUDA;
+        }
+        return HGRN2_OK;
+    }
+    if (!tc) {
+        if (saved) {
+            a.states = const_cast<float *>(static_cast<const float *>(saved));
+        } else {
+            SeqArgs r = a;
+            r.y = nullptr; r.SN = nullptr;
+            r.states = reinterpret_cast<float *>(static_cast<char *>(ws) + sizeof(StatusBlock));
+            if (launch_alu_fwd_gated(r, beta) != cudaSuccess) return HGRN2_ERR_CUDA;
+            a.states = r.states;
+        }
+        return launch_alu_bwd_gated(a, beta, partial, d_beta) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+    }
+    const size_t gb = gate_tensor_bytes(desc);
+    char *gates;
+    SeqArgs k = a;                               // the recurrence proper, on o, the encoded gate, i
+    k.gate_enc = true;
+    if (saved) {
+        gates = const_cast<char *>(static_cast<const char *>(saved));
+    } else {
+        gates = static_cast<char *>(ws) + sizeof(StatusBlock);
+        if (launch_gate_fwd(a, beta, gates, gates + gb, gates + 2 * gb) != cudaSuccess) return HGRN2_ERR_CUDA;
+        SeqArgs r = k;
+        r.o = gates; r.f = gates + gb; r.i = gates + 2 * gb;
+        r.y = nullptr; r.SN = nullptr;
+        r.states = reinterpret_cast<float *>(gates + 3 * gb);
+        if (launch_tc_fwd(r) != cudaSuccess) return HGRN2_ERR_CUDA;
+        k.clear_status = false;
+    }
+    k.o = gates; k.f = gates + gb; k.i = gates + 2 * gb;
+    k.states = reinterpret_cast<float *>(gates + 3 * gb);
+    if (launch_tc_bwd(k) != cudaSuccess) return HGRN2_ERR_CUDA;
+    // d_o, d_f, d_i sit in the output buffers: chain rule through the activations, in place, and d_beta
+    return launch_gate_bwd(a, beta, partial, d_beta) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
 }
 
 hgrn2_status hgrn2_fwd_varlen(const hgrn2_desc *desc, const void *o, const void *f, const void *i,

@@ -35,6 +35,37 @@
 namespace hgrn2 {
 namespace alu {
 
+// What the three input tensors hold.  kGateIsF: o, f, i themselves.  kGateEnc: o, the signed gate encoding
+// (the smaller of f and k = 1 - f, negative when it is k; what the tensor-core path of the gated entry points is
+// handed), i.  kGatePre: the pre-activations zo, zf, zi of Eq. 1 / Eq. 2, turned into
+// o = sigmoid(zo), f = beta + (1 - beta) sigmoid(zf), i = silu(zi) as they are loaded (fp32, so f is never rounded to
+// the I/O type), and the backward returns the gradients with respect to the pre-activations and to beta.
+enum GateMode { kGateIsF = 0, kGateEnc = 1, kGatePre = 2 };
+
+__device__ __forceinline__ float sigmoid_f(float x) { return 1.0f / (1.0f + expf(-x)); }
+
+// Gate values of one (token, key dimension) from what the tensors hold: q, f and k = 1 - f.
+template <int kMode>
+__device__ __forceinline__ void gate_values(float qraw, float fraw, float beta, float &qv, float &fv, float &kv)
+{
+    if (kMode == kGateIsF) { qv = qraw; fv = fraw; kv = 1.0f - fraw; }
+    else if (kMode == kGateEnc) {
+        qv = qraw;
+        const float m = fabsf(fraw);
+        if (signbit(fraw)) { kv = m; fv = 1.0f - m; } else { fv = m; kv = 1.0f - m; }
+    }
+    else {
+        const float g = sigmoid_f(fraw);
+        qv = sigmoid_f(qraw);
+        kv = (1.0f - beta) * (1.0f - g);
+        fv = 1.0f - kv;
+    }
+}
+template <int kMode> __device__ __forceinline__ float value_of(float vraw)
+{
+    return kMode == kGatePre ? vraw * sigmoid_f(vraw) : vraw;
+}
+
 __host__ __device__ constexpr size_t fwd_smem_floats(int dk, int dv, int C)
 {
     const size_t ldk = dk + 1, ldv = dv + 1;
@@ -49,10 +80,12 @@ __host__ __device__ constexpr size_t bwd_smem_floats(int dk, int dv, int C)
 // Forward of one unit, run by every thread of the CTA.  All pointers are the unit's own (token 0, element 0).
 // ST = element type of the kept chunk-start states; the state of chunk c goes to slot c / every when
 // c % every == 0 (every = 1: all chunks).  yu, SNu, states_u may be null.
-template <typename T, typename ST>
+// beta_h: this head's lower bounds [dk] (kGatePre only).
+template <typename T, typename ST, int kMode = kGateIsF>
 __device__ void fwd_unit(float *smem, const T *__restrict__ ou, const T *__restrict__ fu, const T *__restrict__ iu,
                          const float *__restrict__ S0u, T *__restrict__ yu, float *__restrict__ SNu,
-                         ST *__restrict__ states_u, int every, int N, int dk, int dv, int C, int NC)
+                         ST *__restrict__ states_u, int every, int N, int dk, int dv, int C, int NC,
+                         const float *__restrict__ beta_h = nullptr)
 {
     const int ldk = dk + 1, ldv = dv + 1, ldA = C + 1;
     float *q = smem;                 // [C][ldk]   o, later o * Lam
@@ -72,18 +105,17 @@ __device__ void fwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
         const int t0 = c * C;
         for (int x = tid; x < C * dk; x += nt) {
             const int t = x / dk, kx = x - t * dk, tok = t0 + t;
-            float qv = 0.f, fv = 1.f;
-            if (tok < N) {
-                qv = load_f(ou + (long long)tok * dk + kx);
-                fv = load_f(fu + (long long)tok * dk + kx);
-            }
+            float qv = 0.f, fv = 1.f, kv = 0.f;
+            if (tok < N)
+                gate_values<kMode>(load_f(ou + (long long)tok * dk + kx), load_f(fu + (long long)tok * dk + kx),
+                                   kMode == kGatePre ? beta_h[kx] : 0.f, qv, fv, kv);
             q[t * ldk + kx] = qv;
-            k[t * ldk + kx] = 1.0f - fv;
+            k[t * ldk + kx] = kv;
             b[t * ldk + kx] = logf(fmaxf(fv, kFMin));
         }
         for (int x = tid; x < C * dv; x += nt) {
             const int t = x / dv, vx = x - t * dv, tok = t0 + t;
-            v[t * ldv + vx] = tok < N ? load_f(iu + (long long)tok * dv + vx) : 0.f;
+            v[t * ldv + vx] = tok < N ? value_of<kMode>(load_f(iu + (long long)tok * dv + vx)) : 0.f;
         }
         if (states_u && c % every == 0) {
             ST *dst = states_u + (long long)(c / every) * ss;
@@ -145,11 +177,14 @@ __device__ void fwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
 // Backward of one unit.  states_u holds the chunk-start state of chunk c in slot c / every for c % every == 0;
 // with every = 2 the state of an odd chunk is re-created from the slot of the chunk before it and that chunk's
 // tokens into `scratch` ([dk][dv] floats in global memory, this unit's own).  dSNu, dS0u may be null.
-template <typename T, typename ST>
+// kGatePre: beta_h = this head's lower bounds [dk]; dou, dfu, diu receive the gradients with respect to zo, zf, zi
+// and dbeta_u[dk] (nullable) this unit's share of the gradient with respect to beta.
+template <typename T, typename ST, int kMode = kGateIsF>
 __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restrict__ fu, const T *__restrict__ iu,
                          const T *__restrict__ gu, const float *__restrict__ dSNu, const ST *states_u, int every,
                          float *scratch, T *__restrict__ dou, T *__restrict__ dfu, T *__restrict__ diu,
-                         float *__restrict__ dS0u, int N, int dk, int dv, int C, int NC)
+                         float *__restrict__ dS0u, int N, int dk, int dv, int C, int NC,
+                         const float *__restrict__ beta_h = nullptr, float *__restrict__ dbeta_u = nullptr)
 {
     const int ldk = dk + 1, ldv = dv + 1, ldA = C + 1;
     float *q   = smem;               // [C][ldk]  o, later o * Lam
@@ -173,6 +208,7 @@ __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
     }
     __syncthreads();
 
+    float dbeta_acc = 0.f;           // kGatePre: a thread owns one key dimension in the d_f scan (dk <= blockDim.x)
     for (int c = NC - 1; c >= 0; --c) {
         const int t0 = c * C;
         const ST *slot = states_u + (long long)(c / every) * ss;
@@ -182,13 +218,15 @@ __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
             const int p0 = (c - 1) * C;
             for (int x = tid; x < C * dk; x += nt) {
                 const int t = x / dk, kx = x - t * dk;
-                const float fv = load_f(fu + (long long)(p0 + t) * dk + kx);
-                k[t * ldk + kx] = 1.0f - fv;
+                float qv, fv, kv;
+                gate_values<kMode>(0.f, load_f(fu + (long long)(p0 + t) * dk + kx), kMode == kGatePre ? beta_h[kx] : 0.f,
+                                   qv, fv, kv);
+                k[t * ldk + kx] = kv;
                 b[t * ldk + kx] = logf(fmaxf(fv, kFMin));
             }
             for (int x = tid; x < C * dv; x += nt) {
                 const int t = x / dv, vx = x - t * dv;
-                v[t * ldv + vx] = load_f(iu + (long long)(p0 + t) * dv + vx);
+                v[t * ldv + vx] = value_of<kMode>(load_f(iu + (long long)(p0 + t) * dv + vx));
             }
             __syncthreads();
             for (int kx = tid; kx < dk; kx += nt) {
@@ -215,20 +253,19 @@ __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
         auto S_in = [&](int idx) -> float { return recreate ? scratch[idx] : load_f(slot + idx); };
         for (int x = tid; x < C * dk; x += nt) {
             const int t = x / dk, kx = x - t * dk, tok = t0 + t;
-            float qv = 0.f, fv = 1.f;
-            if (tok < N) {
-                qv = load_f(ou + (long long)tok * dk + kx);
-                fv = load_f(fu + (long long)tok * dk + kx);
-            }
+            float qv = 0.f, fv = 1.f, kv = 0.f;
+            if (tok < N)
+                gate_values<kMode>(load_f(ou + (long long)tok * dk + kx), load_f(fu + (long long)tok * dk + kx),
+                                   kMode == kGatePre ? beta_h[kx] : 0.f, qv, fv, kv);
             q[t * ldk + kx] = qv;
-            k[t * ldk + kx] = 1.0f - fv;
+            k[t * ldk + kx] = kv;
             b[t * ldk + kx] = logf(fmaxf(fv, kFMin));
         }
         for (int x = tid; x < C * dv; x += nt) {
             const int t = x / dv, vx = x - t * dv, tok = t0 + t;
             float vv = 0.f, gv = 0.f;
             if (tok < N) {
-                vv = load_f(iu + (long long)tok * dv + vx);
+                vv = value_of<kMode>(load_f(iu + (long long)tok * dv + vx));
                 gv = load_f(gu + (long long)tok * dv + vx);
             }
             v[t * ldv + vx] = vv;
@@ -287,7 +324,7 @@ __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
             const int p = t * ldk + kx;
             const float qv = q[p], kv = k[p], bv = b[p], bC = b[(C - 1) * ldk + kx];
             const float dqv = dq[p];
-            if (tok < N) store_f(dou + (long long)tok * dk + kx, dqv);
+            if (tok < N) store_f(dou + (long long)tok * dk + kx, kMode == kGatePre ? dqv * qv * (1.0f - qv) : dqv);
             dq[p] = qv * dqv - kv * dkk[p] + e[p];
             q[p] = qv * expf(bv);
             k[p] = kv * expf(bC - bv);
@@ -301,6 +338,10 @@ __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
             for (int t = s; t < C; ++t) acc = fmaf(A[t * ldA + s], g[t * ldv + vx], acc);
             const float *ks = k + s * ldk;
             for (int kx = 0; kx < dk; ++kx) acc = fmaf(ks[kx], dS[kx * ldv + vx], acc);
+            if (kMode == kGatePre) {                  // d silu(z) / dz = s (1 + z (1 - s)), s = sigmoid(z)
+                const float z = load_f(iu + (long long)tok * dv + vx), sg = sigmoid_f(z);
+                acc *= sg * (1.0f + z * (1.0f - sg));
+            }
             store_f(diu + (long long)tok * dv + vx, acc);
         }
         // d_f: one thread per key dimension scans the chunk
@@ -320,9 +361,17 @@ __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
                 suf += dq[t * ldk + kx];
                 const int tok = t0 + t;
                 if (tok < N) {
-                    const float fv = load_f(fu + (long long)tok * dk + kx);
+                    const float fraw = load_f(fu + (long long)tok * dk + kx);
+                    float qv, fv, kv;
+                    gate_values<kMode>(0.f, fraw, kMode == kGatePre ? beta_h[kx] : 0.f, qv, fv, kv);
                     const float dg = base + e[t * ldk + kx] + suf;
-                    store_f(dfu + (long long)tok * dk + kx, dg / fmaxf(fv, kFMin) - dkk[t * ldk + kx]);
+                    float dfv = dg / fmaxf(fv, kMode == kGateEnc ? kFDivMinK : kFMin) - dkk[t * ldk + kx];
+                    if (kMode == kGatePre) {          // f = beta + (1 - beta) g:  df/dzf = (1 - beta) g (1 - g),  df/dbeta = 1 - g
+                        const float g = sigmoid_f(fraw);
+                        dbeta_acc += dfv * (1.0f - g);
+                        dfv *= (1.0f - beta_h[kx]) * g * (1.0f - g);
+                    }
+                    store_f(dfu + (long long)tok * dk + kx, dfv);
                 }
             }
         }
@@ -341,6 +390,7 @@ __device__ void bwd_unit(float *smem, const T *__restrict__ ou, const T *__restr
             const int kx = x / dv, vx = x - kx * dv;
             dS0u[x] = dS[kx * ldv + vx];
         }
+    if (kMode == kGatePre && dbeta_u != nullptr && tid < dk) dbeta_u[tid] = dbeta_acc;
 }
 
 }  // namespace alu

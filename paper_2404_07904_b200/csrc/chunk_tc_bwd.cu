@@ -115,7 +115,7 @@ static_assert(alu::bwd_smem_floats(kD, kD, kExactC) * sizeof(float) <= kSmemByte
 // o and f as plain [64][128] bf16 tiles (rows beyond the end of the sequence hold zeros, or in a packed batch the
 // next sequence's tokens: they are patched to the neutral f = 1, o = 0).  Qs and Ks are recomputed from them with the transform's own roundings, so the
 // operand stage does not have to be held until the outputs are done.
-template <bool kUp, bool kRagged>
+template <bool kUp, bool kRagged, bool kEnc>
 __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat16 *oraw, const __nv_bfloat16 *fraw,
                                            int k, __nv_bfloat16 *do_g, int n_valid, float &asum, float &esum)
 {
@@ -135,8 +135,14 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
             const int t = t0 + j;
             fw[j] = reinterpret_cast<const unsigned short *>(fraw)[t * kD + k];
             qw[j] = reinterpret_cast<const unsigned short *>(oraw)[t * kD + k];
-            if (kRagged && t >= n_valid) { fw[j] = 0x3F80u; qw[j] = 0u; }
-            fv[j] = __uint_as_float(fw[j] << 16);
+            if (kRagged && t >= n_valid) { fw[j] = kEnc ? 0x8000u : 0x3F80u; qw[j] = 0u; }
+            if (kEnc) {                       // fw[j] becomes the bf16 bits of k, as the transform formed them
+                float kv;
+                gate_decode(fw[j], fv[j], kv);
+                fw[j] = pack_bf16(kv, 0.f) & 0xFFFFu;        // rounded to bf16 exactly as the transform rounds it
+            } else {
+                fv[j] = __uint_as_float(fw[j] << 16);
+            }
         }
         tmem_wait_ld();
         // scale factors along the walk (sequential in the running product), 1/f
@@ -150,7 +156,7 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
             if (!kUp) cp *= fv[j];
             sq[j] = kUp ? m : mi;
             sk[j] = kUp ? mi : m;
-            rf[j] = rcp_fast(fmaxf(fv[j], kProdFloor));
+            rf[j] = rcp_fast(fmaxf(fv[j], kEnc ? kFDivMinK : kProdFloor));
         }
         // element-wise part, two rows per instruction (packed fp32)
         float a[8], e[8], dk[8];
@@ -164,7 +170,8 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
             // of a cancel in pairs along the chunk only if both sides use the same operand values
             const uint32_t sqp = pack_bf16(sq[j], sq[j + 1]), skp = pack_bf16(sk[j], sk[j + 1]);
             const uint32_t qsp = mul_bf16x2(qw[j] | (qw[j + 1] << 16), sqp);
-            const uint32_t ksp = fma_bf16x2(fw[j] | (fw[j + 1] << 16), skp ^ 0x80008000u, skp);
+            const uint32_t ksp = kEnc ? mul_bf16x2(fw[j] | (fw[j + 1] << 16), skp)
+                                      : fma_bf16x2(fw[j] | (fw[j + 1] << 16), skp ^ 0x80008000u, skp);
             const float2 QS = make_float2(bf16_lo(qsp), bf16_hi(qsp)), KS = make_float2(bf16_lo(ksp), bf16_hi(ksp));
             const float2 dox = mul2(X, make_float2(sq[j], sq[j + 1]));
             const float2 a2 = sub2(mul2(QS, X), mul2(KS, Y));
@@ -200,7 +207,8 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
 // kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens); when false,
 // every per-row validity test below folds away.
 // kMultiCta: a unit runs as several CTAs (segments) of this launch (see the forward kernel).
-template <bool kRagged, bool kMultiCta>
+// kEnc: the f tensor holds the signed gate encoding (see transform_half); d_f stays the gradient with respect to f.
+template <bool kRagged, bool kMultiCta, bool kEnc>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_dy,
@@ -327,9 +335,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int n_valid = kRagged ? N - c * kC : kC;
             // Pm and E of the chunk are not kept: the backward takes them from what the forward saved
             if (n_valid >= kC) {
-                transform_stream<true, kSS, kSlab>(qbuf + kOffQ, qbuf + kOffK, nullptr, nullptr, nullptr, nullptr, kC, tid);
+                transform_stream<true, kEnc, kSS, kSlab>(qbuf + kOffQ, qbuf + kOffK, nullptr, nullptr, nullptr, nullptr, kC, tid);
             } else {
-                transform_stream<false, kSS, kSlab>(qbuf + kOffQ, qbuf + kOffK, nullptr, nullptr, nullptr, nullptr, n_valid, tid);
+                transform_stream<false, kEnc, kSS, kSlab>(qbuf + kOffQ, qbuf + kOffK, nullptr, nullptr, nullptr, nullptr, n_valid, tid);
             }
             fence_proxy_async_smem();
             mbar_arrive(&ctl->t_done[s]);
@@ -466,8 +474,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             tc_fence_after_sync();
             float asum, esum;
             PT_STAMP(status, 14, tid == kWarpE3 * 32 && it == 16)
-            if (half) phase_main<true, kRagged>(tl, oraw, fraw, krow, d_o + crow0 * kD + krow, n_valid, asum, esum);
-            else      phase_main<false, kRagged>(tl, oraw, fraw, krow, d_o + crow0 * kD + krow, n_valid, asum, esum);
+            if (half) phase_main<true, kRagged, kEnc>(tl, oraw, fraw, krow, d_o + crow0 * kD + krow, n_valid, asum, esum);
+            else      phase_main<false, kRagged, kEnc>(tl, oraw, fraw, krow, d_o + crow0 * kD + krow, n_valid, asum, esum);
             mbar_arrive(&ctl->raw_read);
             if (half) xa[krow] = asum; else xe[krow] = esum;
             tmem_wait_st();
@@ -756,7 +764,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     const int n_unit = packed ? N : ex.N;                          // tokens of the whole unit
     const size_t seq = packed ? grow0 * kD : (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
     const size_t slot_u = packed ? slot0 : (size_t)unit * ((ex.N + kC - 1) / kC);
-    alu::bwd_unit<__nv_bfloat16, __nv_bfloat16>(
+    alu::bwd_unit<__nv_bfloat16, __nv_bfloat16, kEnc ? alu::kGateEnc : alu::kGateIsF>(
         reinterpret_cast<float *>(smem), ex.o + seq, ex.f + seq, ex.i + seq, ex.dy + seq, ex.dSN ? ex.dSN + st : nullptr,
         ex.states + slot_u * kD * kD, kC / kExactC, ex.scratch + st, ex.d_o + seq, ex.d_f + seq,
         ex.d_i + seq, ex.dS0 ? ex.dS0 + st : nullptr, n_unit, kD, kD, kExactC, (n_unit + kExactC - 1) / kExactC);
@@ -825,8 +833,12 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
         return cudaErrorInvalidValue;
     const bool ragged = N % kC != 0 || pk.cu != nullptr;
     if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
-    auto kernel = ragged ? tc_bwd_kernel<true, false>
-                         : (ex.o != nullptr && ex.G > 1 ? tc_bwd_kernel<false, true> : tc_bwd_kernel<false, false>);
+    auto kernel = a.gate_enc ? (ragged ? tc_bwd_kernel<true, false, true>
+                                   : (ex.o != nullptr && ex.G > 1 ? tc_bwd_kernel<false, true, true>
+                                                                   : tc_bwd_kernel<false, false, true>))
+                         : (ragged ? tc_bwd_kernel<true, false, false>
+                                   : (ex.o != nullptr && ex.G > 1 ? tc_bwd_kernel<false, true, false>
+                                                                   : tc_bwd_kernel<false, false, false>));
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
@@ -869,7 +881,7 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         float *lam = dS_end + Ut * G * kD * kD;
         int *unit_flag = reinterpret_cast<int *>(lam + Ut * G * kD), *unit_count = unit_flag + Ut;
         // state-gradient contributions of the segments (chunk_tc_state.cu): they hold for every f
-        err = launch_tc_state_bwd(t.o, t.f, t.dy, Ut * G, a.N / G, G_loc, lam, a.status, clear, a.start_aborted, a.stream);
+        err = launch_tc_state_bwd(t.o, t.f, t.dy, Ut * G, a.N / G, G_loc, lam, a.gate_enc, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
         seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G,
                                                                                     unit_flag, unit_count, (int)Ut);

@@ -81,7 +81,8 @@ static_assert(alu::fwd_smem_floats(kD, kD, kExactC) * sizeof(float) <= kSmemByte
 // kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens).
 // kMultiCta: a unit runs as several CTAs (segments) of this launch; the bookkeeping that lets the last of them
 // take the unit's exact path is compiled in only then (its mere presence costs the one-CTA-per-unit launch 3 %).
-template <bool kRagged, bool kMultiCta>
+// kEnc: the f tensor holds k = 1 - f (see transform_half).
+template <bool kRagged, bool kMultiCta, bool kEnc>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
               const __grid_constant__ CUtensorMap map_i, const __grid_constant__ CUtensorMap map_y,
@@ -185,10 +186,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int n_valid = kRagged ? N - c * kC : kC;
             float *tg = totals ? totals + (slot0 + c) * 2 * kD : nullptr;       // Pm, E of the chunk for the backward
             if (n_valid >= kC) {
-                transform_stream<true>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
+                transform_stream<true, kEnc>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
                                        kC, tt);
             } else {
-                transform_stream<false>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
+                transform_stream<false, kEnc>(qbuf, qbuf + kTile, pm + (c & 3) * 128, ee + (c & 3) * 128, tg, tg ? tg + kD : nullptr,
                                         n_valid, tt);
             }
             fence_proxy_async_smem();
@@ -559,7 +560,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
     const int n_unit = packed ? N : ex.N;                          // tokens of the whole unit
     const size_t seq = packed ? ((size_t)zu * N_all + row0) * kD : (size_t)unit * ex.N * kD, st = (size_t)unit * kD * kD;
     const size_t slot_u = packed ? slot0 : (size_t)unit * ((ex.N + kC - 1) / kC);
-    alu::fwd_unit<__nv_bfloat16, __nv_bfloat16>(
+    alu::fwd_unit<__nv_bfloat16, __nv_bfloat16, kEnc ? alu::kGateEnc : alu::kGateIsF>(
         reinterpret_cast<float *>(smem), ex.o + seq, ex.f + seq, ex.i + seq, ex.S0 ? ex.S0 + st : nullptr,
         ex.y ? ex.y + seq : nullptr, ex.SN ? ex.SN + st : nullptr,
         ex.states ? ex.states + slot_u * kD * kD : nullptr, kC / kExactC, n_unit, kD, kD, kExactC,
@@ -724,8 +725,12 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
         return cudaErrorInvalidValue;
     const bool ragged = N % kC != 0 || pk.cu != nullptr;
     if (ex.o != nullptr && ex.G > 1 && ragged) return cudaErrorInvalidValue;      // segments are whole chunks
-    auto kernel = ragged ? tc_fwd_kernel<true, false>
-                         : (ex.o != nullptr && ex.G > 1 ? tc_fwd_kernel<false, true> : tc_fwd_kernel<false, false>);
+    auto kernel = a.gate_enc ? (ragged ? tc_fwd_kernel<true, false, true>
+                                   : (ex.o != nullptr && ex.G > 1 ? tc_fwd_kernel<false, true, true>
+                                                                   : tc_fwd_kernel<false, false, true>))
+                         : (ragged ? tc_fwd_kernel<true, false, false>
+                                   : (ex.o != nullptr && ex.G > 1 ? tc_fwd_kernel<false, true, false>
+                                                                   : tc_fwd_kernel<false, false, false>));
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? a.totals : nullptr;
@@ -784,7 +789,7 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         float *lam = S_start + Ut * G * kD * kD;
         int *unit_flag = reinterpret_cast<int *>(lam + Ut * G * kD), *unit_count = unit_flag + Ut;
         // the state-only pass (chunk_tc_state.cu) holds for every f: it needs no exact path of its own
-        err = launch_tc_state_fwd(t.f, t.i, Ut * G, a.N / G, S_loc, lam, a.status, clear, a.start_aborted, a.stream);
+        err = launch_tc_state_fwd(t.f, t.i, Ut * G, a.N / G, S_loc, lam, a.gate_enc, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
         seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G,
                                                                                 unit_flag, unit_count, (int)Ut);

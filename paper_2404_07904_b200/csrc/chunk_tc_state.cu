@@ -54,7 +54,8 @@ struct Ctl {
 };
 static_assert(sizeof(Ctl) <= 256, "control block");
 
-template <bool kBwd>
+// kEnc: the f tensor holds the signed gate encoding (see transform_half in tc_chunk.cuh).
+template <bool kBwd, bool kEnc>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
                 const __grid_constant__ CUtensorMap map_w, float *__restrict__ out, float *__restrict__ lam, int NC,
@@ -118,8 +119,16 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
             for (int j = 0; j < 32; ++j) {
                 const int r = 32 * half + j;
                 fw[j] = *reinterpret_cast<const uint32_t *>(fbuf + xo[r & 7] + r * 128);
-                h0 *= bf16_lo(fw[j]);
-                h1 *= bf16_hi(fw[j]);
+                float f0, f1, k0, k1;
+                if (kEnc) {
+                    gate_decode(fw[j], f0, k0);
+                    gate_decode(fw[j] >> 16, f1, k1);
+                } else {
+                    f0 = bf16_lo(fw[j]);
+                    f1 = bf16_hi(fw[j]);
+                }
+                h0 *= f0;
+                h1 *= f1;
             }
             float *hb = hp + (n & 1) * 256;
             *reinterpret_cast<float2 *>(hb + half * 128 + col) = make_float2(h0, h1);
@@ -135,16 +144,24 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
                 const int j = kBwd ? i : 31 - i;                      // forward pass: rows from the end backwards
                 const int r = 32 * half + j;
                 const uint32_t off = xo[r & 7] + r * 128;
+                float f0, f1, k0 = 0.f, k1 = 0.f;
+                if (kEnc) {
+                    gate_decode(fw[j], f0, k0);
+                    gate_decode(fw[j] >> 16, f1, k1);
+                } else {
+                    f0 = bf16_lo(fw[j]);
+                    f1 = bf16_hi(fw[j]);
+                }
                 if (kBwd) {                                           // c includes row r: X = q * prod_{<= r} f
-                    a0 *= bf16_lo(fw[j]);
-                    a1 *= bf16_hi(fw[j]);
+                    a0 *= f0;
+                    a1 *= f1;
                     const uint32_t qw = *reinterpret_cast<const uint32_t *>(xbuf + off);
                     *reinterpret_cast<uint32_t *>(xbuf + off) = mul_bf16x2(qw, pack_bf16(a0, a1));
                 } else {                                              // c excludes row r: X = (1 - f) * prod_{> r} f
                     const uint32_t cp = pack_bf16(a0, a1);
-                    *reinterpret_cast<uint32_t *>(xbuf + off) = fma_bf16x2(fw[j], cp ^ 0x80008000u, cp);
-                    a0 *= bf16_lo(fw[j]);
-                    a1 *= bf16_hi(fw[j]);
+                    *reinterpret_cast<uint32_t *>(xbuf + off) = kEnc ? mul_bf16x2(pack_bf16(k0, k1), cp) : fma_bf16x2(fw[j], cp ^ 0x80008000u, cp);
+                    a0 *= f0;
+                    a1 *= f1;
                 }
             }
             fence_proxy_async_smem();
@@ -225,7 +242,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
     if (warp == 0) tmem_dealloc(tmem, 128);
 }
 
-template <bool kBwd>
+template <bool kBwd, bool kEnc>
 cudaError_t launch_state(const void *o, const void *f, const void *w, uint64_t U, int N, int NC, float *out, float *lam,
                          StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream)
 {
@@ -233,10 +250,10 @@ cudaError_t launch_state(const void *o, const void *f, const void *w, uint64_t U
     CUtensorMap mo, mf, mw;
     if (!make_map(&mo, kBwd ? o : f, U, N, kC) || !make_map(&mf, f, U, N, kC) || !make_map(&mw, w, U, N, kC))
         return cudaErrorInvalidValue;
-    cudaError_t err = cudaFuncSetAttribute(tc_state_kernel<kBwd>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t err = cudaFuncSetAttribute(tc_state_kernel<kBwd, kEnc>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)G::kSmemBytes);
     if (err != cudaSuccess) return err;
-    tc_state_kernel<kBwd><<<(unsigned)U, kThreads, G::kSmemBytes, stream>>>(mo, mf, mw, out, lam, NC, status,
+    tc_state_kernel<kBwd, kEnc><<<(unsigned)U, kThreads, G::kSmemBytes, stream>>>(mo, mf, mw, out, lam, NC, status,
                                                                              clear ? 1 : 0, start_aborted);
     return cudaGetLastError();
 }
@@ -244,17 +261,20 @@ cudaError_t launch_state(const void *o, const void *f, const void *w, uint64_t U
 }  // namespace
 
 // Forward: S_loc [U][128][128] and Lambda [U][128] of U segments of N tokens (whole chunks) from f and i.
-cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam,
+cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam, bool gate_enc,
                                 StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream)
 {
-    return launch_state<false>(nullptr, f, i, U, N, N / kC, S_loc, lam, status, clear, start_aborted, stream);
+    if (gate_enc) return launch_state<false, true>(nullptr, f, i, U, N, N / kC, S_loc, lam, status, clear, start_aborted, stream);
+    return launch_state<false, false>(nullptr, f, i, U, N, N / kC, S_loc, lam, status, clear, start_aborted, stream);
 }
 
 // Backward: G_loc [U][128][128] and Lambda [U][128] of U segments of N tokens (whole chunks) from o, f and dy.
 cudaError_t launch_tc_state_bwd(const void *o, const void *f, const void *dy, uint64_t U, int N, float *G_loc,
-                                float *lam, StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream)
+                                float *lam, bool gate_enc, StatusBlock *status, bool clear, int start_aborted,
+                                cudaStream_t stream)
 {
-    return launch_state<true>(o, f, dy, U, N, N / kC, G_loc, lam, status, clear, start_aborted, stream);
+    if (gate_enc) return launch_state<true, true>(o, f, dy, U, N, N / kC, G_loc, lam, status, clear, start_aborted, stream);
+    return launch_state<true, false>(o, f, dy, U, N, N / kC, G_loc, lam, status, clear, start_aborted, stream);
 }
 
 }  // namespace hgrn2

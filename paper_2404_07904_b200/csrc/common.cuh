@@ -12,6 +12,10 @@ namespace hgrn2 {
 // Smallest forget-gate value the chunked kernels distinguish from zero: below it the
 // in-chunk cumulative decay is formed as if f were this value.
 constexpr float kFMin = 7.888609052210118e-31f;   // 2^-100
+// d_f divides the decay gradient (a sum that cancels down to ~f times its terms) by f.  With the gated entry
+// points' encoded gate, f is whatever the sigmoid gave, down to exactly 0; the divisor is kept above 2^-20 there:
+// below it the quotient would be the sum's rounding noise times up to 2^100.
+constexpr float kFDivMinK = 9.5367431640625e-7f;  // 2^-20
 
 // Layout of the 256-byte status block at the start of every workspace.
 struct StatusBlock {
@@ -61,6 +65,7 @@ struct SeqArgs {
     float *totals = nullptr;      // tensor-core path: per-chunk decay totals inside the saved data (set by its launchers)
     bool clear_status = false;    // tensor-core path: the first kernel of the call zeroes the status word itself
     int start_aborted = 0;        // tensor-core path, debugging: every CTA starts as if its first wait had run out
+    bool gate_enc = false;         // the f tensor holds the signed gate encoding (gated entry points)
     const int *cu = nullptr;      // packed batch: device array of B + 1 row offsets (B = sequences, N = total rows per head)
     cudaStream_t stream;
 };
@@ -109,10 +114,11 @@ struct SegPlan {
 SegPlan     tc_seg_plan(uint64_t U, int N, int NC);
 SeqArgs     tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n);
 
-cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam,
+cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam, bool gate_enc,
                                 StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream);
 cudaError_t launch_tc_state_bwd(const void *o, const void *f, const void *dy, uint64_t U, int N, float *G_loc,
-                                float *lam, StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream);
+                                float *lam, bool gate_enc, StatusBlock *status, bool clear, int start_aborted,
+                                cudaStream_t stream);
 cudaError_t launch_step(const StepArgs &a);
 bool        step_multi_supported(int dk, int dv);
 cudaError_t launch_step_multi(const StepArgs &a);

@@ -55,6 +55,16 @@ constexpr size_t kSavedTotalsBytes = 2 * kD * sizeof(float);
 #define PT_DUMP(st, base, n, cond)
 #endif
 
+// Signed gate encoding (kEnc): bits of one bf16 value in the low half of w -> f and k = 1 - f.  Sign clear: the
+// magnitude is f; sign set: the magnitude is k (so the neutral token f = 1, k = 0 is 0x8000).
+__device__ __forceinline__ void gate_decode(uint32_t w, float &f, float &k)
+{
+    const float m = __uint_as_float((w & 0x7FFFu) << 16);
+    const bool is_k = (w & 0x8000u) != 0u;
+    f = is_k ? 1.0f - m : m;
+    k = is_k ? m : 1.0f - m;
+}
+
 __device__ __forceinline__ float rcp_fast(float x)
 {
     float r;
@@ -81,8 +91,10 @@ __device__ __forceinline__ uint4 pack8(const uint32_t *r)
 // load behind the previous row's stores).  Pm (product over rows 0..31) and E (product over rows
 // 32..63) of the chunk are left in pm[128] and ee[128] (shared memory) and / or pm_g[128], ee_g[128]
 // (global memory); either pair may be null.  Rows at or beyond n_valid are the neutral token
-// f = 1, o = 0.
-template <bool kFull, bool kUp, uint32_t kQSlabStride, uint32_t kFSlabStride>
+// f = 1, o = 0.  kEnc: the gate tile holds the SMALLER of f and k = 1 - f, with the sign bit set when it is k
+// (gate_decode below).  The gated entry points hand the kernels that: bf16 then resolves the gate to 2^-9 of
+// min(f, 1 - f) at both ends of [0, 1], whereas a bf16 f close to 1 would distort every decay product.
+template <bool kFull, bool kUp, uint32_t kQSlabStride, uint32_t kFSlabStride, bool kEnc>
 __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, float *tot, float *tot_g, int n_valid,
                                                int p)
 {
@@ -120,8 +132,15 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
         for (int j = 0; j < 8; ++j) {
             const int r = row_of(8 * b + j);
             const uint32_t off = xo[r & 7] + r * 128;
-            if (!kFull && r >= n_valid) { fw[j] = 0x3F803F80u; qw[j] = 0u; }
-            const float f0 = bf16_lo(fw[j]), f1 = bf16_hi(fw[j]);
+            if (!kFull && r >= n_valid) { fw[j] = kEnc ? 0x80008000u : 0x3F803F80u; qw[j] = 0u; }
+            float f0, f1, k0 = 0.f, k1 = 0.f;
+            if (kEnc) {
+                gate_decode(fw[j], f0, k0);
+                gate_decode(fw[j] >> 16, f1, k1);
+            } else {
+                f0 = bf16_lo(fw[j]);
+                f1 = bf16_hi(fw[j]);
+            }
             if (kUp) { a0 *= f0; a1 *= f1; }
             const float m0 = fmaxf(a0, kProdFloor), m1 = fmaxf(a1, kProdFloor);
             const float i0 = rcp_fast(m0), i1 = rcp_fast(m1);
@@ -132,7 +151,8 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
             // (resp. fused multiply-add for k = 1 - f) produces the operand pair
             const uint32_t sqp = pack_bf16(sq0, sq1), skp = pack_bf16(sk0, sk1);
             *reinterpret_cast<uint32_t *>(qbuf + off) = mul_bf16x2(qw[j], sqp);
-            *reinterpret_cast<uint32_t *>(fbuf + off) = fma_bf16x2(fw[j], skp ^ 0x80008000u, skp);
+            *reinterpret_cast<uint32_t *>(fbuf + off) = kEnc ? mul_bf16x2(pack_bf16(k0, k1), skp)
+                                                             : fma_bf16x2(fw[j], skp ^ 0x80008000u, skp);
         }
     }
     // the products only shrink along the walk, so the last one tells whether any row met the floor
@@ -142,12 +162,12 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
 }
 
 // kQSlabStride, kFSlabStride: distance in bytes between the two 64-column slabs of the q tile and of the f tile.
-template <bool kFull, uint32_t kQSlabStride = kSlab, uint32_t kFSlabStride = kSlab>
+template <bool kFull, bool kEnc, uint32_t kQSlabStride = kSlab, uint32_t kFSlabStride = kSlab>
 __device__ __forceinline__ void transform_stream(uint8_t *qbuf, uint8_t *fbuf, float *pm, float *ee, float *pm_g,
                                                  float *ee_g, int n_valid, int tid)
 {
-    if (tid >> 6) transform_half<kFull, true, kQSlabStride, kFSlabStride>(qbuf, fbuf, ee, ee_g, n_valid, tid & 63);
-    else          transform_half<kFull, false, kQSlabStride, kFSlabStride>(qbuf, fbuf, pm, pm_g, n_valid, tid & 63);
+    if (tid >> 6) transform_half<kFull, true, kQSlabStride, kFSlabStride, kEnc>(qbuf, fbuf, ee, ee_g, n_valid, tid & 63);
+    else          transform_half<kFull, false, kQSlabStride, kFSlabStride, kEnc>(qbuf, fbuf, pm, pm_g, n_valid, tid & 63);
 }
 
 // Causal mask + bf16 of 32 columns (32 * half ...) of one 64 x 64 fp32 accumulator in the M = 64

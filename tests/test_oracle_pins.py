@@ -325,3 +325,38 @@ def test_packed_batch_equals_the_same_sequences_as_an_ordinary_batch():
     cu2 = np.array([0, 0, N])
     _, SN2 = ref.hgrn2_fwd_varlen(pack(o)[:, :N], pack(f)[:, :N], pack(i)[:, :N], cu2, S0[:2])
     np.testing.assert_array_equal(SN2[0], S0[0])
+
+
+def test_gated_wrappers_against_finite_differences():
+    # the gate activations of Eq. 1 / Eq. 2 in front of the recurrence: gradients with respect to the three
+    # pre-activations and to the lower bound beta against central differences of L = <dy, y> + <dSN, S_N>
+    rng = np.random.default_rng(17)
+    B, H, N, dk, dv = 2, 2, 5, 3, 2
+    zo = rng.standard_normal((B, H, N, dk)); zf = rng.standard_normal((B, H, N, dk))
+    zi = rng.standard_normal((B, H, N, dv)); beta = rng.uniform(0.0, 0.9, (H, dk))
+    S0 = rng.standard_normal((B, H, dk, dv)); dy = rng.standard_normal((B, H, N, dv))
+    dSN = rng.standard_normal((B, H, dk, dv))
+
+    def loss(zo_, zf_, zi_, beta_):
+        y, SN = ref.hgrn2_fwd_gated(zo_, zf_, zi_, beta_, S0)
+        return float((dy * y).sum() + (dSN * SN).sum())
+
+    got = ref.hgrn2_bwd_gated(zo, zf, zi, beta, S0, dy, dSN)
+    args = [zo, zf, zi, beta]
+    h = 1e-6
+    for which in range(4):
+        x = args[which]
+        num = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            xp = x.copy(); xp[idx] += h
+            xm = x.copy(); xm[idx] -= h
+            ap = list(args); ap[which] = xp
+            am = list(args); am[which] = xm
+            num[idx] = (loss(*ap) - loss(*am)) / (2 * h)
+        assert np.abs(num - got[which]).max() <= 1e-6 * max(1.0, np.abs(num).max()), which
+    # the activations themselves: sigmoid(0) = 1/2, silu(0) = 0, f = beta where the sigmoid vanishes
+    o, f, i = ref.gates(np.zeros((1, 1, 1, 2)), np.full((1, 1, 1, 2), -700.0), np.zeros((1, 1, 1, 2)), np.array([[0.25, 0.5]]))
+    np.testing.assert_allclose(o, 0.5); np.testing.assert_allclose(i, 0.0)
+    np.testing.assert_allclose(f[0, 0, 0], [0.25, 0.5])
