@@ -321,7 +321,47 @@ def run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf):
         del o, f, i, dy, saved, ws, y, d_o, d_f, d_i
         torch.cuda.empty_cache()
     out.append(run_packed_mix(binding, W, dev, timed, peaks, bf))
+    out.append(run_gated(binding, W, dev, timed, peaks, bf))
     return out
+
+
+def run_gated(binding, W, dev, timed, peaks, bf):
+    """lm_2048 through the gated entry points: pre-activations in, gradients of the pre-activations and of the lower
+    bound out (Eq. 1 / Eq. 2 in front of the recurrence).  Algorithmic bytes: the same eleven tensor passes."""
+    import torch
+    w = W.CONFIGS["lm_2048"]
+    rng = np.random.default_rng(11)
+    shape = (w.B, w.H, w.N, w.dk)
+    z = {k: torch.from_numpy(rng.standard_normal(shape, dtype=np.float32)).to(dev).to(bf) for k in ("zo", "zf", "zi", "dy")}
+    beta = torch.full((w.H, w.dk), 0.9, dtype=torch.float32, device=dev)
+    y, _, saved, ws, _ = binding.hgrn2_fwd_gated(z["zo"], z["zf"], z["zi"], beta, None, want_final_state=False)
+    outs = [torch.empty_like(z["zo"]) for _ in range(3)]
+    d_beta = torch.empty_like(beta)
+
+    def fwd():
+        binding.hgrn2_fwd_gated(z["zo"], z["zf"], z["zi"], beta, None, y=y, saved=saved, ws=ws, want_final_state=False)
+
+    def bwd():
+        binding.hgrn2_bwd_gated(z["zo"], z["zf"], z["zi"], beta, None, z["dy"], None, saved, d_zo=outs[0], d_zf=outs[1],
+                                d_zi=outs[2], d_beta=d_beta, ws=ws, want_dS0=False)
+
+    def step():
+        fwd(); bwd()
+
+    for _ in range(3):
+        step()
+    n = 20
+    ms = timed(step, n) / n
+    ms_f = timed(fwd, n) / n
+    ms_b = timed(bwd, n) / n
+    torch.cuda.synchronize()
+    assert binding.hgrn2_poll(ws) == 0
+    ab = train_bytes(w)
+    t_hbm = (ab["fwd"] + ab["bwd"]) / (peaks["hbm_gbs"] * 1e9)
+    return {"workload": "lm_2048_gated", "B": w.B, "H": w.H, "N": w.N, "beta": 0.9, "ms_per_step": ms, "fwd_ms": ms_f,
+            "bwd_ms": ms_b, "tokens_per_s": w.tokens / (ms * 1e-3), "frac_of_hbm_roofline": t_hbm * 1e3 / ms,
+            "exact_path_units": binding.exact_path_units(ws),
+            "note": "tensor-core path: element-wise gate kernels in front (3 tensors in, 3 out) and behind (6 in, 3 out)"}
 
 
 # A ragged batch as a long-context fine-tuning step would see it: 24 sequences between 256 and 4096 tokens

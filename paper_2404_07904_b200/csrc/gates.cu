@@ -25,6 +25,8 @@ constexpr int kGD = 128;                 // the tensor-core path: d_k = d_v = 12
 
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+// sigmoid with the fast exponential and reciprocal (a few ulp: far inside what the bf16 results keep)
+__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
 __device__ __forceinline__ uint32_t bf_pack(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -47,11 +49,11 @@ gate_fwd_kernel(const uint4 *__restrict__ zo, const uint4 *__restrict__ zf, cons
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float z0 = bf_lo(cw[j]), z1 = bf_hi(cw[j]);
-            ow[j] = bf_pack(alu::sigmoid_f(bf_lo(aw[j])), alu::sigmoid_f(bf_hi(aw[j])));
-            const float k0 = (1.0f - bh[2 * j]) * (1.0f - alu::sigmoid_f(bf_lo(bw[j])));
-            const float k1 = (1.0f - bh[2 * j + 1]) * (1.0f - alu::sigmoid_f(bf_hi(bw[j])));
+            ow[j] = bf_pack(sigmoid_fast(bf_lo(aw[j])), sigmoid_fast(bf_hi(aw[j])));
+            const float k0 = (1.0f - bh[2 * j]) * (1.0f - sigmoid_fast(bf_lo(bw[j])));
+            const float k1 = (1.0f - bh[2 * j + 1]) * (1.0f - sigmoid_fast(bf_hi(bw[j])));
             kw[j] = bf_pack(k0 <= 0.5f ? -k0 : 1.0f - k0, k1 <= 0.5f ? -k1 : 1.0f - k1);   // the smaller of f and k; negative = k
-            iw[j] = bf_pack(z0 * alu::sigmoid_f(z0), z1 * alu::sigmoid_f(z1));
+            iw[j] = bf_pack(z0 * sigmoid_fast(z0), z1 * sigmoid_fast(z1));
         }
         o[x] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
         k[x] = make_uint4(kw[0], kw[1], kw[2], kw[3]);
@@ -90,7 +92,7 @@ gate_bwd_kernel(const uint4 *__restrict__ zo, const uint4 *__restrict__ zf, cons
                 const float ziv = e ? bf_hi(cw[j]) : bf_lo(cw[j]);
                 const float dov = e ? bf_hi(dao[j]) : bf_lo(dao[j]), dfv = e ? bf_hi(dbf[j]) : bf_lo(dbf[j]);
                 const float div = e ? bf_hi(dci[j]) : bf_lo(dci[j]);
-                const float so = alu::sigmoid_f(zov), g = alu::sigmoid_f(zfv), si = alu::sigmoid_f(ziv);
+                const float so = sigmoid_fast(zov), g = sigmoid_fast(zfv), si = sigmoid_fast(ziv);
                 res[e] = dov * so * (1.0f - so);
                 res[2 + e] = dfv * (1.0f - bh[2 * j + e]) * g * (1.0f - g);
                 res[4 + e] = div * si * (1.0f + ziv * (1.0f - si));
