@@ -266,6 +266,26 @@ def run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks,
                                  "tokens_per_s": world * wd.B * TM / (ms_l * 1e-3),
                                  "achieved_GBps": mb / (ms_l * 1e-3) / 1e9,
                                  "algorithmic_bytes_per_launch": mb}
+    # ---- longer bursts: hgrn2_step_multi against the prefill kernel used as a T-token step (hgrn2_fwd, saved = NULL)
+    alts = []
+    for TT in (8, 32, 64):
+        if T < TT:
+            continue
+        seq = {k: gates[k][:TT].permute(1, 2, 0, 3).contiguous() for k in gates}
+        yt = torch.empty((wd.B, wd.H, TT, wd.dv), dtype=bf, device=dev)
+        S2 = torch.empty_like(S)
+        desc_t = binding.make_desc(wd.B, wd.H, TT, wd.dk, wd.dv, binding.HGRN2_BF16)
+        ws_t = binding.alloc_workspace(desc_t, dev)
+        f_multi = lambda: binding.hgrn2_step_multi(seq["o"], seq["f"], seq["i"], S, y=yt)
+        f_fwd = lambda: binding.hgrn2_fwd(seq["o"], seq["f"], seq["i"], S, y=yt, SN=S2, saved=None, ws=ws_t,
+                                          save_for_backward=False)
+        for fn in (f_multi, f_fwd):
+            fn()
+        nb = 5
+        t_m = max_over_ranks(timed(f_multi, nb)) / nb
+        t_f = max_over_ranks(timed(f_fwd, nb)) / nb
+        alts.append({"tokens_per_launch": TT, "step_multi_us": t_m * 1e3, "fwd_as_step_us": t_f * 1e3})
+    decode["multi_token_alternatives"] = alts
     if args.only == "decode" and rank == 0:
         print(json.dumps({"only": "decode", "decode": decode}), flush=True)
     return decode
@@ -538,6 +558,11 @@ def run_cuda(args):
         return e0.elapsed_time(e1)
 
     K, Wm = args.steps, max(args.warmup, 3)
+    if args.only == "others":
+        others = run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf)
+        if rank == 0:
+            print(json.dumps({"only": "others", "other_workloads": others}), flush=True)
+        return 0
     if args.only == "decode":
         run_decode(args, binding, W, dev, rank, world, timed, max_over_ranks, peaks, peak_kind, bf)
         return 0
@@ -710,7 +735,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference", "launch-check"])
     ap.add_argument("--min-seconds", type=float, default=2.0,
                     help="repeat the timed K-step batch until this much device time has been spent (median batch reported)")
-    ap.add_argument("--only", default="all", choices=["all", "train", "decode"],
+    ap.add_argument("--only", default="all", choices=["all", "train", "decode", "others"],
                     help="restrict the run to one part (for profiling); the JSON line is printed for 'all' only")
     ap.add_argument("--decode-steps", type=int, default=0, help="decode calls to time (0 = the workload's 512)")
     ap.add_argument("--skip-others", action="store_true", help="do not time the long-context and larger-layer workloads")
