@@ -185,6 +185,33 @@ hgrn2_status hgrn2_bwd_gated(const hgrn2_desc *desc, const void *zo, const void 
                              const void *saved, void *d_zo, void *d_zf, void *d_zi, float *d_beta,
                              float *dS0, void *ws, void *cuda_stream);
 
+/* Sequence (context) parallelism: a sequence cut into R consecutive spans, one per GPU.  Eq. 3 is linear in the
+ * state and the state has constant size (Section 1), so one exchange of d_k + d_k d_v floats per unit and rank is
+ * all the spans need of each other (the library itself never communicates; the caller all-gathers):
+ *   1. hgrn2_span_summary_fwd on the rank's own span: S_loc = the span's end state from a ZERO start state,
+ *      lam = the product of f over the span, per key dimension.  desc->N = tokens of the span.
+ *        f [B][H][N][dk], i [B][H][N][dv] in (desc->io); S_loc [B][H][dk][dv], lam [B][H][dk] float32 out
+ *   2. all-gather S_loc and lam into X_all [R][B][H][dk][dv], lam_all [R][B][H][dk] (the caller's collective)
+ *   3. hgrn2_span_compose(desc, 0, r, 0, X_all, lam_all, S0, S_start): this rank's start state,
+ *        S <- Diag(lam[r']) S + X[r']  for r' = 0 .. r-1, from init = the sequence's S0 (NULL = zero);
+ *      with (0, R) it gives the sequence's final state
+ *   4. hgrn2_fwd on the span with S0 = S_start.
+ * Backward, mirrored: hgrn2_span_summary_bwd gives G_loc = the span's state gradient at its START from a zero
+ * gradient at its end (o, f [..][dk], dy [..][dv] in); after the all-gather
+ * hgrn2_span_compose(desc, r + 1, R, 1, G_all, lam_all, dSN, dS_end) folds r' = R-1 .. r+1 downwards from the
+ * sequence's dS_N (NULL = zero), and hgrn2_bwd runs on the span with S0 = S_start, dSN = dS_end; with (0, R, 1)
+ * the fold gives the sequence's dS_0.
+ * r0 <= r' < r1 selects the spans folded; reverse = 0 ascending, 1 descending; an empty range copies init (or
+ * writes zero).  ws: at least 256 bytes (status block).  Shapes and errors as for hgrn2_fwd; the summaries run on
+ * the tensor cores for bf16, dk = dv = 128 and N a multiple of 64, on plain fp32 loops otherwise. */
+hgrn2_status hgrn2_span_summary_fwd(const hgrn2_desc *desc, const void *f, const void *i, float *S_loc,
+                                    float *lam, void *ws, void *cuda_stream);
+hgrn2_status hgrn2_span_summary_bwd(const hgrn2_desc *desc, const void *o, const void *f, const void *dy,
+                                    float *G_loc, float *lam, void *ws, void *cuda_stream);
+hgrn2_status hgrn2_span_compose(const hgrn2_desc *desc, int32_t r0, int32_t r1, int32_t reverse,
+                                const float *X_all, const float *lam_all, const float *init, float *out,
+                                void *cuda_stream);
+
 /* Largest chunk-state scratch, in bytes, that hgrn2_bwd_static_scratch can serve. */
 #define HGRN2_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
 

@@ -29,7 +29,7 @@ EXPORTS = (
     "hgrn2_saved_bytes", "hgrn2_workspace_bytes", "hgrn2_fwd", "hgrn2_bwd", "hgrn2_step",
     "hgrn2_step_multi", "hgrn2_poll", "hgrn2_status_string", "hgrn2_chunk", "hgrn2_path", "hgrn2_bwd_static_scratch",
     "hgrn2_exact_path_units", "hgrn2_saved_bytes_varlen", "hgrn2_workspace_bytes_varlen", "hgrn2_fwd_varlen",
-    "hgrn2_bwd_varlen", "hgrn2_saved_bytes_gated", "hgrn2_workspace_bytes_gated", "hgrn2_fwd_gated", "hgrn2_bwd_gated",
+    "hgrn2_bwd_varlen", "hgrn2_span_summary_fwd", "hgrn2_span_summary_bwd", "hgrn2_span_compose", "hgrn2_saved_bytes_gated", "hgrn2_workspace_bytes_gated", "hgrn2_fwd_gated", "hgrn2_bwd_gated",
 )
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
@@ -86,6 +86,12 @@ def load() -> ctypes.CDLL:
     lib.hgrn2_fwd_varlen.argtypes = [dp] + [vp] * 10
     lib.hgrn2_bwd_varlen.restype = ctypes.c_int
     lib.hgrn2_bwd_varlen.argtypes = [dp] + [vp] * 14
+    lib.hgrn2_span_summary_fwd.restype = ctypes.c_int
+    lib.hgrn2_span_summary_fwd.argtypes = [dp] + [vp] * 6
+    lib.hgrn2_span_summary_bwd.restype = ctypes.c_int
+    lib.hgrn2_span_summary_bwd.argtypes = [dp] + [vp] * 7
+    lib.hgrn2_span_compose.restype = ctypes.c_int
+    lib.hgrn2_span_compose.argtypes = [dp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32] + [vp] * 5
     lib.hgrn2_saved_bytes_gated.restype = ctypes.c_size_t
     lib.hgrn2_saved_bytes_gated.argtypes = [dp]
     lib.hgrn2_workspace_bytes_gated.restype = ctypes.c_size_t
@@ -256,6 +262,43 @@ def hgrn2_bwd_varlen(o, f, i, cu_seqlens, S0, dy, dSN=None, saved=None, *, d_o=N
                                 _stream(stream))
     _check(code, "hgrn2_bwd_varlen")
     return d_o, d_f, d_i, dS0, ws
+
+
+def span_summary_fwd(f, i, *, ws=None, chunk=0, flags=0, stream=None):
+    """A span's end state from a zero start state and its total decay: (S_loc [B,H,dk,dv], lam [B,H,dk])."""
+    B, H, N, dk = f.shape
+    dv = i.shape[-1]
+    desc = make_desc(B, H, N, dk, dv, _io_code(f), chunk, flags)
+    S_loc = torch.empty((B, H, dk, dv), dtype=torch.float32, device=f.device)
+    lam = torch.empty((B, H, dk), dtype=torch.float32, device=f.device)
+    ws = torch.empty(256, dtype=torch.uint8, device=f.device) if ws is None else ws
+    _check(load().hgrn2_span_summary_fwd(ctypes.byref(desc), _ptr(f), _ptr(i), _ptr(S_loc), _ptr(lam), _ptr(ws),
+                                         _stream(stream)), "hgrn2_span_summary_fwd")
+    return S_loc, lam
+
+
+def span_summary_bwd(o, f, dy, *, ws=None, chunk=0, flags=0, stream=None):
+    """A span's state gradient at its start from a zero gradient at its end, and its total decay."""
+    B, H, N, dk = o.shape
+    dv = dy.shape[-1]
+    desc = make_desc(B, H, N, dk, dv, _io_code(o), chunk, flags)
+    G_loc = torch.empty((B, H, dk, dv), dtype=torch.float32, device=o.device)
+    lam = torch.empty((B, H, dk), dtype=torch.float32, device=o.device)
+    ws = torch.empty(256, dtype=torch.uint8, device=o.device) if ws is None else ws
+    _check(load().hgrn2_span_summary_bwd(ctypes.byref(desc), _ptr(o), _ptr(f), _ptr(dy), _ptr(G_loc), _ptr(lam), _ptr(ws),
+                                         _stream(stream)), "hgrn2_span_summary_bwd")
+    return G_loc, lam
+
+
+def span_compose(X_all, lam_all, r0, r1, reverse=False, init=None, *, stream=None):
+    """Fold the spans r0 <= r < r1 (ascending, or descending when `reverse`) of X_all [R,B,H,dk,dv], lam_all [R,B,H,dk]
+    onto `init` (None = zero): S <- Diag(lam[r]) S + X[r].  Returns [B,H,dk,dv] float32."""
+    R, B, H, dk, dv = X_all.shape
+    desc = make_desc(B, H, 0, dk, dv, HGRN2_F32)
+    out = torch.empty((B, H, dk, dv), dtype=torch.float32, device=X_all.device)
+    _check(load().hgrn2_span_compose(ctypes.byref(desc), int(r0), int(r1), int(bool(reverse)), _ptr(X_all), _ptr(lam_all),
+                                     _ptr(init), _ptr(out), _stream(stream)), "hgrn2_span_compose")
+    return out
 
 
 def hgrn2_fwd_gated(zo, zf, zi, beta, S0=None, *, y=None, SN=None, saved=None, ws=None, want_final_state=True,

@@ -16,6 +16,11 @@ size_t      tc_saved_bytes(const hgrn2_desc *d, int C);
 size_t      tc_segment_scratch_bytes(const hgrn2_desc *d, int C);
 size_t      tc_exact_scratch_bytes(const hgrn2_desc *d);
 size_t      tc_saved_bytes_packed(const hgrn2_desc *d);
+// span summaries for sequence parallelism (span.cu)
+cudaError_t launch_span_summary(bool bwd, int io, const void *x, const void *f, const void *w, long long U, int N, int dk,
+                                int dv, float *out, float *lam, cudaStream_t stream);
+cudaError_t launch_span_compose(const float *X_all, const float *lam_all, const float *init, float *out, long long U,
+                                int dk, int dv, int r0, int r1, int reverse, cudaStream_t stream);
 // gate activations (gates.cu)
 int         gate_bwd_slices(long long U, int N);
 cudaError_t launch_gate_fwd(const SeqArgs &a, const float *beta, void *o_out, void *k_out, void *i_out);
@@ -438,6 +443,74 @@ hgrn2_status hgrn2_bwd_gated(const hgrn2_desc *desc, const void *zo, const void 
     if (launch_tc_bwd(k) != cudaSuccess) return HGRN2_ERR_CUDA;
     // d_o, d_f, d_i sit in the output buffers: chain rule through the activations, in place, and d_beta
     return launch_gate_bwd(a, beta, partial, d_beta) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+hgrn2_status hgrn2_span_summary_fwd(const hgrn2_desc *desc, const void *f, const void *i, float *S_loc, float *lam,
+                                    void *ws, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    const int C = resolve_chunk(desc);
+    if (C == 0) return HGRN2_ERR_UNSUPPORTED;
+    if (!ws) return HGRN2_ERR_WORKSPACE;
+    const long long U = (long long)desc->B * desc->H;
+    const bool empty = U * desc->N == 0;
+    const void *req[] = {ws, S_loc, lam, f, i};
+    const void *opt[] = {f, i};
+    hgrn2_status st = check_ptrs(req, U == 0 ? 1 : (empty ? 3 : 5), opt, 2);
+    if (st != HGRN2_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (U == 0) return cudaMemsetAsync(ws, 0, sizeof(StatusBlock), stream) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+    cudaError_t e;
+    if (use_tc(desc) && desc->N > 0 && desc->N % C == 0) {
+        e = launch_tc_state_fwd(f, i, (uint64_t)U, desc->N, S_loc, lam, false, static_cast<StatusBlock *>(ws), true,
+                                (desc->flags & HGRN2_FLAG_DEBUG_EXPIRE_WAITS) ? 1 : 0, stream);
+    } else {
+        if (cudaMemsetAsync(ws, 0, sizeof(StatusBlock), stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+        e = launch_span_summary(false, desc->io, nullptr, f, i, U, desc->N, desc->dk, desc->dv, S_loc, lam, stream);
+    }
+    return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+hgrn2_status hgrn2_span_summary_bwd(const hgrn2_desc *desc, const void *o, const void *f, const void *dy, float *G_loc,
+                                    float *lam, void *ws, void *cuda_stream)
+{
+    if (!desc_ok(desc)) return HGRN2_ERR_INVALID_ARG;
+    const int C = resolve_chunk(desc);
+    if (C == 0) return HGRN2_ERR_UNSUPPORTED;
+    if (!ws) return HGRN2_ERR_WORKSPACE;
+    const long long U = (long long)desc->B * desc->H;
+    const bool empty = U * desc->N == 0;
+    const void *req[] = {ws, G_loc, lam, o, f, dy};
+    const void *opt[] = {o, f, dy};
+    hgrn2_status st = check_ptrs(req, U == 0 ? 1 : (empty ? 3 : 6), opt, 3);
+    if (st != HGRN2_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (U == 0) return cudaMemsetAsync(ws, 0, sizeof(StatusBlock), stream) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+    cudaError_t e;
+    if (use_tc(desc) && desc->N > 0 && desc->N % C == 0) {
+        e = launch_tc_state_bwd(o, f, dy, (uint64_t)U, desc->N, G_loc, lam, false, static_cast<StatusBlock *>(ws), true,
+                                (desc->flags & HGRN2_FLAG_DEBUG_EXPIRE_WAITS) ? 1 : 0, stream);
+    } else {
+        if (cudaMemsetAsync(ws, 0, sizeof(StatusBlock), stream) != cudaSuccess) return HGRN2_ERR_CUDA;
+        e = launch_span_summary(true, desc->io, o, f, dy, U, desc->N, desc->dk, desc->dv, G_loc, lam, stream);
+    }
+    return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
+}
+
+hgrn2_status hgrn2_span_compose(const hgrn2_desc *desc, int32_t r0, int32_t r1, int32_t reverse, const float *X_all,
+                                const float *lam_all, const float *init, float *out, void *cuda_stream)
+{
+    if (!desc_ok(desc) || r0 < 0 || r1 < r0) return HGRN2_ERR_INVALID_ARG;
+    if (!dim_ok(desc->dk) || !dim_ok(desc->dv)) return HGRN2_ERR_UNSUPPORTED;
+    const long long U = (long long)desc->B * desc->H;
+    if (U == 0) return HGRN2_OK;
+    const void *req[] = {out, X_all, lam_all};
+    const void *opt[] = {init};
+    hgrn2_status st = check_ptrs(req, r1 > r0 ? 3 : 1, opt, 1);
+    if (st != HGRN2_OK) return st;
+    cudaError_t e = launch_span_compose(X_all, lam_all, init, out, U, desc->dk, desc->dv, r0, r1, reverse ? 1 : 0,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
 }
 
 hgrn2_status hgrn2_fwd_varlen(const hgrn2_desc *desc, const void *o, const void *f, const void *i,
