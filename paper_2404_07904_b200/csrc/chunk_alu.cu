@@ -65,7 +65,7 @@ template <typename T>
 cudaError_t launch_fwd_t(const SeqArgs &a)
 {
     const size_t smem = alu::fwd_smem_floats(a.dk, a.dv, a.C) * sizeof(float);
-    cudaError_t err = cudaFuncSetAttribute(alu_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(alu_fwd_kernel<T>), smem);
     if (err != cudaSuccess) return err;
     alu_fwd_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i), a.S0,
@@ -77,7 +77,7 @@ template <typename T>
 cudaError_t launch_bwd_t(const SeqArgs &a)
 {
     const size_t smem = alu::bwd_smem_floats(a.dk, a.dv, a.C) * sizeof(float);
-    cudaError_t err = cudaFuncSetAttribute(alu_bwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(alu_bwd_kernel<T>), smem);
     if (err != cudaSuccess) return err;
     alu_bwd_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i),

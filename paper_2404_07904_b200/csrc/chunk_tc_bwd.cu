@@ -839,7 +839,7 @@ static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
                          : (ragged ? tc_bwd_kernel<true, false, false>
                                    : (ex.o != nullptr && ex.G > 1 ? tc_bwd_kernel<false, true, false>
                                                                    : tc_bwd_kernel<false, false, false>));
-    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), kSmemBytes);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(
         mo, mf, mi, mg, ms, mor, mfr,

@@ -731,7 +731,7 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
                          : (ragged ? tc_fwd_kernel<true, false, false>
                                    : (ex.o != nullptr && ex.G > 1 ? tc_fwd_kernel<false, true, false>
                                                                    : tc_fwd_kernel<false, false, false>));
-    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), kSmemBytes);
     if (err != cudaSuccess) return err;
     float *totals = want_saved ? a.totals : nullptr;
     kernel<<<(unsigned)U, kThreads, kSmemBytes, a.stream>>>(mo, mf, mi, my, ms, S0, SN, totals, want_y,

@@ -250,8 +250,7 @@ cudaError_t launch_state(const void *o, const void *f, const void *w, uint64_t U
     CUtensorMap mo, mf, mw;
     if (!make_map(&mo, kBwd ? o : f, U, N, kC) || !make_map(&mf, f, U, N, kC) || !make_map(&mw, w, U, N, kC))
         return cudaErrorInvalidValue;
-    cudaError_t err = cudaFuncSetAttribute(tc_state_kernel<kBwd, kEnc>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)G::kSmemBytes);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(tc_state_kernel<kBwd, kEnc>), G::kSmemBytes);
     if (err != cudaSuccess) return err;
     tc_state_kernel<kBwd, kEnc><<<(unsigned)U, kThreads, G::kSmemBytes, stream>>>(mo, mf, mw, out, lam, NC, status,
                                                                              clear ? 1 : 0, start_aborted);

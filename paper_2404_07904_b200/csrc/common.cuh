@@ -5,6 +5,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+#include <vector>
+
 #include "hgrn2.h"
 
 namespace hgrn2 {
@@ -43,6 +46,29 @@ template <> __device__ __forceinline__ void store_f<__nv_bfloat16>(__nv_bfloat16
 __device__ __forceinline__ void report_error(StatusBlock *sb, int code, int where)
 {
     if (sb != nullptr && atomicCAS(&sb->code, 0, code) == 0) sb->where = where;
+}
+
+// A kernel's dynamic shared-memory limit has to be raised once per device before its first launch with more than
+// 48 KB; later calls find the (kernel, device) pair here and skip the runtime call.
+inline cudaError_t ensure_dynamic_smem(const void *kernel, size_t bytes)
+{
+    struct Entry { const void *kernel; int device; size_t bytes; };
+    static std::mutex mu;
+    static std::vector<Entry> done;
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    std::lock_guard<std::mutex> lock(mu);
+    for (Entry &e : done)
+        if (e.kernel == kernel && e.device == dev) {
+            if (e.bytes >= bytes) return cudaSuccess;
+            err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+            if (err == cudaSuccess) e.bytes = bytes;
+            return err;
+        }
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (err == cudaSuccess) done.push_back(Entry{kernel, dev, bytes});
+    return err;
 }
 
 // ---- internal launchers (defined in the .cu files, called from api.cu) ----------------------

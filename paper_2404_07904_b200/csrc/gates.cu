@@ -166,7 +166,7 @@ template <typename T>
 cudaError_t alu_gated_fwd_t(const SeqArgs &a, const float *beta)
 {
     const size_t smem = alu::fwd_smem_floats(a.dk, a.dv, a.C) * sizeof(float);
-    cudaError_t err = cudaFuncSetAttribute(alu_fwd_gated_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(alu_fwd_gated_kernel<T>), smem);
     if (err != cudaSuccess) return err;
     alu_fwd_gated_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i), beta, a.S0,
@@ -178,7 +178,7 @@ template <typename T>
 cudaError_t alu_gated_bwd_t(const SeqArgs &a, const float *beta, float *partial)
 {
     const size_t smem = alu::bwd_smem_floats(a.dk, a.dv, a.C) * sizeof(float);
-    cudaError_t err = cudaFuncSetAttribute(alu_bwd_gated_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(alu_bwd_gated_kernel<T>), smem);
     if (err != cudaSuccess) return err;
     alu_bwd_gated_kernel<T><<<(unsigned)((long long)a.B * a.H), kAluThreads, smem, a.stream>>>(
         static_cast<const T *>(a.o), static_cast<const T *>(a.f), static_cast<const T *>(a.i), beta,

@@ -85,7 +85,7 @@ cudaError_t launch_summary_t(const void *x, const void *f, const void *w, long l
                              float *lam, cudaStream_t stream)
 {
     const size_t smem = ((size_t)dk * dv + 2 * dk + dv) * sizeof(float);
-    cudaError_t err = cudaFuncSetAttribute(span_summary_kernel<T, kBwd>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(span_summary_kernel<T, kBwd>), smem);
     if (err != cudaSuccess) return err;
     span_summary_kernel<T, kBwd><<<(unsigned)U, 256, smem, stream>>>(static_cast<const T *>(x), static_cast<const T *>(f),
                                                                    static_cast<const T *>(w), out, lam, N, dk, dv);
