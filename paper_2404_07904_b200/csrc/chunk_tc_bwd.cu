@@ -357,6 +357,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             PT_MARK(0)
             // a total on the floor: the decay across that half chunk is more than the rescaled operands can carry
             if (fminf(pm_c, ee_c) <= kProdFloor) ctl->exact_flag = 1;
+            const float pm_old = pm_prev, ee_old = ee_c;
             const float factor = pm_prev * ee_c;
             pm_prev = pm_c;
             if (it + 1 < NC) {
@@ -390,8 +391,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                     tmem_ld32(tmem + lane_base + kColDS + 32 * part, r);
                     tmem_wait_ld();
                 }
+                if (factor >= kFactorSafe) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 2) scale2(r[j], r[j + 1], factor);
+                    for (int j = 0; j < 32; j += 2) scale2(r[j], r[j + 1], factor);
+                } else {                         // see the forward kernel: the two decays one after the other
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * pm_old * ee_old);
+                }
                 tmem_st32(tmem + lane_base + kColDS + 32 * part, r);
 #pragma unroll
                 for (int j = 0; j < 4; ++j)

@@ -209,6 +209,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_wait(&ctl->t_done[c % kStages], (c / kStages) & 1, abort_flag);
             PT_MARK(0)
             const float pm_c = pm[(c & 3) * 128 + krow];
+            const float e_old = e_prev;
             const float factor = e_prev * pm_c;
             e_prev = ee[(c & 3) * 128 + krow];
             // a total on the floor: the decay across that half chunk is more than the rescaled operands can carry
@@ -235,8 +236,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 tmem_ld32(tmem + lane_base + kColS + v0 + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
                 tmem_wait_ld();
             }
+            // Each of the two decays is above the floor, but their product can leave fp32's range although the
+            // accumulator, which sits in the previous chunk's frame, is as large as that decay is small: then the
+            // two are applied one after the other (key dimensions whose decay over those 64 tokens is below
+            // 2^-120: rare, so a branch around the single multiply).
+            if (factor >= kFactorSafe) {
 #pragma unroll
-            for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
+                for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * factor);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * e_old * pm_c);
+            }
             tmem_st32(tmem + lane_base + kColS + v0, *reinterpret_cast<uint32_t(*)[32]>(r));
             tmem_st32(tmem + lane_base + kColS + v0 + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
             uint4 sw[8];

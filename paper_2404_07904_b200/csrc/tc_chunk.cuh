@@ -34,6 +34,7 @@ constexpr uint32_t kTile = 2 * kSlab;           // one [64][128] bf16 tile
 constexpr uint32_t kStateSlab = kD * 128;       // bytes of one slab of a [128][128] bf16 state copy
 constexpr uint32_t kStateTile = 2 * kStateSlab;
 constexpr float kProdFloor = 7.888609052210118e-31f;   // 2^-100
+constexpr float kFactorSafe = 7.52316384526264e-37f;    // 2^-120: below it the product of two decay totals is applied in two steps
 constexpr uint32_t kTmemCols = 512;
 constexpr int kTransformThreads = 128;          // threads that run transform_stream together
 // Saved-for-backward buffer of the tensor-core path, per (unit, chunk): the bf16 state S' in the mid

@@ -135,3 +135,15 @@ def test_hard_forget_units_in_full_wave_and_left_over_part():
     want = G.oracle_fwd_bwd(inp, [(0, 7), (0, 8), (0, H - 2), (0, H - 1)])
     for (b, h), wu in want.items():
         G.assert_close({k: got[k][b:b + 1, h:h + 1] for k in wu}, wu, TOL, f"unit {(b, h)}")
+
+
+def test_decay_within_range_per_half_chunk_but_not_per_chunk():
+    # f == 0.2 in a few key dimensions: 0.2^32 = 2^-74 per half chunk stays inside the operands' range (no exact path),
+    # but the product of two such totals, 2^-149, is below fp32's range: the state rescaling between two chunks must
+    # apply them one after the other (the accumulator it scales is as large as the first of them is small)
+    w, inp = _base(B=1, H=2, N=300, seed=15)
+    inp["f"][:, :, :, [0, 17, 64, 127]] = W.round_to_bf16(np.float32(0.2))
+    for use_saved in (True, False):
+        got, n_fwd, n_bwd = _run(inp, use_saved)
+        assert n_fwd == 0 and n_bwd == 0
+        G.assert_close(got, G.oracle_fwd_bwd(inp), TOL, "f == 0.2 in four key dimensions")
