@@ -42,3 +42,31 @@ def test_random_case_against_the_oracle(seed):
     units = sorted({(0, 0), (B - 1, H - 1), (B // 2, H // 2)})
     for (b, h), want in G.oracle_fwd_bwd(inp, units).items():
         G.assert_close({k: got[k][b:b + 1, h:h + 1] for k in want}, want, 2e-2, f"{what}, unit {(b, h)}")
+
+
+@pytest.mark.parametrize("seed", range(200, 206))
+def test_random_packed_batch_against_the_oracle(seed):
+    from tests import test_gpu_varlen as TV
+    rng = np.random.default_rng(seed)
+    lengths = [int(rng.choice([0, 1, 30, 64, 65, 128, 200, 300, 700])) for _ in range(int(rng.integers(1, 6)))]
+    if sum(lengths) == 0:
+        lengths.append(70)
+    inp = TV._packed_inputs(lengths, H=int(rng.integers(1, 4)), d=128, io="bf16", seed=seed,
+                            gamma=float(rng.choice([0.0, 0.3, 0.9, 0.99])), with_states=bool(rng.integers(0, 2)),
+                            pad_rows=int(rng.integers(0, 20)))
+    T = inp["o"].shape[1]
+    got, _ = TV._run_gpu(inp, "bf16", use_saved=bool(rng.integers(0, 2)))
+    G.assert_close(TV._mask_rows(got, inp["cu"], T), TV._mask_rows(TV._oracle(inp), inp["cu"], T), 2e-2,
+                   f"seed {seed}: lengths {lengths}")
+
+
+@pytest.mark.parametrize("seed", range(300, 306))
+def test_random_gated_case_against_the_oracle(seed):
+    from tests import test_gpu_gated as TG
+    rng = np.random.default_rng(seed)
+    B, H = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    N = int(rng.choice([5, 64, 129, 300, 511, 1024]))
+    inp = TG._inputs(B, H, N, 128, "bf16", seed=seed, beta_lo=0.0, beta_hi=float(rng.choice([0.0, 0.9, 0.999])),
+                     zf_shift=float(rng.choice([0.0, -2.0, 2.0])), states=bool(rng.integers(0, 2)))
+    got, _ = TG._run(inp, "bf16", use_saved=bool(rng.integers(0, 2)))
+    G.assert_close(got, TG._oracle(inp), 2e-2, f"seed {seed}: B{B} H{H} N{N}")
