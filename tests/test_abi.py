@@ -106,6 +106,44 @@ def test_host_side_argument_errors_launch_nothing(lib):
     assert lib.hgrn2_poll(None) == 1
 
 
+def test_new_entry_points_reject_bad_arguments_on_the_host(lib):
+    vp = ctypes.c_void_p
+    ok = 0x1000  # never dereferenced
+    d = binding.make_desc(2, 1, 100, 64, 64, binding.HGRN2_F32)
+    # packed batches: args o f i cu S0 y SN saved ws stream
+    call = lambda a: lib.hgrn2_fwd_varlen(ctypes.byref(d), *[vp(p) for p in a])
+    assert call([ok, ok, ok, 0, 0, ok, 0, 0, ok, 0]) == 1                      # no offsets
+    assert call([ok, ok, ok, ok + 2, 0, ok, 0, 0, ok, 0]) == 3                 # misaligned offsets
+    assert call([ok, ok, ok, ok, 0, ok, 0, 0, 0, 0]) == 4                      # no workspace
+    assert call([ok, 0, ok, ok, 0, ok, 0, 0, ok, 0]) == 1                      # NULL f
+    bwd = [ok, ok, ok, ok, 0, ok, 0, 0, ok, ok, ok, 0, ok, 0]
+    a = list(bwd); a[3] = 0
+    assert lib.hgrn2_bwd_varlen(ctypes.byref(d), *[vp(p) for p in a]) == 1
+    a = list(bwd); a[9] = 0
+    assert lib.hgrn2_bwd_varlen(ctypes.byref(d), *[vp(p) for p in a]) == 1     # NULL d_f
+    assert lib.hgrn2_saved_bytes_varlen(ctypes.byref(d)) == 1 * (100 // 64 + 2 + 1) * 64 * 64 * 4
+    assert lib.hgrn2_workspace_bytes_varlen(ctypes.byref(binding.make_desc(2, 1, 100, 48, 64, 0))) == 0
+    # gated: args zo zf zi beta S0 y SN saved ws stream
+    call = lambda a: lib.hgrn2_fwd_gated(ctypes.byref(d), *[vp(p) for p in a])
+    assert call([ok, ok, ok, 0, 0, ok, 0, 0, ok, 0]) == 1                      # no beta
+    assert call([ok, ok, ok, ok + 4, 0, ok, 0, 0, ok, 0]) == 3                 # misaligned beta
+    assert call([ok, ok, ok, ok, 0, ok, 0, 0, 0, 0]) == 4                      # no workspace
+    gb = [ok, ok, ok, ok, 0, ok, 0, 0, ok, ok, ok, 0, 0, ok, 0]
+    a = list(gb); a[10] = 0
+    assert lib.hgrn2_bwd_gated(ctypes.byref(d), *[vp(p) for p in a]) == 1      # NULL d_zi
+    tc = binding.make_desc(2, 3, 256, 128, 128, binding.HGRN2_BF16)
+    assert lib.hgrn2_saved_bytes_gated(ctypes.byref(tc)) == 3 * 2 * 3 * 256 * 128 * 2 + binding.saved_bytes(tc)
+    assert lib.hgrn2_saved_bytes_gated(ctypes.byref(d)) == binding.saved_bytes(d)
+    # spans: summary args f i S_loc lam ws stream; compose args r0 r1 reverse X lam init out stream
+    assert lib.hgrn2_span_summary_fwd(ctypes.byref(d), *[vp(p) for p in [ok, ok, 0, ok, ok, 0]]) == 1
+    assert lib.hgrn2_span_summary_fwd(ctypes.byref(d), *[vp(p) for p in [ok, ok, ok, ok, 0, 0]]) == 4
+    assert lib.hgrn2_span_summary_bwd(ctypes.byref(d), *[vp(p) for p in [ok, ok + 8, ok, ok, ok, ok, 0]]) == 3
+    assert lib.hgrn2_span_compose(ctypes.byref(d), 2, 1, 0, vp(ok), vp(ok), None, vp(ok), None) == 1    # r1 < r0
+    assert lib.hgrn2_span_compose(ctypes.byref(d), 0, 2, 0, vp(ok), vp(ok), None, None, None) == 1      # no output
+    assert lib.hgrn2_span_compose(ctypes.byref(d), 0, 2, 0, None, vp(ok), None, vp(ok), None) == 1      # no summaries
+    assert lib.hgrn2_exact_path_units(None) == -1
+
+
 def test_binding_refuses_cpu_tensors(lib):
     import torch
     o = torch.zeros(1, 1, 4, 64)
