@@ -110,28 +110,32 @@ constexpr int kExactC = 32;       // chunk length of the exact fp32 routines at 
 static_assert(alu::bwd_smem_floats(kD, kD, kExactC) * sizeof(float) <= kSmemBytes, "exact path fits the CTA's shared memory");
 
 // d_o and the nearly finished d_f of one thread: key dimension k, local times [32 * kUp, 32 * kUp + 32),
-// walked outwards from the middle of the chunk in blocks of eight.  Returns this half's sums of a and e.
+// walked outwards from the middle of the chunk in blocks of four rows (a short loop body: the role shares its
+// scheduler's instruction stream with four others).  Returns this half's sums of a and e.
 // do_g points at element (row 0 of the chunk, column k) of d_o in global memory.  oraw, fraw: the chunk's raw
-// o and f as plain [64][128] bf16 tiles (rows beyond the end of the sequence hold zeros, or in a packed batch the
-// next sequence's tokens: they are patched to the neutral f = 1, o = 0).  Qs and Ks are recomputed from them with the transform's own roundings, so the
-// operand stage does not have to be held until the outputs are done.
+// o and f as plain [64][128] bf16 tiles (rows beyond the end of the sequence hold zeros, or in a packed batch
+// the next sequence's tokens: they are patched to the neutral f = 1, o = 0).  Qs and Ks are recomputed from
+// them with the transform's own roundings, so the operand stage does not have to be held until the outputs
+// are done.  The role is bound by its instruction count: per element one reciprocal (1/f is the ratio of two
+// consecutive products), fused packed multiply-adds, and a single running sum.
 template <bool kUp, bool kRagged, bool kEnc>
 __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat16 *oraw, const __nv_bfloat16 *fraw,
                                            int k, __nv_bfloat16 *do_g, int n_valid, float &asum, float &esum)
 {
-    float cp = 1.f;                 // running product of f between the middle and the current row
-    float G = 0.f, H = 0.f;         // running sums of a and e over the rows visited so far
+    float cp = 1.f, ci = 1.f;       // running product of f between the middle and the current row, and its reciprocal
+    float W = 0.f;                  // running sum of a - e over the rows visited so far
+    float2 Gp = make_float2(0.f, 0.f);   // sum of a over the rows visited so far, even and odd rows apart
 #pragma unroll 1
-    for (int b = 0; b < 4; ++b) {
-        const int t0 = kUp ? 32 + 8 * b : 24 - 8 * b;          // lowest row of the block (a multiple of 8)
-        uint32_t x[8], y[8], z[8];
-        tmem_ld8(tmem_lane + kColDQ + t0, x);
-        tmem_ld8(tmem_lane + kColDKi + t0, y);
-        tmem_ld8(tmem_lane + kColDKx + t0, z);
-        uint32_t fw[8], qw[8];         // raw bf16 bits
-        float fv[8];
+    for (int b = 0; b < 8; ++b) {
+        const int t0 = kUp ? 32 + 4 * b : 28 - 4 * b;          // lowest row of the block (a multiple of 4)
+        uint32_t x[4], y[4], z[4];
+        tmem_ld4(tmem_lane + kColDQ + t0, x);
+        tmem_ld4(tmem_lane + kColDKi + t0, y);
+        tmem_ld4(tmem_lane + kColDKx + t0, z);
+        uint32_t fw[4], qw[4];         // raw bf16 bits
+        float fv[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < 4; ++j) {
             const int t = t0 + j;
             fw[j] = reinterpret_cast<const unsigned short *>(fraw)[t * kD + k];
             qw[j] = reinterpret_cast<const unsigned short *>(oraw)[t * kD + k];
@@ -145,63 +149,67 @@ __device__ __forceinline__ void phase_main(uint32_t tmem_lane, const __nv_bfloat
             }
         }
         tmem_wait_ld();
-        // scale factors along the walk (sequential in the running product), 1/f
-        float sq[8], sk[8], rf[8];
+        // Scale factors along the walk (sequential in the running product) and 1/f.  No floor here: a product
+        // that would need one has put the unit on the exact path already (the totals the state warps test are
+        // never larger than any product formed here), and what this pass writes for such a unit is overwritten.
+        // 1/f is the ratio of two consecutive products, so one reciprocal per element serves both.
+        float sq[4], sk[4], rf[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int j = kUp ? i : 7 - i;                      // visiting order: away from the middle
-            if (kUp) cp *= fv[j];
-            const float m = fmaxf(cp, kProdFloor);
-            const float mi = rcp_fast(m);
-            if (!kUp) cp *= fv[j];
-            sq[j] = kUp ? m : mi;
-            sk[j] = kUp ? mi : m;
-            rf[j] = rcp_fast(fmaxf(fv[j], kEnc ? kFDivMinK : kProdFloor));
+        for (int i = 0; i < 4; ++i) {
+            const int j = kUp ? i : 3 - i;                      // visiting order: away from the middle
+            const float c0 = cp, i0 = ci;
+            cp *= fv[j];
+            ci = rcp_fast(cp);
+            sq[j] = kUp ? cp : i0;
+            sk[j] = kUp ? ci : c0;
+            rf[j] = kEnc ? rcp_fast(fmaxf(fv[j], kFDivMinK)) : c0 * ci;
         }
         // element-wise part, two rows per instruction (packed fp32)
-        float a[8], e[8], dk[8];
+        float w[4], dk[4];
 #pragma unroll
-        for (int p = 0; p < 4; ++p) {
+        for (int p = 0; p < 2; ++p) {
             const int j = 2 * p;
             const float2 X = make_float2(__uint_as_float(x[j]), __uint_as_float(x[j + 1]));
             const float2 Y = make_float2(__uint_as_float(y[j]), __uint_as_float(y[j + 1]));
             const float2 Z = make_float2(__uint_as_float(z[j]), __uint_as_float(z[j + 1]));
-            // Qs, Ks of the two rows exactly as the transform warps rounded them for the products: the terms
+            // Qs and -Ks of the two rows exactly as the transform warps rounded them for the products: the terms
             // of a cancel in pairs along the chunk only if both sides use the same operand values
             const uint32_t sqp = pack_bf16(sq[j], sq[j + 1]), skp = pack_bf16(sk[j], sk[j + 1]);
             const uint32_t qsp = mul_bf16x2(qw[j] | (qw[j + 1] << 16), sqp);
-            const uint32_t ksp = kEnc ? mul_bf16x2(fw[j] | (fw[j + 1] << 16), skp)
-                                      : fma_bf16x2(fw[j] | (fw[j + 1] << 16), skp ^ 0x80008000u, skp);
-            const float2 QS = make_float2(bf16_lo(qsp), bf16_hi(qsp)), KS = make_float2(bf16_lo(ksp), bf16_hi(ksp));
+            const uint32_t ksn = kEnc ? mul_bf16x2(fw[j] | (fw[j + 1] << 16), skp ^ 0x80008000u)
+                                      : fma_bf16x2(fw[j] | (fw[j + 1] << 16), skp, skp ^ 0x80008000u);
+            const float2 QS = make_float2(bf16_lo(qsp), bf16_hi(qsp)), KSn = make_float2(bf16_lo(ksn), bf16_hi(ksn));
             const float2 dox = mul2(X, make_float2(sq[j], sq[j + 1]));
-            const float2 a2 = sub2(mul2(QS, X), mul2(KS, Y));
-            const float2 e2 = mul2(KS, Z);
+            const float2 a2 = fma2(KSn, Y, mul2(QS, X));
+            const float2 w2 = fma2(KSn, Z, a2);                 // a - e
+            Gp = add2(Gp, a2);
             const float2 dk2 = mul2(add2(Y, Z), make_float2(sk[j], sk[j + 1]));
             if (!kRagged || t0 + j < n_valid) do_g[(size_t)(t0 + j) * kD] = __float2bfloat16_rn(dox.x);
             if (!kRagged || t0 + j + 1 < n_valid) do_g[(size_t)(t0 + j + 1) * kD] = __float2bfloat16_rn(dox.y);
-            a[j] = a2.x; a[j + 1] = a2.y;
-            e[j] = e2.x; e[j + 1] = e2.y;
+            w[j] = w2.x; w[j + 1] = w2.y;
             dk[j] = dk2.x; dk[j + 1] = dk2.y;
         }
-        // running sums along the walk
-        float u[8];
+        // With K = R + (sum of a over the second half) + (sum of e over the first half), which the final pass
+        // adds, dg_t = K - sum_{32 <= s < t} (a_s - e_s) after the middle and K + sum_{t <= j < 32} (a_j - e_j)
+        // before it: one running sum along the walk
+        float u[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int j = kUp ? i : 7 - i;
-            if (kUp) {              // rows after the middle: sums over the rows strictly before t
-                u[j] = fmaf(H - G, rf[j], -dk[j]);
-                G += a[j]; H += e[j];
-            } else {                // rows before the middle: sums over the rows from t on
-                G += a[j]; H += e[j];
-                u[j] = fmaf(G - H, rf[j], -dk[j]);
+        for (int i = 0; i < 4; ++i) {
+            const int j = kUp ? i : 3 - i;
+            if (kUp) {
+                u[j] = fmaf(-W, rf[j], -dk[j]);
+                W += w[j];
+            } else {
+                W += w[j];
+                u[j] = fmaf(W, rf[j], -dk[j]);
             }
         }
         // park u and 1/f in the columns just read
-        tmem_st8(tmem_lane + kColDQ + t0, u);
-        tmem_st8(tmem_lane + kColDKi + t0, rf);
+        tmem_st4(tmem_lane + kColDQ + t0, u);
+        tmem_st4(tmem_lane + kColDKi + t0, rf);
     }
-    asum = G;
-    esum = H;
+    asum = Gp.x + Gp.y;
+    esum = asum - W;
 }
 
 // kRagged: N is not a whole number of chunks (the tail chunk is padded with neutral tokens); when false,
@@ -414,20 +422,21 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             // ---- R_k = sum_v dS''[k,v] S'[k,v] from the two bf16 copies
             mbar_wait(&ctl->sfull, it & 1, abort_flag);
             PT_MARK(3)
-            float racc = 0.f;
+            float2 racc2 = make_float2(0.f, 0.f);
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
-#pragma unroll
+#pragma unroll 2
                 for (int j = 0; j < 8; ++j) {
                     const uint32_t off = h * kStateSlab + slab_chunk_off(krow, j);
                     const uint4 dw = *reinterpret_cast<const uint4 *>(dsbuf + off);
                     const uint4 sw = *reinterpret_cast<const uint4 *>(sbuf + off);
-                    racc = fmaf(bf16_lo(dw.x), bf16_lo(sw.x), racc); racc = fmaf(bf16_hi(dw.x), bf16_hi(sw.x), racc);
-                    racc = fmaf(bf16_lo(dw.y), bf16_lo(sw.y), racc); racc = fmaf(bf16_hi(dw.y), bf16_hi(sw.y), racc);
-                    racc = fmaf(bf16_lo(dw.z), bf16_lo(sw.z), racc); racc = fmaf(bf16_hi(dw.z), bf16_hi(sw.z), racc);
-                    racc = fmaf(bf16_lo(dw.w), bf16_lo(sw.w), racc); racc = fmaf(bf16_hi(dw.w), bf16_hi(sw.w), racc);
+                    racc2 = fma2(make_float2(bf16_lo(dw.x), bf16_hi(dw.x)), make_float2(bf16_lo(sw.x), bf16_hi(sw.x)), racc2);
+                    racc2 = fma2(make_float2(bf16_lo(dw.y), bf16_hi(dw.y)), make_float2(bf16_lo(sw.y), bf16_hi(sw.y)), racc2);
+                    racc2 = fma2(make_float2(bf16_lo(dw.z), bf16_hi(dw.z)), make_float2(bf16_lo(sw.z), bf16_hi(sw.z)), racc2);
+                    racc2 = fma2(make_float2(bf16_lo(dw.w), bf16_hi(dw.w)), make_float2(bf16_lo(sw.w), bf16_hi(sw.w)), racc2);
                 }
             }
+            const float racc = racc2.x + racc2.y;
             rr[(it & 1) * 128 + krow] = racc;
             mbar_arrive(&ctl->r_ready[it & 1]);
             PT_MARK(4)

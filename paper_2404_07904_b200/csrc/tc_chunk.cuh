@@ -16,10 +16,14 @@
 // The factors exp(b_t - b_m) are in-chunk cumulative PRODUCTS of f taken outward from the middle
 // (the linear-space image of the log-space cumulative sum): rows after m multiply by prod f, rows
 // before m divide by it.  The two factors of a pair can be represented only while the decay across each
-// half of the chunk stays above 2^-100 per key dimension.  Products are floored there (so nothing becomes
-// Inf or NaN); a half whose total Pm or E sits on the floor has left the range, which the state warps of
-// both kernels see when they pick the totals up: they raise the CTA's exact-path flag and the kernels then
-// redo the whole unit with the pairwise-safe fp32 routines of chunk_alu.cuh, which hold on all of [0, 1].
+// half of the chunk stays above 2^-100 per key dimension.  The totals Pm and E are floored there; a half whose
+// total sits on the floor has left the range, which the state warps of both kernels see when they pick the
+// totals up: they raise the CTA's exact-path flag and the kernels then redo the whole unit with the
+// pairwise-safe fp32 routines of chunk_alu.cuh, which hold on all of [0, 1].  The running products inside a
+// half are NOT floored (every one of them is at least as large as the half's total, so inside the range none
+// needs it, and two instructions per element pair in the role that paces the forward are worth 5 % of it):
+// outside the range they may reach zero and the operands Inf or NaN, which stay inside that unit's own
+// accumulators and outputs, all of which the exact path then rewrites.
 #pragma once
 
 #include "tc_common.cuh"
@@ -143,11 +147,10 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
                 f1 = bf16_hi(fw[j]);
             }
             if (kUp) { a0 *= f0; a1 *= f1; }
-            const float m0 = fmaxf(a0, kProdFloor), m1 = fmaxf(a1, kProdFloor);
-            const float i0 = rcp_fast(m0), i1 = rcp_fast(m1);
+            const float i0 = rcp_fast(a0), i1 = rcp_fast(a1);            // no floor: see the file header
+            const float sq0 = kUp ? a0 : i0, sq1 = kUp ? a1 : i1;
+            const float sk0 = kUp ? i0 : a0, sk1 = kUp ? i1 : a1;
             if (!kUp) { a0 *= f0; a1 *= f1; }
-            const float sq0 = kUp ? m0 : i0, sq1 = kUp ? m1 : i1;
-            const float sk0 = kUp ? i0 : m0, sk1 = kUp ? i1 : m1;
             // packed bf16 arithmetic: the scale factors are rounded to bf16 first, then one bf16x2 multiply
             // (resp. fused multiply-add for k = 1 - f) produces the operand pair
             const uint32_t sqp = pack_bf16(sq0, sq1), skp = pack_bf16(sk0, sk1);
@@ -156,7 +159,7 @@ __device__ __forceinline__ void transform_half(uint8_t *qbuf, uint8_t *fbuf, flo
                                                              : fma_bf16x2(fw[j], skp ^ 0x80008000u, skp);
         }
     }
-    // the products only shrink along the walk, so the last one tells whether any row met the floor
+    // the products only shrink along the walk, so the last one tells whether the half stayed inside the range
     const float2 t2 = make_float2(fmaxf(a0, kProdFloor), fmaxf(a1, kProdFloor));
     if (tot) *reinterpret_cast<float2 *>(tot + col) = t2;
     if (tot_g) *reinterpret_cast<float2 *>(tot_g + col) = t2;
