@@ -21,23 +21,28 @@
 // Warp roles (hand-offs are mbarriers, every wait is bounded; loops stay rolled to keep the
 // instruction footprint of the concurrently running roles small):
 //   T   4 warps: raw o, f tiles -> Qs, Ks in place, one chunk ahead (two TMA stages); paced so that it does not
-//       run alongside the output phase and the final d_f pass two chunks back;
+//       run alongside the output walk two chunks back;
 //   E1  4 warps: rescale the dS accumulator and publish its bf16 copy dS'' (the chain between chunks), R;
-//   E3  8 warps: first the causal masks of A and dA into operand slabs (one 32 x 32 block per warp), then d_o
-//       and most of d_f from dQs^T, dKs_intra^T, dKs_inter^T.  A thread owns (key dim, half of the chunk)
-//       and walks its 32 steps outwards from the middle, carrying the decay product and the running sums;
+//   E3  8 warps: d_o and d_f from dQs^T, dKs_intra^T, dKs_inter^T.  A thread owns (key dim, half of the chunk)
+//       and walks its 32 steps outwards from the middle, carrying the decay product and one running sum;
 //       what is still missing then is one constant per key dimension (R plus the two halves' sums), so the
-//       almost finished d_f and 1/f are parked in the TMEM columns just read.  It works from a second,
-//       unswizzled copy of raw o and f and recomputes Qs, Ks with the transform's roundings, so the operand
-//       stage is free as soon as the chunk's products are done;
-//   O   4 warps: d_i from dV^T, and d_f completed from the parked values;
+//       almost finished d_f and 1/f are parked in the TMEM columns just read, and once all eight warps are
+//       through each thread completes its own 32 rows.  It works from a second, unswizzled copy of raw o and f
+//       and recomputes Qs, Ks with the transform's roundings, so the operand stage is free as soon as the
+//       chunk's products are done;
+//   O   4 warps: the causal masks of A and dA into operand slabs (32 rows per warp), and d_i from dV^T;
 //   L   1 warp: TMA loads (o, f, dy stage; v; saved S'; raw o, f), each refilled when its last reader is done;
-//   MX, MY1, MY2  1 warp each: tcgen05.mma issue of the three groups below (one lane issuing all 56
+//   MX, MY1, MY2  1 warp each: tcgen05.mma issue of the groups below (one lane issuing all 56
 //       products of a chunk is itself a bottleneck: its instruction stream is long and serial).
-// Per chunk the tensor pipe runs
-//   X : dS' += Qs^T dY | A | dA            (overlaps the outputs of the previous chunk)
-//   Y1: dKs_inter^T | dV^T = dS''^T Ks^T   (needs the previous chunk's dKs_inter^T, dV^T read out)
-//   Y2: dQs^T | dKs_intra^T | dV^T += dY^T A   (needs tril(A), tril(dA), S', and the parked values consumed)
+// Per chunk the tensor pipe runs, each group as soon as what it overwrites has been read out
+//   X  (MX) : dS' += Qs^T dY | A | dA      (overlaps the outputs of the previous chunk)
+//   Y1a (MY1): dV^T = dS''^T Ks^T           (needs the previous chunk's d_i out: early)
+//   Y1b (MY1): dKs_inter^T                  (needs the previous chunk's output walk finished)
+//   Y2a (MY2): dV^T += dY^T A               (needs tril(A), and Y1a complete)
+//   Y2b (MY2): dQs^T | dKs_intra^T          (needs tril(dA), S', and the previous chunk's parked values consumed)
+// Event stamps of one CTA put the chunk period at: output walk (3.7 k cycles) -> completion of d_f (1.3 k) ->
+// Y2b (1.1 k) -> next walk; with a single Y1 group behind the walk and the masks and the completion pass in the
+// other roles' hands the same stamps showed a second, equally long chain through Y1 and Y2.
 //
 // Tensor-memory plan (512 columns, no spare): dS [0,128); A [128,192) in lanes 0..63 and dA [192,256) in
 // lanes 64..127 (products of the stacked operand (Qs; dY), M = 128); dQs^T [256,320); dKs_intra^T [320,384);
@@ -86,20 +91,21 @@ struct Ctl {
     uint64_t t_done[kStages];     // T -> M, E1
     uint64_t sfull;               // TMA (saved S') -> E1, M
     uint64_t m_done;              // E1 -> M: dS'' is in TMEM and in shared memory
-    uint64_t barX;                // tcgen05.commit -> E1, E3, L: dS' update, A, dA complete
-    uint64_t pd_ready;            // E3 -> M: tril(A), tril(dA) are in shared memory
-    uint64_t barY1;               // tcgen05.commit -> E1: dS'' copy no longer read
-    uint64_t barY2;               // tcgen05.commit -> E3, L: every product of the chunk complete
-    uint64_t r_ready[2];          // E1 -> O, L: R of the chunk is in shared memory, S' no longer read by threads
+    uint64_t barX;                // tcgen05.commit -> E1, O, L: dS' update, A, dA complete
+    uint64_t pd_ready;            // O -> M: tril(A), tril(dA) are in shared memory
+    uint64_t barY1a;              // tcgen05.commit -> MY2: dV^T = dS''^T Ks^T complete
+    uint64_t barY1;               // tcgen05.commit -> E1, L, MY2: both products of dS'' complete (its copy and v no longer read)
+    uint64_t barY2;               // tcgen05.commit -> E3, O, L: every product of the chunk complete
+    uint64_t r_ready[2];          // E1 -> E3, L: R of the chunk is in shared memory, S' no longer read by threads
                                   // (two barriers: the slower of the two waiters must not be lapped)
     uint64_t acc_free1;           // E3 -> M: dKs_inter^T has been read out
     uint64_t acc_freeV;           // O -> M: dV^T has been read out
-    uint64_t parked;              // E3 -> O: the parked values and the halves' sums are in place
-    uint64_t acc_free2;           // O -> M: dQs^T and dKs_intra^T columns are free again
+    uint64_t parked;              // E3 -> E3: every thread's parked values and the halves' sums are in place
+    uint64_t acc_free2;           // E3 -> M: dQs^T and dKs_intra^T columns are free again
     uint64_t drain;               // tcgen05.commit (MX, MY1, MY2, after their loops): every product issued has completed
     int abort_flag;               // set by the first wait that runs out: every later wait returns at once
     uint32_t tmem_base;
-    int o_done;                   // O -> T: final passes finished so far, counted per warp (pacing only)
+    int o_done;                   // E3 -> T: output walks finished so far, counted per warp (pacing only)
     int exact_flag;               // E1: a decay of this CTA's tokens left the range of the rescaled operands
     int l_stage, l_v, l_state, l_raw;   // L: fills asked for so far, per buffer, for the abort epilogue
 };
@@ -290,7 +296,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->sfull, 1);
         mbar_init(&ctl->m_done, kE1Threads);
         mbar_init(&ctl->barX, 1);
-        mbar_init(&ctl->pd_ready, kE3Threads);
+        mbar_init(&ctl->pd_ready, kOThreads);
+        mbar_init(&ctl->barY1a, 1);
         mbar_init(&ctl->barY1, 1);
         mbar_init(&ctl->barY2, 1);
         mbar_init(&ctl->r_ready[0], kE1Threads);
@@ -298,7 +305,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
         mbar_init(&ctl->acc_free1, kE3Threads);
         mbar_init(&ctl->acc_freeV, kOThreads);
         mbar_init(&ctl->parked, kE3Threads);
-        mbar_init(&ctl->acc_free2, kOThreads);
+        mbar_init(&ctl->acc_free2, kE3Threads);
         mbar_init(&ctl->drain, 3);
         ctl->abort_flag = start_aborted;
         ctl->o_done = 0;
@@ -330,12 +337,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int s = it % kStages, c = NC - 1 - it;
             uint8_t *qbuf = smem + s * kStageBytes;
             mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
-            // Pacing, not a data dependence: the transform of chunk `it` starts only when the final d_f pass of
-            // chunk it - 2 is over.  Its tiles are there well before, but run earlier it shares the issue slots
-            // with the output phase and that final pass, the longest stretch of the per-chunk loop (measured:
-            // starting as soon as the tiles land costs 2 %, starting even earlier, via an L2 prefetch, 15 %).
+            // Pacing, not a data dependence: the transform of chunk `it` starts only when the output walk of chunk
+            // it - 2 is over (its completion pass may still run).  The tiles are there well before, but run earlier
+            // the transform shares the issue slots with that walk, the longest stretch of the per-chunk loop
+            // (event stamps: waiting for the completion pass as well made this the longest chain of the kernel;
+            // no pacing at all measured the same as this).
             if (it >= 2) {
-                if (lane == 0) count_wait(&ctl->o_done, kOWarps * (it - 1), abort_flag);   // one poller per warp
+                if (lane == 0) count_wait(&ctl->o_done, kE3Warps * (it - 1), abort_flag);   // one poller per warp
                 __syncwarp();
             }
             PT_MARK(0)
@@ -461,7 +469,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             }
         }
     } else if (warp < kWarpO) {
-        // ================= E3: d_o and the parked part of d_f =================
+        // ================= E3: d_o and d_f =================
         const int half = (warp - kWarpE3) >> 2;                      // half of the chunk: local times [32 * half, +32)
         const uint32_t tl = tmem + lane_base;
         PT_DECL
@@ -469,19 +477,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
             const size_t crow0 = grow0 + (size_t)c * kC;
-            // ---- tril(A), tril(dA) -> operand slabs, one 32 x 32 block per warp.  The
-            // previous chunk's products have read the slabs: this role waited for them before its outputs.
-            mbar_wait(&ctl->barX, it & 1, abort_flag);
-            PT_MARK(0)
-            PT_STAMP(status, 7, tid == kWarpE3 * 32 && it == 16)
-            tc_fence_after_sync();
-            // rows of A sit in lanes 0..63, rows of dA in lanes 64..127: a warp converts 32 rows x 32 columns
-            tril_row_block(tl + (sub < 2 ? kColA : kColDA) + 32 * half, sub < 2 ? pbuf : dpbuf, krow & 63, half);
-            fence_proxy_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&ctl->pd_ready);
-            PT_MARK(1)
-            PT_STAMP(status, 8, tid == kWarpE3 * 32 && it == 16)
             // ---- outputs
             mbar_wait(&ctl->rawfull, it & 1, abort_flag);
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
@@ -497,18 +492,56 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_free1);
             mbar_arrive(&ctl->parked);
+            __syncwarp();
+            if (lane == 0) atomicAdd(&ctl->o_done, 1);
             PT_MARK(3)
             PT_STAMP(status, 15, tid == kWarpE3 * 32 && it == 16)
+            // ---- d_f completed from the parked values, each thread its own 32 rows, once both halves' sums and R
+            // of the chunk are there
+            mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
+            mbar_wait(&ctl->parked, it & 1, abort_flag);
+            tc_fence_after_sync();
+            {
+                const float K = rr[(it & 1) * 128 + krow] + xa[krow] + xe[krow];
+                __nv_bfloat16 *df_g = d_f + crow0 * kD + krow;
+#pragma unroll 1
+                for (int b = 0; b < 4; ++b) {
+                    const int t0 = 32 * half + 8 * b;
+                    uint32_t uu[8], rf[8];
+                    tmem_ld8(tl + kColDQ + t0, uu);
+                    tmem_ld8(tl + kColDKi + t0, rf);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (!kRagged || t0 + j < n_valid)
+                            df_g[(size_t)(t0 + j) * kD] =
+                                __float2bfloat16_rn(fmaf(K, __uint_as_float(rf[j]), __uint_as_float(uu[j])));
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->acc_free2);
+            PT_MARK(4)
         }
-        PT_DUMP(status, 7, 4, tid == kWarpE3 * 32)
+        PT_DUMP(status, 7, 5, tid == kWarpE3 * 32)
     } else if (warp < kWarpLoad) {
-        // ================= O: d_i, and d_f completed from the parked values =================
+        // ================= O: causal masks, d_i =================
         const uint32_t tl = tmem + lane_base;
         PT_DECL
         for (int it = 0; it < NC; ++it) {
             const int c = NC - 1 - it;
             const int n_valid = kRagged ? min(kC, N - c * kC) : kC;
             const size_t crow0 = grow0 + (size_t)c * kC;
+            // ---- tril(A), tril(dA) -> operand slabs: rows of A sit in lanes 0..63, rows of dA in lanes 64..127, a
+            // warp converts its 32 rows.  The previous chunk's products have read the slabs: this role waited for
+            // them before that chunk's d_i.
+            mbar_wait(&ctl->barX, it & 1, abort_flag);
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int hh = 0; hh < 2; ++hh)
+                tril_row_block(tl + (sub < 2 ? kColA : kColDA) + 32 * hh, sub < 2 ? pbuf : dpbuf, krow & 63, hh);
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&ctl->pd_ready);
             mbar_wait(&ctl->barY2, it & 1, abort_flag);
             PT_MARK(0)
             PT_STAMP(status, 16, tid == kWarpO * 32 && it == 16)
@@ -528,30 +561,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             mbar_arrive(&ctl->acc_freeV);
             PT_MARK(1)
             PT_STAMP(status, 17, tid == kWarpO * 32 && it == 16)
-            mbar_wait(&ctl->r_ready[it & 1], (it >> 1) & 1, abort_flag);
-            mbar_wait(&ctl->parked, it & 1, abort_flag);
-            PT_MARK(2)
-            PT_STAMP(status, 18, tid == kWarpO * 32 && it == 16)
-            tc_fence_after_sync();
-            const float K = rr[(it & 1) * 128 + krow] + xa[krow] + xe[krow];
-#pragma unroll 1
-            for (int b = 0; b < 8; ++b) {
-                uint32_t uu[8], rf[8];
-                tmem_ld8(tl + kColDQ + 8 * b, uu);
-                tmem_ld8(tl + kColDKi + 8 * b, rf);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (8 * b + j < n_valid)
-                        d_f[(crow0 + 8 * b + j) * kD + krow] =
-                            __float2bfloat16_rn(fmaf(K, __uint_as_float(rf[j]), __uint_as_float(uu[j])));
-            }
-            tc_fence_before_sync();
-            mbar_arrive(&ctl->acc_free2);
-            __syncwarp();
-            if (lane == 0) atomicAdd(&ctl->o_done, 1);
-            PT_MARK(3)
-            PT_STAMP(status, 19, tid == kWarpO * 32 && it == 16)
         }
         PT_DUMP(status, 11, 4, tid == kWarpO * 32)
     } else if (warp == kWarpLoad) {
@@ -680,21 +689,23 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 mbar_wait(&ctl->full[s], (it / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->t_done[s], (it / kStages) & 1, abort_flag);
                 mbar_wait(&ctl->m_done, it & 1, abort_flag);          // bf16 dS'' in shared memory
-                mbar_wait(&ctl->vfull, it & 1, abort_flag);
                 PT_MARK(0)
-                if (it > 0) {
-                    mbar_wait(&ctl->acc_free1, (it - 1) & 1, abort_flag);
-                    mbar_wait(&ctl->acc_freeV, (it - 1) & 1, abort_flag);
-                }
+                // dV^T first: its accumulator is free as soon as d_i of the previous chunk is out, long before the
+                // output warps have finished with dKs_inter^T
+                if (it > 0) mbar_wait(&ctl->acc_freeV, (it - 1) & 1, abort_flag);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)              // dV^T = dS''^T Ks^T
+                    mma_bf16_ss(tmem + kColDV, ddsm + (uint64_t)(kk * 128), dfk + kmaj(kk), idMK, kk > 0);
+                mma_commit(&ctl->barY1a);
+                mbar_wait(&ctl->vfull, it & 1, abort_flag);
+                if (it > 0) mbar_wait(&ctl->acc_free1, (it - 1) & 1, abort_flag);
                 PT_MARK(1)
                 PT_STAMP(status, 10, it == 16)
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)              // dKs_inter^T = dS'' V^T
                     mma_bf16_ss(tmem + kColDKx, ddsk + kmaj_s(kk), dvk + kmaj(kk), idKK, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)              // dV^T = dS''^T Ks^T
-                    mma_bf16_ss(tmem + kColDV, ddsm + (uint64_t)(kk * 128), dfk + kmaj(kk), idMK, kk > 0);
                 mma_commit(&ctl->barY1);
                 PT_MARK(2)
             }
@@ -705,7 +716,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
                 const uint64_t so = (uint64_t)s * (kStageBytes >> 4);
                 const uint64_t dqm = dqm0 + so, dfm = dfm0 + so, dgk = dgk0 + so, dgm = dgm0 + so;
                 mbar_wait(&ctl->pd_ready, it & 1, abort_flag);   // tril(A), tril(dA); implies X and T of the chunk
-                mbar_wait(&ctl->barY1, it & 1, abort_flag);           // dV^T += ... must follow dV^T = ...
+                mbar_wait(&ctl->barY1a, it & 1, abort_flag);          // dV^T += ... must follow dV^T = ...
                 PT_MARK(0)
                 PT_STAMP(status, 11, it == 16)
                 tc_fence_after_sync();
@@ -727,6 +738,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)              // dKs_intra^T = Qs^T dA
                     mma_bf16_ss(tmem + kColDKi, dqm + (uint64_t)(kk * 128), ddpm + (uint64_t)(kk * 128), idMM, kk > 0);
+                // barY2 stands for every product of the chunk: dKs_inter^T is another lane's, so wait for it first
+                // (it was issued when the output warps finished the previous chunk, well before this point)
+                mbar_wait(&ctl->barY1, it & 1, abort_flag);
                 mma_commit(&ctl->barY2);
                 PT_MARK(2)
                 PT_STAMP(status, 13, it == 16)
