@@ -77,9 +77,21 @@ gate_bwd_kernel(const uint4 *__restrict__ zo, const uint4 *__restrict__ zf, cons
 #pragma unroll
     for (int j = 0; j < 8; ++j) { bh[j] = beta[(size_t)h * kGD + cg * 8 + j]; db[j] = 0.f; }
     const int r1 = min(N, (p + 1) * rows_per);
-    for (int r = p * rows_per + rl; r < r1; r += 16) {
+    // The gradients are rewritten in place, so the compiler must keep every load behind the previous row's
+    // stores: the next row's six loads are therefore issued by hand before the current row is worked on.
+    uint4 na, nb, nc, nda, ndb, ndc;
+    int r = p * rows_per + rl;
+    if (r < r1) {
         const size_t x = ((size_t)u * N + r) * 16 + cg;
-        const uint4 a = zo[x], b = zf[x], c = zi[x], da = g_o[x], dbv = g_f[x], dc = g_i[x];
+        na = zo[x]; nb = zf[x]; nc = zi[x]; nda = g_o[x]; ndb = g_f[x]; ndc = g_i[x];
+    }
+    for (; r < r1; r += 16) {
+        const size_t x = ((size_t)u * N + r) * 16 + cg;
+        const uint4 a = na, b = nb, c = nc, da = nda, dbv = ndb, dc = ndc;
+        if (r + 16 < r1) {
+            const size_t xn = x + 16 * 16;
+            na = zo[xn]; nb = zf[xn]; nc = zi[xn]; nda = g_o[xn]; ndb = g_f[xn]; ndc = g_i[xn];
+        }
         const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w}, cw[4] = {c.x, c.y, c.z, c.w};
         const uint32_t dao[4] = {da.x, da.y, da.z, da.w}, dbf[4] = {dbv.x, dbv.y, dbv.z, dbv.w}, dci[4] = {dc.x, dc.y, dc.z, dc.w};
         uint32_t ro[4], rf[4], ri[4];
@@ -192,7 +204,7 @@ cudaError_t alu_gated_bwd_t(const SeqArgs &a, const float *beta, float *partial)
 // Row slices per unit of the element-wise backward: enough blocks to fill the GPU several times over.
 int gate_bwd_slices(long long U, int N)
 {
-    long long P = (592 + U - 1) / (U > 0 ? U : 1);
+    long long P = (8 * 592 + U - 1) / (U > 0 ? U : 1);
     const long long most = (N + 63) / 64;
     if (P > most) P = most;
     return (int)(P < 1 ? 1 : P);
