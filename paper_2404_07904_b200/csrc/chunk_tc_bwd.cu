@@ -504,19 +504,16 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
             {
                 const float K = rr[(it & 1) * 128 + krow] + xa[krow] + xe[krow];
                 __nv_bfloat16 *df_g = d_f + crow0 * kD + krow;
-#pragma unroll 1
-                for (int b = 0; b < 4; ++b) {
-                    const int t0 = 32 * half + 8 * b;
-                    uint32_t uu[8], rf[8];
-                    tmem_ld8(tl + kColDQ + t0, uu);
-                    tmem_ld8(tl + kColDKi + t0, rf);
-                    tmem_wait_ld();
+                // the thread's 64 parked values in two reads (the pass is on the chunk's critical chain)
+                uint32_t uu[32], rf[32];
+                tmem_ld32(tl + kColDQ + 32 * half, uu);
+                tmem_ld32(tl + kColDKi + 32 * half, rf);
+                tmem_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        if (!kRagged || t0 + j < n_valid)
-                            df_g[(size_t)(t0 + j) * kD] =
-                                __float2bfloat16_rn(fmaf(K, __uint_as_float(rf[j]), __uint_as_float(uu[j])));
-                }
+                for (int j = 0; j < 32; ++j)
+                    if (!kRagged || 32 * half + j < n_valid)
+                        df_g[(size_t)(32 * half + j) * kD] =
+                            __float2bfloat16_rn(fmaf(K, __uint_as_float(rf[j]), __uint_as_float(uu[j])));
             }
             tc_fence_before_sync();
             mbar_arrive(&ctl->acc_free2);
