@@ -277,7 +277,9 @@ hgrn2_status hgrn2_poll(const void *ws);
 /* Number of (batch, head) unit passes that the last tensor-core call using `ws` (a device pointer) redid on
  * the exact fp32 path because the unit's decay left the range described at the top of this file (Eq. 3 holds
  * on all of [0, 1]; the rescaled-operand form of the chunkwise products does not).  A backward that re-creates
- * its states (saved = NULL) counts a unit once for each of its two passes.  Blocking copy: synchronise the
+ * its states (saved = NULL) counts a unit once for each of its two passes; few long sequences whose length is
+ * not a whole number of 64-token chunks run as segments, each of which is redone and counted on its own.
+ * Blocking copy: synchronise the
  * stream first.  0 on the fp32 kernels; -1 if `ws` is NULL or the copy failed. */
 int32_t hgrn2_exact_path_units(const void *ws);
 

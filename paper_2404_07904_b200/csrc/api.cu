@@ -461,7 +461,7 @@ hgrn2_status hgrn2_span_summary_fwd(const hgrn2_desc *desc, const void *f, const
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (U == 0) return cudaMemsetAsync(ws, 0, sizeof(StatusBlock), stream) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
     cudaError_t e;
-    if (use_tc(desc) && desc->N > 0 && desc->N % C == 0) {
+    if (use_tc(desc) && desc->N > 0) {
         e = launch_tc_state_fwd(f, i, (uint64_t)U, desc->N, S_loc, lam, false, static_cast<StatusBlock *>(ws), true,
                                 (desc->flags & HGRN2_FLAG_DEBUG_EXPIRE_WAITS) ? 1 : 0, stream);
     } else {
@@ -487,7 +487,7 @@ hgrn2_status hgrn2_span_summary_bwd(const hgrn2_desc *desc, const void *o, const
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (U == 0) return cudaMemsetAsync(ws, 0, sizeof(StatusBlock), stream) == cudaSuccess ? HGRN2_OK : HGRN2_ERR_CUDA;
     cudaError_t e;
-    if (use_tc(desc) && desc->N > 0 && desc->N % C == 0) {
+    if (use_tc(desc) && desc->N > 0) {
         e = launch_tc_state_bwd(o, f, dy, (uint64_t)U, desc->N, G_loc, lam, false, static_cast<StatusBlock *>(ws), true,
                                 (desc->flags & HGRN2_FLAG_DEBUG_EXPIRE_WAITS) ? 1 : 0, stream);
     } else {

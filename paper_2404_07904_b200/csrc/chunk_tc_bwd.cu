@@ -800,10 +800,11 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 
 // ---- sequences split into segments (see chunk_tc_fwd.cu) ----------------------------------------------
 // Chains the segments in reverse: dS_end[r] = gradient w.r.t. the state at the end of segment r.
+// seg_major: see seg_combine_kernel.
 __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const float *__restrict__ G_loc,
                                        const float *__restrict__ lam, float *__restrict__ dS_end,
                                        float *__restrict__ dS0, int G, int *__restrict__ unit_flag,
-                                       int *__restrict__ unit_count, int units)
+                                       int *__restrict__ unit_count, int units, int seg_major, size_t U)
 {
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
     if (e < (size_t)units) {             // exact-path bookkeeping of the full pass that follows starts at zero
@@ -815,7 +816,7 @@ __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const floa
     const size_t kv = e % (kD * kD);
     float D = dSN ? dSN[e] : 0.f;
     for (int r = G - 1; r >= 0; --r) {
-        const size_t ur = u * G + r;
+        const size_t ur = seg_major ? (size_t)r * U + u : u * G + r;
         dS_end[ur * kD * kD + kv] = D;
         D = fmaf(lam[ur * kD + k], D, G_loc[ur * kD * kD + kv]);
     }
@@ -886,6 +887,37 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         return launch_bwd_once(a, U, a.N, 0, a.dSN, a.dS0, a.clear_status, exact_args(a, a.N, 1, nullptr, nullptr),
                                pk);
     }
+    const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{1, 0};
+    if (rp.G > 1) {
+        // ragged segments (see launch_tc_fwd): state-gradient summaries per segment, chained in reverse, then the
+        // full pass per segment through the packed-batch geometry
+        const int G = rp.G;
+        const uint64_t CT = U * G;
+        char *base = static_cast<char *>(a.seg_scratch);
+        int *cu = reinterpret_cast<int *>(base);
+        float *G_loc = reinterpret_cast<float *>(base + kRSegOffsetsBytes);
+        float *dS_end = G_loc + CT * kD * kD;
+        float *lam = dS_end + CT * kD * kD;
+        launch_seg_offsets(cu, G, rp.Lc * kC, a.N, a.stream);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        PackedArgs pk;
+        pk.cu = cu;
+        pk.H = (int)U;
+        pk.slots_per_head = a.N / kC + G + 1;
+        a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
+                                             (size_t)U * pk.slots_per_head * kSavedStateBytes);
+        err = launch_tc_state_bwd(a.o, a.f, a.dy, U, a.N, G_loc, lam, a.gate_enc, a.status, a.clear_status,
+                                  a.start_aborted, a.stream, cu, G);
+        if (err != cudaSuccess) return err;
+        seg_combine_bwd_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.dSN, G_loc, lam, dS_end, a.dS0, G,
+                                                                                   nullptr, nullptr, 0, 1, (size_t)U);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        SeqArgs t = a;
+        t.dSN = dS_end;
+        t.dS0 = nullptr;
+        return launch_bwd_once(t, CT, a.N, 0, dS_end, nullptr, false, exact_args(t, a.N, 1, nullptr, nullptr), pk);
+    }
     a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
     const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
     cudaError_t err = cudaSuccess;
@@ -910,7 +942,7 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         err = launch_tc_state_bwd(t.o, t.f, t.dy, Ut * G, a.N / G, G_loc, lam, a.gate_enc, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
         seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G,
-                                                                                    unit_flag, unit_count, (int)Ut);
+                                                                                    unit_flag, unit_count, (int)Ut, 0, (size_t)Ut);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false,
                               exact_args(t, a.N, G, unit_flag, unit_count));

@@ -589,7 +589,11 @@ bool tc_chunk_supported(int C) { return C == kC; }
 size_t tc_saved_bytes(const hgrn2_desc *d, int C)
 {
     const size_t NC = ((size_t)d->N + C - 1) / C;
-    return (size_t)d->B * d->H * NC * (kSavedStateBytes + kSavedTotalsBytes);
+    const uint64_t U = (uint64_t)d->B * d->H;
+    const RSegPlan rp = tc_rseg_plan(U, d->N, (int)NC);
+    // ragged segments use the packed batch's slot numbering: N / C + (segments) + 1 slots per unit
+    const size_t slots = rp.G > 1 ? (size_t)d->N / C + rp.G + 1 : NC;
+    return (size_t)U * slots * (kSavedStateBytes + kSavedTotalsBytes);
 }
 
 // ---- sequences split into segments ----------------------------------------------------------------------
@@ -599,9 +603,12 @@ size_t tc_saved_bytes(const hgrn2_desc *d, int C)
 // its total decay Lambda = prod f; (2) a small kernel chains them, S_start[r+1] = Diag(Lambda[r]) S_start[r] + S_local[r];
 // (3) every segment runs in full from its S_start.  Token (r, t) of unit u is token t of "unit" u * G + r of a
 // [U * G][N / G][128] view of the same memory, so the kernel itself does not know about segments.
+// seg_major = 0: segment r of unit u sits at index u * G + r; 1: at r * U + u (the packed-batch order of the
+// ragged segments).
 __global__ void seg_combine_kernel(const float *__restrict__ S0, const float *__restrict__ S_loc,
                                    const float *__restrict__ lam, float *__restrict__ S_start, float *__restrict__ SN,
-                                   int G, int *__restrict__ unit_flag, int *__restrict__ unit_count, int units)
+                                   int G, int *__restrict__ unit_flag, int *__restrict__ unit_count, int units,
+                                   int seg_major, size_t U)
 {
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
     if (e < (size_t)units) {             // exact-path bookkeeping of the full pass that follows starts at zero
@@ -613,7 +620,7 @@ __global__ void seg_combine_kernel(const float *__restrict__ S0, const float *__
     const size_t kv = e % (kD * kD);
     float S = S0 ? S0[e] : 0.f;
     for (int r = 0; r < G; ++r) {
-        const size_t ur = u * G + r;
+        const size_t ur = seg_major ? (size_t)r * U + u : u * G + r;
         S_start[ur * kD * kD + kv] = S;
         S = fmaf(lam[ur * kD + k], S, S_loc[ur * kD * kD + kv]);
     }
@@ -637,6 +644,34 @@ int segments_for(uint64_t U, int N, int NC)
     if (G > 8) G = 8;
     while (G >= 2 && (NC % G != 0 || NC / G < 8)) --G;
     return G >= 2 ? G : 1;
+}
+
+// Sequences that are not whole chunks, few units: segments of Lc chunks (at least 8), the last one shorter.
+RSegPlan tc_rseg_plan(uint64_t U, int N, int NC)
+{
+    RSegPlan p{1, 0};
+    const int sms = sm_count();
+    if (U == 0 || sms == 0 || N % kC == 0 || U > (uint64_t)sms) return p;
+    int G0 = sms / (int)U;
+    if (G0 > 8) G0 = 8;
+    if (G0 < 2) return p;
+    int Lc = (NC + G0 - 1) / G0;
+    if (Lc < 8) Lc = 8;
+    const int G = (NC + Lc - 1) / Lc;
+    if (G < 2) return p;
+    return RSegPlan{G, Lc};
+}
+
+// cu[r] = first row of segment r (r = 0 .. G), segments of L rows, the last one ends at N
+__global__ void seg_offsets_kernel(int *__restrict__ cu, int G, int L, int N)
+{
+    const int r = threadIdx.x;
+    if (r <= G) cu[r] = min(r * L, N);
+}
+
+void launch_seg_offsets(int *cu, int G, int L, int N, cudaStream_t stream)
+{
+    seg_offsets_kernel<<<1, 32, 0, stream>>>(cu, G, L, N);
 }
 
 // Few units (no more than SMs): all of them are split.  More units than SMs: the units beyond the last full
@@ -693,12 +728,19 @@ size_t tc_segment_scratch_bytes(const hgrn2_desc *d, int C)
 {
     const uint64_t U = (uint64_t)d->B * d->H;
     const int NC = (d->N + C - 1) / C;
+    const RSegPlan rp = tc_rseg_plan(U, d->N, NC);
+    if (rp.G > 1) return kRSegOffsetsBytes + (size_t)U * rp.G * (2 * kD * kD + kD) * sizeof(float);
     const SegPlan p = tc_seg_plan(U, d->N, NC);
     return p.tail_units ? (size_t)p.tail_units * p.G * (2 * kD * kD + kD) * sizeof(float) + seg_flag_bytes(p.tail_units) : 0;
 }
 
 // One float matrix per unit for the exact path of the backward (chunk_alu.cuh, bwd_unit).
-size_t tc_exact_scratch_bytes(const hgrn2_desc *d) { return (size_t)d->B * d->H * kD * kD * sizeof(float); }
+size_t tc_exact_scratch_bytes(const hgrn2_desc *d)
+{
+    const uint64_t U = (uint64_t)d->B * d->H;
+    const RSegPlan rp = tc_rseg_plan(U, d->N, (d->N + kC - 1) / kC);      // ragged segments: one matrix per segment
+    return (size_t)U * (rp.G > 1 ? rp.G : 1) * kD * kD * sizeof(float);
+}
 
 static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag, int *unit_count)
 {
@@ -777,9 +819,43 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         return launch_fwd_once(a, U, a.N, 0, a.S0, a.SN, a.y != nullptr, a.states != nullptr, a.clear_status,
                                exact_args(a, a.N, 1, nullptr, nullptr), pk);
     }
+    const bool want_y = a.y != nullptr, want_saved = a.states != nullptr;
+    const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{1, 0};
+    if (rp.G > 1) {
+        // ragged segments: the three steps of the whole-chunk segments below, with per-CTA rows from an offsets
+        // array (the packed-batch geometry: "sequence" r of "head" u = segment r of unit u); every segment CTA
+        // takes its own exact path from its start state, which the state-only pass gives for every f
+        const int G = rp.G;
+        const uint64_t CT = U * G;
+        char *base = static_cast<char *>(a.seg_scratch);
+        int *cu = reinterpret_cast<int *>(base);
+        float *S_loc = reinterpret_cast<float *>(base + kRSegOffsetsBytes);
+        float *S_start = S_loc + CT * kD * kD;
+        float *lam = S_start + CT * kD * kD;
+        launch_seg_offsets(cu, G, rp.Lc * kC, a.N, a.stream);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        PackedArgs pk;
+        pk.cu = cu;
+        pk.H = (int)U;
+        pk.slots_per_head = a.N / kC + G + 1;
+        if (a.states)
+            a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
+                                                 (size_t)U * pk.slots_per_head * kSavedStateBytes);
+        err = launch_tc_state_fwd(a.f, a.i, U, a.N, S_loc, lam, a.gate_enc, a.status, a.clear_status, a.start_aborted,
+                                  a.stream, cu, G);
+        if (err != cudaSuccess) return err;
+        seg_combine_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.S0, S_loc, lam, S_start, a.SN, G,
+                                                                               nullptr, nullptr, 0, 1, (size_t)U);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        SeqArgs t = a;
+        t.S0 = S_start;
+        t.SN = nullptr;
+        return launch_fwd_once(t, CT, a.N, 0, S_start, nullptr, want_y, want_saved, false,
+                               exact_args(t, a.N, 1, nullptr, nullptr), pk);
+    }
     if (a.states) a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) + U * a.NC * kSavedStateBytes);
     const SegPlan plan = a.seg_scratch ? tc_seg_plan(U, a.N, a.NC) : SegPlan{U, 0, 1};
-    const bool want_y = a.y != nullptr, want_saved = a.states != nullptr;
     cudaError_t err = cudaSuccess;
     bool clear = a.clear_status;                                  // for the first kernel launched only
     if (plan.main_units) {
@@ -802,7 +878,7 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         err = launch_tc_state_fwd(t.f, t.i, Ut * G, a.N / G, S_loc, lam, a.gate_enc, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
         seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G,
-                                                                                unit_flag, unit_count, (int)Ut);
+                                                                                unit_flag, unit_count, (int)Ut, 0, (size_t)Ut);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, want_y, want_saved, false,
                               exact_args(t, a.N, G, unit_flag, unit_count));

@@ -19,6 +19,11 @@
 // its half's f, exchanges that with the other half through shared memory, then walks its rows), L 1 warp (TMA
 // loads, four stages), M 1 warp (tcgen05.mma issue, 4 K-steps per chunk into one 128 x 128 fp32 accumulator);
 // at the end the T warps move the accumulator to global memory.  Every wait is bounded (tc_common.cuh).
+//
+// kRagged instantiations: the segment need not be a whole number of chunks (rows past its end act as the
+// neutral token f = 1, q = 0), and a CTA may take its rows from an offsets array: CTA u = b * planes + h then
+// covers rows [cu[b], cu[b + 1]) of plane h of the [planes][rows][128] tensors (sequences cut into segments of
+// unequal length, chunk_tc_fwd.cu).
 #include "tc_chunk.cuh"
 
 namespace hgrn2 {
@@ -55,11 +60,12 @@ struct Ctl {
 static_assert(sizeof(Ctl) <= 256, "control block");
 
 // kEnc: the f tensor holds the signed gate encoding (see transform_half in tc_chunk.cuh).
-template <bool kBwd, bool kEnc>
+template <bool kBwd, bool kEnc, bool kRagged>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__ CUtensorMap map_f,
-                const __grid_constant__ CUtensorMap map_w, float *__restrict__ out, float *__restrict__ lam, int NC,
-                StatusBlock *status, int clear_status, int start_aborted)
+                const __grid_constant__ CUtensorMap map_w, float *__restrict__ out, float *__restrict__ lam, int N_all,
+                int NC_all, const int *__restrict__ cu, int planes, StatusBlock *status, int clear_status,
+                int start_aborted)
 {
     using G = Geo<kBwd>;
     if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -75,6 +81,26 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int u = blockIdx.x;
+    // this CTA's segment: rows [row0, row0 + N) of plane zu, NC chunks
+    int row0 = 0, zu = u, N = N_all, NC = NC_all;
+    if constexpr (kRagged) {
+        if (cu != nullptr) {
+            const int b = u / planes;
+            zu = u - b * planes;
+            row0 = __ldg(cu + b);
+            N = __ldg(cu + b + 1) - row0;
+            if (row0 < 0 || N < 0 || row0 + N > N_all) {          // malformed offsets: report, touch nothing
+                if (tid == 0) report_error(status, HGRN2_ERR_INVALID_ARG, 6);
+                return;
+            }
+        }
+        NC = (N + kC - 1) / kC;
+        if (N <= 0) {                    // an empty segment contributes nothing and does not decay
+            for (int x = tid; x < kD * kD; x += kThreads) out[(size_t)u * kD * kD + x] = 0.f;
+            if (lam != nullptr && tid < kD) lam[(size_t)u * kD + tid] = 1.f;
+            return;
+        }
+    }
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -112,6 +138,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
             uint8_t *xbuf = smem + s * G::kStageBytes + G::kOffX;
             const uint8_t *fbuf = smem + s * G::kStageBytes + G::kOffF;
             mbar_wait(&ctl->full[s], (n / kStages) & 1, abort_flag);
+            const int n_valid = kRagged ? N - (kBwd ? n : NC - 1 - n) * kC : kC;     // rows of the chunk inside the segment
             // this half's f (32 rows of the column pair) and its product
             uint32_t fw[32];
             float h0 = 1.f, h1 = 1.f;
@@ -119,6 +146,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
             for (int j = 0; j < 32; ++j) {
                 const int r = 32 * half + j;
                 fw[j] = *reinterpret_cast<const uint32_t *>(fbuf + xo[r & 7] + r * 128);
+                if (kRagged && r >= n_valid) fw[j] = kEnc ? 0x80008000u : 0x3F803F80u;      // f = 1, k = 0
                 float f0, f1, k0, k1;
                 if (kEnc) {
                     gate_decode(fw[j], f0, k0);
@@ -155,7 +183,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
                 if (kBwd) {                                           // c includes row r: X = q * prod_{<= r} f
                     a0 *= f0;
                     a1 *= f1;
-                    const uint32_t qw = *reinterpret_cast<const uint32_t *>(xbuf + off);
+                    uint32_t qw = *reinterpret_cast<const uint32_t *>(xbuf + off);
+                    if (kRagged && r >= n_valid) qw = 0u;
                     *reinterpret_cast<uint32_t *>(xbuf + off) = mul_bf16x2(qw, pack_bf16(a0, a1));
                 } else {                                              // c excludes row r: X = (1 - f) * prod_{> r} f
                     const uint32_t cp = pack_bf16(a0, a1);
@@ -200,9 +229,9 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
                 }
                 mbar_arrive_expect_tx(&ctl->full[s], G::kStageBytes);
                 for (int b = 0; b < 2; ++b) {
-                    if (kBwd) tma_load_3d(st + G::kOffX + b * kSlab, &map_o, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + G::kOffF + b * kSlab, &map_f, &ctl->full[s], 64 * b, c * kC, u);
-                    tma_load_3d(st + G::kOffW + b * kSlab, &map_w, &ctl->full[s], 64 * b, c * kC, u);
+                    if (kBwd) tma_load_3d(st + G::kOffX + b * kSlab, &map_o, &ctl->full[s], 64 * b, row0 + c * kC, zu);
+                    tma_load_3d(st + G::kOffF + b * kSlab, &map_f, &ctl->full[s], 64 * b, row0 + c * kC, zu);
+                    tma_load_3d(st + G::kOffW + b * kSlab, &map_w, &ctl->full[s], 64 * b, row0 + c * kC, zu);
                 }
                 issued = n + 1;
             }
@@ -242,38 +271,56 @@ tc_state_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant
     if (warp == 0) tmem_dealloc(tmem, 128);
 }
 
-template <bool kBwd, bool kEnc>
-cudaError_t launch_state(const void *o, const void *f, const void *w, uint64_t U, int N, int NC, float *out, float *lam,
-                         StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream)
+template <bool kBwd, bool kEnc, bool kRagged>
+cudaError_t launch_state_t(const void *o, const void *f, const void *w, uint64_t planes, int N, uint64_t ctas, const int *cu,
+                           float *out, float *lam, StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream)
 {
     using G = Geo<kBwd>;
     CUtensorMap mo, mf, mw;
-    if (!make_map(&mo, kBwd ? o : f, U, N, kC) || !make_map(&mf, f, U, N, kC) || !make_map(&mw, w, U, N, kC))
+    if (!make_map(&mo, kBwd ? o : f, planes, N, kC) || !make_map(&mf, f, planes, N, kC) || !make_map(&mw, w, planes, N, kC))
         return cudaErrorInvalidValue;
-    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(tc_state_kernel<kBwd, kEnc>), G::kSmemBytes);
+    auto kernel = tc_state_kernel<kBwd, kEnc, kRagged>;
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), G::kSmemBytes);
     if (err != cudaSuccess) return err;
-    tc_state_kernel<kBwd, kEnc><<<(unsigned)U, kThreads, G::kSmemBytes, stream>>>(mo, mf, mw, out, lam, NC, status,
-                                                                             clear ? 1 : 0, start_aborted);
+    kernel<<<(unsigned)ctas, kThreads, G::kSmemBytes, stream>>>(mo, mf, mw, out, lam, N, N / kC, cu, (int)planes, status,
+                                                             clear ? 1 : 0, start_aborted);
     return cudaGetLastError();
+}
+
+// planes x N rows; without offsets one CTA per plane, with offsets nseq CTAs per plane (see the kernel)
+template <bool kBwd>
+cudaError_t launch_state(const void *o, const void *f, const void *w, uint64_t planes, int N, const int *cu, int nseq,
+                         float *out, float *lam, bool gate_enc, StatusBlock *status, bool clear, int start_aborted,
+                         cudaStream_t stream)
+{
+    const bool ragged = cu != nullptr || N % kC != 0;
+    const uint64_t ctas = cu ? planes * (uint64_t)nseq : planes;
+    if (ctas == 0 || N <= 0) return cudaSuccess;
+    if (ctas > 0x7fffffffull) return cudaErrorInvalidConfiguration;
+    if (gate_enc)
+        return ragged ? launch_state_t<kBwd, true, true>(o, f, w, planes, N, ctas, cu, out, lam, status, clear, start_aborted, stream)
+                      : launch_state_t<kBwd, true, false>(o, f, w, planes, N, ctas, cu, out, lam, status, clear, start_aborted, stream);
+    return ragged ? launch_state_t<kBwd, false, true>(o, f, w, planes, N, ctas, cu, out, lam, status, clear, start_aborted, stream)
+                  : launch_state_t<kBwd, false, false>(o, f, w, planes, N, ctas, cu, out, lam, status, clear, start_aborted, stream);
 }
 
 }  // namespace
 
-// Forward: S_loc [U][128][128] and Lambda [U][128] of U segments of N tokens (whole chunks) from f and i.
+// Forward: S_loc [.][128][128] and Lambda [.][128] from f and i.  Without `cu`: one segment per plane, the N rows
+// of each of the U planes.  With `cu` (device, nseq + 1 offsets): segment b * U + h = rows [cu[b], cu[b + 1]) of plane h.
 cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam, bool gate_enc,
-                                StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream)
+                                StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream, const int *cu,
+                                int nseq)
 {
-    if (gate_enc) return launch_state<false, true>(nullptr, f, i, U, N, N / kC, S_loc, lam, status, clear, start_aborted, stream);
-    return launch_state<false, false>(nullptr, f, i, U, N, N / kC, S_loc, lam, status, clear, start_aborted, stream);
+    return launch_state<false>(nullptr, f, i, U, N, cu, nseq, S_loc, lam, gate_enc, status, clear, start_aborted, stream);
 }
 
-// Backward: G_loc [U][128][128] and Lambda [U][128] of U segments of N tokens (whole chunks) from o, f and dy.
+// Backward: G_loc and Lambda of the same segments from o, f and dy.
 cudaError_t launch_tc_state_bwd(const void *o, const void *f, const void *dy, uint64_t U, int N, float *G_loc,
                                 float *lam, bool gate_enc, StatusBlock *status, bool clear, int start_aborted,
-                                cudaStream_t stream)
+                                cudaStream_t stream, const int *cu, int nseq)
 {
-    if (gate_enc) return launch_state<true, true>(o, f, dy, U, N, N / kC, G_loc, lam, status, clear, start_aborted, stream);
-    return launch_state<true, false>(o, f, dy, U, N, N / kC, G_loc, lam, status, clear, start_aborted, stream);
+    return launch_state<true>(o, f, dy, U, N, cu, nseq, G_loc, lam, gate_enc, status, clear, start_aborted, stream);
 }
 
 }  // namespace hgrn2

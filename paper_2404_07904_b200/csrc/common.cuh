@@ -138,13 +138,23 @@ struct SegPlan {
     int G;
 };
 SegPlan     tc_seg_plan(uint64_t U, int N, int NC);
+// Few units whose sequences are NOT whole chunks: every sequence is cut into G segments of Lc chunks (the last one
+// shorter), which run through the packed-batch geometry (per-CTA rows from an offsets array).  G = 1: not split.
+struct RSegPlan {
+    int G;
+    int Lc;
+};
+RSegPlan    tc_rseg_plan(uint64_t U, int N, int NC);
+constexpr size_t kRSegOffsetsBytes = 256;      // the offsets array of the ragged segments, in front of their scratch
+void        launch_seg_offsets(int *cu, int G, int L, int N, cudaStream_t stream);
 SeqArgs     tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n);
 
 cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam, bool gate_enc,
-                                StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream);
+                                StatusBlock *status, bool clear, int start_aborted, cudaStream_t stream,
+                                const int *cu = nullptr, int nseq = 1);
 cudaError_t launch_tc_state_bwd(const void *o, const void *f, const void *dy, uint64_t U, int N, float *G_loc,
                                 float *lam, bool gate_enc, StatusBlock *status, bool clear, int start_aborted,
-                                cudaStream_t stream);
+                                cudaStream_t stream, const int *cu = nullptr, int nseq = 1);
 cudaError_t launch_step(const StepArgs &a);
 bool        step_multi_supported(int dk, int dv);
 cudaError_t launch_step_multi(const StepArgs &a);
