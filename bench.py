@@ -298,8 +298,10 @@ def run_other_workloads(args, binding, W, dev, rank, timed, peaks, bf):
     out = []
     if rank != 0:
         return out
-    for name, gamma in (("long_16k", None),) + tuple(("lm_2560", g) for g in W.LM_2560_GAMMAS):
-        w = W.CONFIGS[name]
+    # prefill_5000: few long sequences whose length is not a whole number of chunks (16 heads x 5000 tokens), the
+    # recipe of long_16k at another shape
+    for name, gamma in (("long_16k", None),) + tuple(("lm_2560", g) for g in W.LM_2560_GAMMAS) + (("prefill_5000", None),):
+        w = W.scaled(W.CONFIGS["long_16k"], B=1, H=16, N=5000) if name == "prefill_5000" else W.CONFIGS[name]
         inp = W.make_inputs(w, gamma=gamma)
         t = {k: (None if v is None else torch.from_numpy(v).to(dev)) for k, v in inp.items()}
         o, f, i, dy = (t[k].to(bf) for k in ("o", "f", "i", "dy"))

@@ -87,7 +87,10 @@ typedef struct hgrn2_desc {
 
 /* Bytes of the `saved` buffer that hgrn2_fwd fills for hgrn2_bwd: the state at the
  * start of every chunk (derived from Eq. 3 by unrolling C steps) and, on the tensor-core
- * path, the two per-chunk decay totals of every key dimension.  0 on a bad desc. */
+ * path, the two per-chunk decay totals of every key dimension.  On that path the layout is private
+ * to the library and, for few long sequences that are not a whole number of chunks (which run as
+ * segments), a little larger than one state per chunk: the size then depends on the current device,
+ * and forward and backward of one buffer must run on devices with the same SM count.  0 on a bad desc. */
 size_t hgrn2_saved_bytes(const hgrn2_desc *desc);
 
 /* Bytes of the workspace `ws` every call takes: a 256-byte status block, room for the
