@@ -14,7 +14,8 @@ int         tc_default_chunk();
 bool        tc_chunk_supported(int C);
 size_t      tc_saved_bytes(const hgrn2_desc *d, int C);
 size_t      tc_segment_scratch_bytes(const hgrn2_desc *d, int C);
-size_t      tc_exact_scratch_bytes(const hgrn2_desc *d);
+size_t      tc_exact_scratch_bytes(const hgrn2_desc *d, bool packed);
+size_t      tc_segment_scratch_bytes_packed(const hgrn2_desc *d);
 size_t      tc_saved_bytes_packed(const hgrn2_desc *d);
 // span summaries for sequence parallelism (span.cu)
 cudaError_t launch_span_summary(bool bwd, int io, const void *x, const void *f, const void *w, long long U, int N, int dk,
@@ -88,7 +89,9 @@ size_t saved_bytes_for(const hgrn2_desc *d, int C, bool packed = false)
 size_t workspace_bytes_for(const hgrn2_desc *d, int C, bool packed)
 {
     return sizeof(StatusBlock) + saved_bytes_for(d, C, packed) +
-           (use_tc(d) ? (packed ? 0 : tc_segment_scratch_bytes(d, C)) + tc_exact_scratch_bytes(d) : 0);
+           (use_tc(d) ? (packed ? tc_segment_scratch_bytes_packed(d) : tc_segment_scratch_bytes(d, C)) +
+                            tc_exact_scratch_bytes(d, packed)
+                      : 0);
 }
 
 void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream, void *ws, const int32_t *cu = nullptr)
@@ -102,7 +105,7 @@ void fill_args(SeqArgs &a, const hgrn2_desc *d, int C, void *stream, void *ws, c
     a.exact_scratch = nullptr;
     if (use_tc(d)) {
         char *p = static_cast<char *>(ws) + sizeof(StatusBlock) + saved_bytes_for(d, C, cu != nullptr);
-        const size_t seg = cu ? 0 : tc_segment_scratch_bytes(d, C);
+        const size_t seg = cu ? tc_segment_scratch_bytes_packed(d) : tc_segment_scratch_bytes(d, C);
         if (seg != 0) a.seg_scratch = p;
         a.exact_scratch = reinterpret_cast<float *>(p + seg);
     }
@@ -297,7 +300,7 @@ size_t beta_partial_bytes(const hgrn2_desc *d)
 size_t workspace_bytes_gated(const hgrn2_desc *d, int C)
 {
     return sizeof(StatusBlock) + saved_bytes_gated(d, C) +
-           (use_tc(d) ? tc_segment_scratch_bytes(d, C) + tc_exact_scratch_bytes(d) : 0) + beta_partial_bytes(d);
+           (use_tc(d) ? tc_segment_scratch_bytes(d, C) + tc_exact_scratch_bytes(d, false) : 0) + beta_partial_bytes(d);
 }
 
 // Pointers into the workspace behind the saved-data room.
@@ -310,7 +313,7 @@ void gated_ws_layout(SeqArgs &a, const hgrn2_desc *d, int C, void *ws, float **p
         const size_t seg = tc_segment_scratch_bytes(d, C);
         if (seg != 0) a.seg_scratch = p;
         a.exact_scratch = reinterpret_cast<float *>(p + seg);
-        p += seg + tc_exact_scratch_bytes(d);
+        p += seg + tc_exact_scratch_bytes(d, false);
     }
     *partial = reinterpret_cast<float *>(p);
 }

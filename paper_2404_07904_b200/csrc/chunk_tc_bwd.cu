@@ -804,7 +804,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap map_o, const __grid_constant__
 __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const float *__restrict__ G_loc,
                                        const float *__restrict__ lam, float *__restrict__ dS_end,
                                        float *__restrict__ dS0, int G, int *__restrict__ unit_flag,
-                                       int *__restrict__ unit_count, int units, int seg_major, size_t U)
+                                       int *__restrict__ unit_count, int units, int seg_major, size_t U, int H)
 {
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
     if (e < (size_t)units) {             // exact-path bookkeeping of the full pass that follows starts at zero
@@ -816,7 +816,7 @@ __global__ void seg_combine_bwd_kernel(const float *__restrict__ dSN, const floa
     const size_t kv = e % (kD * kD);
     float D = dSN ? dSN[e] : 0.f;
     for (int r = G - 1; r >= 0; --r) {
-        const size_t ur = seg_major ? (size_t)r * U + u : u * G + r;
+        const size_t ur = seg_index(seg_major, u, r, G, U, H);
         dS_end[ur * kD * kD + kv] = D;
         D = fmaf(lam[ur * kD + k], D, G_loc[ur * kD * kD + kv]);
     }
@@ -845,7 +845,7 @@ static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag,
     return ex;
 }
 
-PackedArgs tc_packed_args(const SeqArgs &a);
+PackedArgs tc_packed_args(const SeqArgs &a, int G);
 
 // U CTAs; ordinary layout: U planes of N rows; packed batch (pk.cu set): pk.H planes of N rows shared by the U units.
 static cudaError_t launch_bwd_once(const SeqArgs &a, uint64_t U, int N, int NC, const float *dSN, float *dS0,
@@ -881,11 +881,34 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
     SeqArgs a = a0;
     if (a.cu) {
         // packed batch: one CTA per (sequence, head), every CTA reads its own rows from the offsets array
-        const PackedArgs pk = tc_packed_args(a);
+        const int G = a.seg_scratch ? tc_packed_segments(U) : 1;
+        PackedArgs pk = tc_packed_args(a, G);
         a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
                                              (size_t)pk.H * pk.slots_per_head * kSavedStateBytes);
-        return launch_bwd_once(a, U, a.N, 0, a.dSN, a.dS0, a.clear_status, exact_args(a, a.N, 1, nullptr, nullptr),
-                               pk);
+        if (G <= 1)
+            return launch_bwd_once(a, U, a.N, 0, a.dSN, a.dS0, a.clear_status, exact_args(a, a.N, 1, nullptr, nullptr),
+                                   pk);
+        // few units: every sequence as G segments (see launch_tc_fwd)
+        const uint64_t CT = U * G;
+        char *base = static_cast<char *>(a.seg_scratch);
+        int *cu_seg = reinterpret_cast<int *>(base);
+        float *G_loc = reinterpret_cast<float *>(base + tc_packed_offsets_bytes(a.B, G));
+        float *dS_end = G_loc + CT * kD * kD;
+        float *lam = dS_end + CT * kD * kD;
+        launch_seg_offsets_packed(a.cu, a.B, G, cu_seg, a.stream);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        pk.cu = cu_seg;
+        err = launch_tc_state_bwd(a.o, a.f, a.dy, (uint64_t)a.H, a.N, G_loc, lam, a.gate_enc, a.status, a.clear_status,
+                                  a.start_aborted, a.stream, cu_seg, a.B * G);
+        if (err != cudaSuccess) return err;
+        seg_combine_bwd_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.dSN, G_loc, lam, dS_end, a.dS0, G,
+                                                                                   nullptr, nullptr, 0, 2, (size_t)U, a.H);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        SeqArgs t = a;
+        t.dSN = dS_end;
+        t.dS0 = nullptr;
+        return launch_bwd_once(t, CT, a.N, 0, dS_end, nullptr, false, exact_args(t, a.N, 1, nullptr, nullptr), pk);
     }
     const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{1, 0};
     if (rp.G > 1) {
@@ -911,7 +934,7 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
                                   a.start_aborted, a.stream, cu, G);
         if (err != cudaSuccess) return err;
         seg_combine_bwd_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.dSN, G_loc, lam, dS_end, a.dS0, G,
-                                                                                   nullptr, nullptr, 0, 1, (size_t)U);
+                                                                                   nullptr, nullptr, 0, 1, (size_t)U, 1);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         SeqArgs t = a;
         t.dSN = dS_end;
@@ -942,7 +965,7 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         err = launch_tc_state_bwd(t.o, t.f, t.dy, Ut * G, a.N / G, G_loc, lam, a.gate_enc, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
         seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G,
-                                                                                    unit_flag, unit_count, (int)Ut, 0, (size_t)Ut);
+                                                                                    unit_flag, unit_count, (int)Ut, 0, (size_t)Ut, 1);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         err = launch_bwd_once(t, Ut * G, a.N / G, a.NC / G, dS_end, nullptr, false,
                               exact_args(t, a.N, G, unit_flag, unit_count));

@@ -604,11 +604,12 @@ size_t tc_saved_bytes(const hgrn2_desc *d, int C)
 // (3) every segment runs in full from its S_start.  Token (r, t) of unit u is token t of "unit" u * G + r of a
 // [U * G][N / G][128] view of the same memory, so the kernel itself does not know about segments.
 // seg_major = 0: segment r of unit u sits at index u * G + r; 1: at r * U + u (the packed-batch order of the
-// ragged segments).
+// ragged segments); 2: unit u = (sequence b, head h) of a packed batch with H heads, its segment r at
+// (b * G + r) * H + h.
 __global__ void seg_combine_kernel(const float *__restrict__ S0, const float *__restrict__ S_loc,
                                    const float *__restrict__ lam, float *__restrict__ S_start, float *__restrict__ SN,
                                    int G, int *__restrict__ unit_flag, int *__restrict__ unit_count, int units,
-                                   int seg_major, size_t U)
+                                   int seg_major, size_t U, int H)
 {
     const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // element of [U][128][128]
     if (e < (size_t)units) {             // exact-path bookkeeping of the full pass that follows starts at zero
@@ -620,7 +621,7 @@ __global__ void seg_combine_kernel(const float *__restrict__ S0, const float *__
     const size_t kv = e % (kD * kD);
     float S = S0 ? S0[e] : 0.f;
     for (int r = 0; r < G; ++r) {
-        const size_t ur = seg_major ? (size_t)r * U + u : u * G + r;
+        const size_t ur = seg_index(seg_major, u, r, G, U, H);
         S_start[ur * kD * kD + kv] = S;
         S = fmaf(lam[ur * kD + k], S, S_loc[ur * kD * kD + kv]);
     }
@@ -673,6 +674,43 @@ void launch_seg_offsets(int *cu, int G, int L, int N, cudaStream_t stream)
 {
     seg_offsets_kernel<<<1, 32, 0, stream>>>(cu, G, L, N);
 }
+
+// Packed batch: sequence b = rows [cu[b], cu[b + 1]) becomes G segments of Lc = max(8, ceil(chunks / G)) chunks
+// each (the last one shorter, those beyond the sequence's end empty); segment b * G + r starts at cu_seg[b * G + r]
+// and ends where the next one starts.  Malformed offsets give segments of negative length, which every kernel
+// that reads them reports and skips.
+__global__ void seg_offsets_packed_kernel(const int *__restrict__ cu, int B, int G, int *__restrict__ cu_seg)
+{
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x > B * G) return;
+    if (x == B * G) {
+        cu_seg[x] = cu[B];
+        return;
+    }
+    const int b = x / G, r = x - b * G;
+    const int start = cu[b], n = cu[b + 1] - start;
+    const int nc = (n + kC - 1) / kC;
+    int Lc = (nc + G - 1) / G;
+    if (Lc < 8) Lc = 8;
+    cu_seg[x] = start + (n <= 0 ? (r == 0 ? 0 : n) : min(r * Lc * kC, n));
+}
+
+void launch_seg_offsets_packed(const int *cu, int B, int G, int *cu_seg, cudaStream_t stream)
+{
+    const int n = B * G + 1;
+    seg_offsets_packed_kernel<<<(n + 127) / 128, 128, 0, stream>>>(cu, B, G, cu_seg);
+}
+
+// Segments per sequence of a packed batch: as many as fill the SMs when the units alone fill at most half of them.
+int tc_packed_segments(uint64_t U)
+{
+    const int sms = sm_count();
+    if (U == 0 || sms == 0 || 2 * U > (uint64_t)sms) return 1;
+    const int G = sms / (int)U;
+    return G > 8 ? 8 : G;
+}
+
+size_t tc_packed_offsets_bytes(int B, int G) { return (((size_t)B * G + 1) * sizeof(int) + 255) & ~(size_t)255; }
 
 // Few units (no more than SMs): all of them are split.  More units than SMs: the units beyond the last full
 // wave of CTAs would keep a few SMs busy for a whole sequence while the rest idle, so those - when they are at
@@ -735,11 +773,12 @@ size_t tc_segment_scratch_bytes(const hgrn2_desc *d, int C)
 }
 
 // One float matrix per unit for the exact path of the backward (chunk_alu.cuh, bwd_unit).
-size_t tc_exact_scratch_bytes(const hgrn2_desc *d)
+size_t tc_exact_scratch_bytes(const hgrn2_desc *d, bool packed)
 {
     const uint64_t U = (uint64_t)d->B * d->H;
-    const RSegPlan rp = tc_rseg_plan(U, d->N, (d->N + kC - 1) / kC);      // ragged segments: one matrix per segment
-    return (size_t)U * (rp.G > 1 ? rp.G : 1) * kD * kD * sizeof(float);
+    // sequences run as segments of their own geometry: one matrix per segment
+    const int G = packed ? tc_packed_segments(U) : tc_rseg_plan(U, d->N, (d->N + kC - 1) / kC).G;
+    return (size_t)U * (G > 1 ? G : 1) * kD * kD * sizeof(float);
 }
 
 static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag, int *unit_count)
@@ -792,18 +831,28 @@ static cudaError_t launch_fwd_once(const SeqArgs &a, uint64_t U, int N, int NC, 
     return cudaGetLastError();
 }
 
-PackedArgs tc_packed_args(const SeqArgs &a)
+// G segments per sequence: B * G pseudo-sequences share the slot numbering
+PackedArgs tc_packed_args(const SeqArgs &a, int G)
 {
     PackedArgs pk;
     pk.cu = a.cu;
     pk.H = a.H;
-    pk.slots_per_head = a.N / kC + a.B + 1;
+    pk.slots_per_head = a.N / kC + a.B * G + 1;
     return pk;
 }
 
 size_t tc_saved_bytes_packed(const hgrn2_desc *d)
 {
-    return (size_t)d->H * ((size_t)d->N / kC + d->B + 1) * (kSavedStateBytes + kSavedTotalsBytes);
+    const int G = tc_packed_segments((uint64_t)d->B * d->H);
+    return (size_t)d->H * ((size_t)d->N / kC + (size_t)d->B * G + 1) * (kSavedStateBytes + kSavedTotalsBytes);
+}
+
+// offsets of the segments | S_local, S_start (or G_local, dS_end) [B * G * H][128][128] | Lambda [B * G * H][128]
+size_t tc_segment_scratch_bytes_packed(const hgrn2_desc *d)
+{
+    const int G = tc_packed_segments((uint64_t)d->B * d->H);
+    if (G <= 1) return 0;
+    return tc_packed_offsets_bytes(d->B, G) + (size_t)d->B * G * d->H * (2 * kD * kD + kD) * sizeof(float);
 }
 
 cudaError_t launch_tc_fwd(const SeqArgs &a0)
@@ -812,12 +861,37 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
     SeqArgs a = a0;
     if (a.cu) {
         // packed batch: one CTA per (sequence, head), every CTA reads its own rows from the offsets array
-        const PackedArgs pk = tc_packed_args(a);
+        const int G = a.seg_scratch ? tc_packed_segments(U) : 1;
+        PackedArgs pk = tc_packed_args(a, G);
         if (a.states)
             a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
                                                  (size_t)pk.H * pk.slots_per_head * kSavedStateBytes);
-        return launch_fwd_once(a, U, a.N, 0, a.S0, a.SN, a.y != nullptr, a.states != nullptr, a.clear_status,
-                               exact_args(a, a.N, 1, nullptr, nullptr), pk);
+        if (G <= 1)
+            return launch_fwd_once(a, U, a.N, 0, a.S0, a.SN, a.y != nullptr, a.states != nullptr, a.clear_status,
+                                   exact_args(a, a.N, 1, nullptr, nullptr), pk);
+        // few units: every sequence as G segments (state-only pass, chaining, full pass: see below), the segments'
+        // offsets derived from the batch's on the device
+        const uint64_t CT = U * G;
+        char *base = static_cast<char *>(a.seg_scratch);
+        int *cu_seg = reinterpret_cast<int *>(base);
+        float *S_loc = reinterpret_cast<float *>(base + tc_packed_offsets_bytes(a.B, G));
+        float *S_start = S_loc + CT * kD * kD;
+        float *lam = S_start + CT * kD * kD;
+        launch_seg_offsets_packed(a.cu, a.B, G, cu_seg, a.stream);
+        cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        pk.cu = cu_seg;
+        err = launch_tc_state_fwd(a.f, a.i, (uint64_t)a.H, a.N, S_loc, lam, a.gate_enc, a.status, a.clear_status,
+                                  a.start_aborted, a.stream, cu_seg, a.B * G);
+        if (err != cudaSuccess) return err;
+        seg_combine_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.S0, S_loc, lam, S_start, a.SN, G,
+                                                                               nullptr, nullptr, 0, 2, (size_t)U, a.H);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        SeqArgs t = a;
+        t.S0 = S_start;
+        t.SN = nullptr;
+        return launch_fwd_once(t, CT, a.N, 0, S_start, nullptr, a.y != nullptr, a.states != nullptr, false,
+                               exact_args(t, a.N, 1, nullptr, nullptr), pk);
     }
     const bool want_y = a.y != nullptr, want_saved = a.states != nullptr;
     const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{1, 0};
@@ -846,7 +920,7 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
                                   a.stream, cu, G);
         if (err != cudaSuccess) return err;
         seg_combine_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.S0, S_loc, lam, S_start, a.SN, G,
-                                                                               nullptr, nullptr, 0, 1, (size_t)U);
+                                                                               nullptr, nullptr, 0, 1, (size_t)U, 1);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         SeqArgs t = a;
         t.S0 = S_start;
@@ -878,7 +952,7 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
         err = launch_tc_state_fwd(t.f, t.i, Ut * G, a.N / G, S_loc, lam, a.gate_enc, a.status, clear, a.start_aborted, a.stream);
         if (err != cudaSuccess) return err;
         seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G,
-                                                                                unit_flag, unit_count, (int)Ut, 0, (size_t)Ut);
+                                                                                unit_flag, unit_count, (int)Ut, 0, (size_t)Ut, 1);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         err = launch_fwd_once(t, Ut * G, a.N / G, a.NC / G, S_start, nullptr, want_y, want_saved, false,
                               exact_args(t, a.N, G, unit_flag, unit_count));

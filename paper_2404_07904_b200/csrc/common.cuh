@@ -147,6 +147,12 @@ struct RSegPlan {
 RSegPlan    tc_rseg_plan(uint64_t U, int N, int NC);
 constexpr size_t kRSegOffsetsBytes = 256;      // the offsets array of the ragged segments, in front of their scratch
 void        launch_seg_offsets(int *cu, int G, int L, int N, cudaStream_t stream);
+// Packed batch on few units: every sequence is cut into the same number G of segments (short sequences leave
+// some of theirs empty); the lengths are known on the device only, so the offsets of the B * G segments are
+// written there.  G = 1: not split.
+int         tc_packed_segments(uint64_t U);
+size_t      tc_packed_offsets_bytes(int B, int G);
+void        launch_seg_offsets_packed(const int *cu, int B, int G, int *cu_seg, cudaStream_t stream);
 SeqArgs     tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n);
 
 cudaError_t launch_tc_state_fwd(const void *f, const void *i, uint64_t U, int N, float *S_loc, float *lam, bool gate_enc,

@@ -218,6 +218,16 @@ __device__ __forceinline__ void tril_row_block(uint32_t taddr, uint8_t *dstbuf, 
     }
 }
 
+// Where segment r of unit u sits among the segment summaries (chunk_tc_fwd.cu, sequences split into segments):
+// order 0: u * G + r; order 1: r * U + u (ragged segments of an ordinary batch); order 2: unit u = (sequence b,
+// head h) of a packed batch with H heads, its segment r at (b * G + r) * H + h.
+__device__ __forceinline__ size_t seg_index(int order, size_t u, int r, int G, size_t U, int H)
+{
+    if (order == 1) return (size_t)r * U + u;
+    if (order == 2) return ((u / H) * G + r) * H + u % H;
+    return u * G + r;
+}
+
 // ---- host side: tensor maps ---------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,

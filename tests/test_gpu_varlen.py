@@ -89,7 +89,9 @@ def test_packed_bf16_empty_sequences_and_unused_tail_rows():
 
 
 def test_packed_equals_separate_calls_bitwise():
-    # the packed call must give exactly what one ordinary call per sequence gives (same kernels, same order)
+    # the packed call must give exactly what one ordinary call per sequence gives (same kernels, same order); the
+    # boundary states come out of the segment chaining (few units: every sequence runs as segments, these short ones
+    # as a single one each), i.e. from the state-only kernel, and agree within the bf16 tolerance
     lengths = [200, 64, 129]
     inp = _packed_inputs(lengths, H=2, d=128, io="bf16", seed=23)
     got, _ = _run_gpu(inp, "bf16")
@@ -99,8 +101,8 @@ def test_packed_equals_separate_calls_bitwise():
         one = G.gpu_fwd_bwd(sub, "bf16")
         for k in ("y", "d_o", "d_f", "d_i"):
             np.testing.assert_array_equal(got[k][:, s:e], one[k][0])
-        np.testing.assert_array_equal(got["SN"][b], one["SN"][0])
-        np.testing.assert_array_equal(got["dS0"][b], one["dS0"][0])
+        assert G.rel_err(got["SN"][b], one["SN"][0]) <= 2e-2
+        assert G.rel_err(got["dS0"][b], one["dS0"][0]) <= 2e-2
 
 
 def test_packed_hard_forget_sequence_takes_the_exact_path():
@@ -111,6 +113,31 @@ def test_packed_hard_forget_sequence_takes_the_exact_path():
     got, ws = _run_gpu(inp, "bf16")
     assert binding.exact_path_units(ws) == 1
     G.assert_close(got, _oracle(inp), 2e-2, "packed, one hard-forget unit")
+
+
+def test_packed_long_sequences_run_as_segments():
+    # few units: every sequence is cut into segments on the device (its length is known only there); a hard-forget
+    # stretch in a late segment of one sequence puts that segment alone on the exact path
+    lengths = [3000, 0, 5000, 700]
+    inp = _packed_inputs(lengths, H=2, d=128, io="bf16", seed=27)
+    d = binding.make_desc(len(lengths), 2, int(sum(lengths)), 128, 128, binding.HGRN2_BF16)
+    assert lib_ws_has_segments(d)
+    s = int(inp["cu"][2])
+    inp["f"][1, s + 4000:s + 4070, 11] = W.round_to_bf16(np.float32(0.02))
+    got, ws = _run_gpu(inp, "bf16")
+    assert binding.exact_path_units(ws) == 1
+    G.assert_close(got, _oracle(inp), 2e-2, "packed long sequences")
+    got2, _ = _run_gpu(inp, "bf16", use_saved=False)
+    for k in got:
+        np.testing.assert_array_equal(got[k], got2[k])
+
+
+def lib_ws_has_segments(d):
+    lib = binding.load()
+    import ctypes
+    ws = lib.hgrn2_workspace_bytes_varlen(ctypes.byref(d))
+    saved = lib.hgrn2_saved_bytes_varlen(ctypes.byref(d))
+    return ws > 256 + saved + 8 * d.B * d.H * 128 * 128 * 4          # room for eight segments per unit
 
 
 @pytest.mark.parametrize("io,d,flags", [("f32", 64, 0), ("bf16", 128, binding.FLAG_FORCE_ALU)])
