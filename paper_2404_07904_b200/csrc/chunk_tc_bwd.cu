@@ -910,33 +910,41 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
         t.dS0 = nullptr;
         return launch_bwd_once(t, CT, a.N, 0, dS_end, nullptr, false, exact_args(t, a.N, 1, nullptr, nullptr), pk);
     }
-    const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{1, 0};
-    if (rp.G > 1) {
+    const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{U, 0, 1, 0};
+    if (rp.tail_units) {
         // ragged segments (see launch_tc_fwd): state-gradient summaries per segment, chained in reverse, then the
         // full pass per segment through the packed-batch geometry
         const int G = rp.G;
-        const uint64_t CT = U * G;
+        const uint64_t Ut = rp.tail_units, CT = Ut * G;
+        const size_t spp = (size_t)(a.N / kC + G + 1);
+        a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
+                                             ((size_t)rp.main_units * a.NC + (size_t)Ut * spp) * kSavedStateBytes);
+        cudaError_t err = cudaSuccess;
+        bool clear = a.clear_status;
+        if (rp.main_units) {
+            const SeqArgs m = tc_slice_units(a, 0, rp.main_units);
+            err = launch_bwd_once(m, rp.main_units, a.N, a.NC, m.dSN, m.dS0, clear, exact_args(m, a.N, 1, nullptr, nullptr));
+            if (err != cudaSuccess) return err;
+            clear = false;
+        }
+        SeqArgs t = tc_slice_units(a, rp.main_units, Ut);
         char *base = static_cast<char *>(a.seg_scratch);
         int *cu = reinterpret_cast<int *>(base);
         float *G_loc = reinterpret_cast<float *>(base + kRSegOffsetsBytes);
         float *dS_end = G_loc + CT * kD * kD;
         float *lam = dS_end + CT * kD * kD;
         launch_seg_offsets(cu, G, rp.Lc * kC, a.N, a.stream);
-        cudaError_t err = cudaGetLastError();
-        if (err != cudaSuccess) return err;
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
         PackedArgs pk;
         pk.cu = cu;
-        pk.H = (int)U;
-        pk.slots_per_head = a.N / kC + G + 1;
-        a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
-                                             (size_t)U * pk.slots_per_head * kSavedStateBytes);
-        err = launch_tc_state_bwd(a.o, a.f, a.dy, U, a.N, G_loc, lam, a.gate_enc, a.status, a.clear_status,
-                                  a.start_aborted, a.stream, cu, G);
+        pk.H = (int)Ut;
+        pk.slots_per_head = (int)spp;
+        err = launch_tc_state_bwd(t.o, t.f, t.dy, Ut, a.N, G_loc, lam, a.gate_enc, a.status, clear, a.start_aborted,
+                                  a.stream, cu, G);
         if (err != cudaSuccess) return err;
-        seg_combine_bwd_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.dSN, G_loc, lam, dS_end, a.dS0, G,
-                                                                                   nullptr, nullptr, 0, 1, (size_t)U, 1);
+        seg_combine_bwd_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.dSN, G_loc, lam, dS_end, t.dS0, G,
+                                                                                    nullptr, nullptr, 0, 1, (size_t)Ut, 1);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        SeqArgs t = a;
         t.dSN = dS_end;
         t.dS0 = nullptr;
         return launch_bwd_once(t, CT, a.N, 0, dS_end, nullptr, false, exact_args(t, a.N, 1, nullptr, nullptr), pk);

@@ -592,8 +592,9 @@ size_t tc_saved_bytes(const hgrn2_desc *d, int C)
     const uint64_t U = (uint64_t)d->B * d->H;
     const RSegPlan rp = tc_rseg_plan(U, d->N, (int)NC);
     // ragged segments use the packed batch's slot numbering: N / C + (segments) + 1 slots per unit
-    const size_t slots = rp.G > 1 ? (size_t)d->N / C + rp.G + 1 : NC;
-    return (size_t)U * slots * (kSavedStateBytes + kSavedTotalsBytes);
+    const size_t slots = rp.tail_units ? (size_t)rp.main_units * NC + (size_t)rp.tail_units * ((size_t)d->N / C + rp.G + 1)
+                                       : (size_t)U * NC;
+    return slots * (kSavedStateBytes + kSavedTotalsBytes);
 }
 
 // ---- sequences split into segments ----------------------------------------------------------------------
@@ -647,20 +648,27 @@ int segments_for(uint64_t U, int N, int NC)
     return G >= 2 ? G : 1;
 }
 
-// Sequences that are not whole chunks, few units: segments of Lc chunks (at least 8), the last one shorter.
+// Sequences that are not whole chunks: segments of Lc chunks (at least 8), the last one shorter, for all units
+// when they are few and for the units beyond the last full wave otherwise (the rule of tc_seg_plan).
 RSegPlan tc_rseg_plan(uint64_t U, int N, int NC)
 {
-    RSegPlan p{1, 0};
-    const int sms = sm_count();
-    if (U == 0 || sms == 0 || N % kC == 0 || U > (uint64_t)sms) return p;
-    int G0 = sms / (int)U;
+    RSegPlan p{U, 0, 1, 0};
+    const uint64_t sms = (uint64_t)sm_count();
+    if (U == 0 || sms == 0 || N % kC == 0) return p;
+    uint64_t split = U, whole = 0;
+    if (U > sms) {
+        split = U % sms;
+        whole = U - split;
+        if (split == 0 || 2 * split > sms) return p;
+    }
+    int G0 = (int)(sms / split);
     if (G0 > 8) G0 = 8;
     if (G0 < 2) return p;
     int Lc = (NC + G0 - 1) / G0;
     if (Lc < 8) Lc = 8;
     const int G = (NC + Lc - 1) / Lc;
     if (G < 2) return p;
-    return RSegPlan{G, Lc};
+    return RSegPlan{whole, split, G, Lc};
 }
 
 // cu[r] = first row of segment r (r = 0 .. G), segments of L rows, the last one ends at N
@@ -767,7 +775,7 @@ size_t tc_segment_scratch_bytes(const hgrn2_desc *d, int C)
     const uint64_t U = (uint64_t)d->B * d->H;
     const int NC = (d->N + C - 1) / C;
     const RSegPlan rp = tc_rseg_plan(U, d->N, NC);
-    if (rp.G > 1) return kRSegOffsetsBytes + (size_t)U * rp.G * (2 * kD * kD + kD) * sizeof(float);
+    if (rp.tail_units) return kRSegOffsetsBytes + (size_t)rp.tail_units * rp.G * (2 * kD * kD + kD) * sizeof(float);
     const SegPlan p = tc_seg_plan(U, d->N, NC);
     return p.tail_units ? (size_t)p.tail_units * p.G * (2 * kD * kD + kD) * sizeof(float) + seg_flag_bytes(p.tail_units) : 0;
 }
@@ -777,8 +785,9 @@ size_t tc_exact_scratch_bytes(const hgrn2_desc *d, bool packed)
 {
     const uint64_t U = (uint64_t)d->B * d->H;
     // sequences run as segments of their own geometry: one matrix per segment
-    const int G = packed ? tc_packed_segments(U) : tc_rseg_plan(U, d->N, (d->N + kC - 1) / kC).G;
-    return (size_t)U * (G > 1 ? G : 1) * kD * kD * sizeof(float);
+    if (packed) return (size_t)U * tc_packed_segments(U) * kD * kD * sizeof(float);
+    const RSegPlan rp = tc_rseg_plan(U, d->N, (d->N + kC - 1) / kC);
+    return ((size_t)rp.main_units + (size_t)rp.tail_units * rp.G) * kD * kD * sizeof(float);
 }
 
 static ExactArgs exact_args(const SeqArgs &a, int N_unit, int G, int *unit_flag, int *unit_count)
@@ -894,35 +903,45 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
                                exact_args(t, a.N, 1, nullptr, nullptr), pk);
     }
     const bool want_y = a.y != nullptr, want_saved = a.states != nullptr;
-    const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{1, 0};
-    if (rp.G > 1) {
+    const RSegPlan rp = a.seg_scratch ? tc_rseg_plan(U, a.N, a.NC) : RSegPlan{U, 0, 1, 0};
+    if (rp.tail_units) {
         // ragged segments: the three steps of the whole-chunk segments below, with per-CTA rows from an offsets
         // array (the packed-batch geometry: "sequence" r of "head" u = segment r of unit u); every segment CTA
-        // takes its own exact path from its start state, which the state-only pass gives for every f
+        // takes its own exact path from its start state, which the state-only pass gives for every f.  Saved
+        // states: the whole units' slots first, then the split units' in the packed slot numbering.
         const int G = rp.G;
-        const uint64_t CT = U * G;
+        const uint64_t Ut = rp.tail_units, CT = Ut * G;
+        const size_t spp = (size_t)(a.N / kC + G + 1);
+        if (a.states)
+            a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
+                                                 ((size_t)rp.main_units * a.NC + (size_t)Ut * spp) * kSavedStateBytes);
+        cudaError_t err = cudaSuccess;
+        bool clear = a.clear_status;
+        if (rp.main_units) {
+            const SeqArgs m = tc_slice_units(a, 0, rp.main_units);
+            err = launch_fwd_once(m, rp.main_units, a.N, a.NC, m.S0, m.SN, want_y, want_saved, clear,
+                                  exact_args(m, a.N, 1, nullptr, nullptr));
+            if (err != cudaSuccess) return err;
+            clear = false;
+        }
+        SeqArgs t = tc_slice_units(a, rp.main_units, Ut);
         char *base = static_cast<char *>(a.seg_scratch);
         int *cu = reinterpret_cast<int *>(base);
         float *S_loc = reinterpret_cast<float *>(base + kRSegOffsetsBytes);
         float *S_start = S_loc + CT * kD * kD;
         float *lam = S_start + CT * kD * kD;
         launch_seg_offsets(cu, G, rp.Lc * kC, a.N, a.stream);
-        cudaError_t err = cudaGetLastError();
-        if (err != cudaSuccess) return err;
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
         PackedArgs pk;
         pk.cu = cu;
-        pk.H = (int)U;
-        pk.slots_per_head = a.N / kC + G + 1;
-        if (a.states)
-            a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
-                                                 (size_t)U * pk.slots_per_head * kSavedStateBytes);
-        err = launch_tc_state_fwd(a.f, a.i, U, a.N, S_loc, lam, a.gate_enc, a.status, a.clear_status, a.start_aborted,
+        pk.H = (int)Ut;
+        pk.slots_per_head = (int)spp;
+        err = launch_tc_state_fwd(t.f, t.i, Ut, a.N, S_loc, lam, a.gate_enc, a.status, clear, a.start_aborted,
                                   a.stream, cu, G);
         if (err != cudaSuccess) return err;
-        seg_combine_kernel<<<(unsigned)(U * kD * kD / 256), 256, 0, a.stream>>>(a.S0, S_loc, lam, S_start, a.SN, G,
-                                                                               nullptr, nullptr, 0, 1, (size_t)U, 1);
+        seg_combine_kernel<<<(unsigned)(Ut * kD * kD / 256), 256, 0, a.stream>>>(t.S0, S_loc, lam, S_start, t.SN, G,
+                                                                                nullptr, nullptr, 0, 1, (size_t)Ut, 1);
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        SeqArgs t = a;
         t.S0 = S_start;
         t.SN = nullptr;
         return launch_fwd_once(t, CT, a.N, 0, S_start, nullptr, want_y, want_saved, false,

@@ -138,9 +138,12 @@ struct SegPlan {
     int G;
 };
 SegPlan     tc_seg_plan(uint64_t U, int N, int NC);
-// Few units whose sequences are NOT whole chunks: every sequence is cut into G segments of Lc chunks (the last one
-// shorter), which run through the packed-batch geometry (per-CTA rows from an offsets array).  G = 1: not split.
+// Sequences that are NOT whole chunks, few or left-over units (as SegPlan): those units' sequences are cut into G
+// segments of Lc chunks (the last one shorter), which run through the packed-batch geometry (per-CTA rows from an
+// offsets array).
 struct RSegPlan {
+    uint64_t main_units;   // units [0, main_units) run as one CTA each
+    uint64_t tail_units;   // units [main_units, main_units + tail_units) run as G segments each (0: nothing is split)
     int G;
     int Lc;
 };

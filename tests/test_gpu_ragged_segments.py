@@ -67,3 +67,20 @@ def test_gated_entry_points_on_ragged_segments():
     inp = TG._inputs(1, 2, 1000, 128, "bf16", seed=97, beta_lo=0.0, beta_hi=0.9, zf_shift=1.0, states=True)
     got, _ = TG._run(inp, "bf16", use_saved=True)
     G.assert_close(got, TG._oracle(inp), TOL, "gated, 1000 tokens in two segments")
+
+
+@pytest.mark.parametrize("use_saved", [True, False])
+def test_units_beyond_the_last_full_wave_with_ragged_sequences(use_saved):
+    # more units than SMs and sequences that are not whole chunks: the full wave runs whole, the left-over units as
+    # ragged segments; units on both sides of the split are compared
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    H = sms + 12
+    w = W.scaled(W.CONFIGS["long_16k"], B=1, H=H, N=1000, has_S0=True, has_dSN=True, seed=98)
+    d = binding.make_desc(1, H, 1000, 128, 128, binding.HGRN2_BF16)
+    assert binding.workspace_bytes(d) > 256 + binding.saved_bytes(d) + H * 128 * 128 * 4, "segments expected"
+    inp = W.make_inputs(w)
+    inp["f"][0, H - 3, 600:660, 5] = W.round_to_bf16(np.float32(0.02))      # second segment of a left-over unit
+    got = G.gpu_fwd_bwd(inp, "bf16", use_saved=use_saved)
+    units = [(0, 0), (0, sms - 1), (0, sms), (0, H - 3), (0, H - 1)]
+    for (b, h), want in G.oracle_fwd_bwd(inp, units).items():
+        G.assert_close({k: got[k][b:b + 1, h:h + 1] for k in want}, want, TOL, f"unit {(b, h)}")
