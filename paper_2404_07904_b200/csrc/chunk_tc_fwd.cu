@@ -638,7 +638,7 @@ int sm_count()
 }
 
 // Number of segments per sequence (1 = do not split): as many as fill the SMs, at most 8, dividing the chunk
-// count, each at least 8 chunks long; only for sequences made of whole chunks.
+// count, each at least 8 chunks long; for sequences made of whole chunks (others: tc_rseg_plan).
 int segments_for(uint64_t U, int N, int NC)
 {
     if (U == 0 || N % kC != 0) return 1;
