@@ -43,9 +43,9 @@ NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu captures summarised under
 # profiles/ (same workloads as timed here: lm_2048 and the full decode batch); nothing here measures traffic.
 # None = the kernel has changed since its counters were taken.
-NCU_TRAFFIC_BYTES = {"fwd": 201.41e6 + 154.72e6, "bwd": 406.96e6 + 172.24e6, "step": 271.60e6 + 212.48e6}
-NCU_TRAFFIC_SOURCE = {"fwd": "profiles/tc_fwd_bwd_lm2048.md (captured 2026-11-30, kernels as of the regrouped backward products)",
-                      "bwd": "profiles/tc_fwd_bwd_lm2048.md (captured 2026-11-30, kernels as of the regrouped backward products)",
+NCU_TRAFFIC_BYTES = {"fwd": 201.41e6 + 154.02e6, "bwd": 406.96e6 + 170.88e6, "step": 271.60e6 + 212.48e6}
+NCU_TRAFFIC_SOURCE = {"fwd": "profiles/tc_fwd_bwd_lm2048.md (captured 2026-11-30, kernels as of the two-read completion pass of the backward)",
+                      "bwd": "profiles/tc_fwd_bwd_lm2048.md (captured 2026-11-30, kernels as of the two-read completion pass of the backward)",
                       "step": "profiles/step_kernel_decode.md"}
 
 
