@@ -143,7 +143,7 @@ hgrn2_status hgrn2_bwd(const hgrn2_desc *desc, const void *o, const void *f, con
  *   ws     hgrn2_workspace_bytes_varlen(desc) bytes.
  * Everything else - ownership, streams, errors, the closed interval for f - is as for hgrn2_fwd / hgrn2_bwd.
  * One CTA serves one (sequence, head) unit, dispatched in index order: with more units than SMs, put long
- * sequences first.  With few units (no more than half the SMs) every sequence runs as up to eight segments,
+ * sequences first.  With few units (no more than half the SMs; T > 512) every sequence runs as up to eight segments,
  * cut on the device; the two size queries then depend on the current device, and the boundary states SN and
  * dS0 come from the chaining of the segments' summaries (same tolerance, other rounding than hgrn2_fwd). */
 size_t hgrn2_saved_bytes_varlen(const hgrn2_desc *desc);

@@ -881,7 +881,7 @@ cudaError_t launch_tc_bwd(const SeqArgs &a0)
     SeqArgs a = a0;
     if (a.cu) {
         // packed batch: one CTA per (sequence, head), every CTA reads its own rows from the offsets array
-        const int G = a.seg_scratch ? tc_packed_segments(U) : 1;
+        const int G = a.seg_scratch ? tc_packed_segments(U, a.N) : 1;
         PackedArgs pk = tc_packed_args(a, G);
         a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +
                                              (size_t)pk.H * pk.slots_per_head * kSavedStateBytes);

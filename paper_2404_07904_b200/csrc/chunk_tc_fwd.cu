@@ -709,11 +709,12 @@ void launch_seg_offsets_packed(const int *cu, int B, int G, int *cu_seg, cudaStr
     seg_offsets_packed_kernel<<<(n + 127) / 128, 128, 0, stream>>>(cu, B, G, cu_seg);
 }
 
-// Segments per sequence of a packed batch: as many as fill the SMs when the units alone fill at most half of them.
-int tc_packed_segments(uint64_t U)
+// Segments per sequence of a packed batch of T rows per head: as many as fill the SMs when the units alone fill at
+// most half of them; none when no sequence can be longer than one segment (8 chunks).
+int tc_packed_segments(uint64_t U, int T)
 {
     const int sms = sm_count();
-    if (U == 0 || sms == 0 || 2 * U > (uint64_t)sms) return 1;
+    if (U == 0 || sms == 0 || 2 * U > (uint64_t)sms || T <= 8 * kC) return 1;
     const int G = sms / (int)U;
     return G > 8 ? 8 : G;
 }
@@ -785,7 +786,7 @@ size_t tc_exact_scratch_bytes(const hgrn2_desc *d, bool packed)
 {
     const uint64_t U = (uint64_t)d->B * d->H;
     // sequences run as segments of their own geometry: one matrix per segment
-    if (packed) return (size_t)U * tc_packed_segments(U) * kD * kD * sizeof(float);
+    if (packed) return (size_t)U * tc_packed_segments(U, d->N) * kD * kD * sizeof(float);
     const RSegPlan rp = tc_rseg_plan(U, d->N, (d->N + kC - 1) / kC);
     return ((size_t)rp.main_units + (size_t)rp.tail_units * rp.G) * kD * kD * sizeof(float);
 }
@@ -852,14 +853,14 @@ PackedArgs tc_packed_args(const SeqArgs &a, int G)
 
 size_t tc_saved_bytes_packed(const hgrn2_desc *d)
 {
-    const int G = tc_packed_segments((uint64_t)d->B * d->H);
+    const int G = tc_packed_segments((uint64_t)d->B * d->H, d->N);
     return (size_t)d->H * ((size_t)d->N / kC + (size_t)d->B * G + 1) * (kSavedStateBytes + kSavedTotalsBytes);
 }
 
 // offsets of the segments | S_local, S_start (or G_local, dS_end) [B * G * H][128][128] | Lambda [B * G * H][128]
 size_t tc_segment_scratch_bytes_packed(const hgrn2_desc *d)
 {
-    const int G = tc_packed_segments((uint64_t)d->B * d->H);
+    const int G = tc_packed_segments((uint64_t)d->B * d->H, d->N);
     if (G <= 1) return 0;
     return tc_packed_offsets_bytes(d->B, G) + (size_t)d->B * G * d->H * (2 * kD * kD + kD) * sizeof(float);
 }
@@ -870,7 +871,7 @@ cudaError_t launch_tc_fwd(const SeqArgs &a0)
     SeqArgs a = a0;
     if (a.cu) {
         // packed batch: one CTA per (sequence, head), every CTA reads its own rows from the offsets array
-        const int G = a.seg_scratch ? tc_packed_segments(U) : 1;
+        const int G = a.seg_scratch ? tc_packed_segments(U, a.N) : 1;
         PackedArgs pk = tc_packed_args(a, G);
         if (a.states)
             a.totals = reinterpret_cast<float *>(reinterpret_cast<char *>(a.states) +

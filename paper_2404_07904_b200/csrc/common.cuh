@@ -153,7 +153,7 @@ void        launch_seg_offsets(int *cu, int G, int L, int N, cudaStream_t stream
 // Packed batch on few units: every sequence is cut into the same number G of segments (short sequences leave
 // some of theirs empty); the lengths are known on the device only, so the offsets of the B * G segments are
 // written there.  G = 1: not split.
-int         tc_packed_segments(uint64_t U);
+int         tc_packed_segments(uint64_t U, int T);
 size_t      tc_packed_offsets_bytes(int B, int G);
 void        launch_seg_offsets_packed(const int *cu, int B, int G, int *cu_seg, cudaStream_t stream);
 SeqArgs     tc_slice_units(const SeqArgs &a, uint64_t u0, uint64_t n);

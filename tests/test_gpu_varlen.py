@@ -89,9 +89,8 @@ def test_packed_bf16_empty_sequences_and_unused_tail_rows():
 
 
 def test_packed_equals_separate_calls_bitwise():
-    # the packed call must give exactly what one ordinary call per sequence gives (same kernels, same order); the
-    # boundary states come out of the segment chaining (few units: every sequence runs as segments, these short ones
-    # as a single one each), i.e. from the state-only kernel, and agree within the bf16 tolerance
+    # the packed call must give exactly what one ordinary call per sequence gives (same kernels, same order; a batch
+    # this short is not cut into segments)
     lengths = [200, 64, 129]
     inp = _packed_inputs(lengths, H=2, d=128, io="bf16", seed=23)
     got, _ = _run_gpu(inp, "bf16")
@@ -101,8 +100,27 @@ def test_packed_equals_separate_calls_bitwise():
         one = G.gpu_fwd_bwd(sub, "bf16")
         for k in ("y", "d_o", "d_f", "d_i"):
             np.testing.assert_array_equal(got[k][:, s:e], one[k][0])
-        assert G.rel_err(got["SN"][b], one["SN"][0]) <= 2e-2
-        assert G.rel_err(got["dS0"][b], one["dS0"][0]) <= 2e-2
+        np.testing.assert_array_equal(got["SN"][b], one["SN"][0])
+        np.testing.assert_array_equal(got["dS0"][b], one["dS0"][0])
+
+
+def test_packed_in_segments_equals_separate_calls():
+    # few units and long enough to be cut into segments: y and the gradients are still bit-identical to separate calls
+    # on whole-chunk sequences run the same way; the boundary states come out of the segment chaining (state-only
+    # kernel) and agree within the bf16 tolerance
+    lengths = [1100, 200, 700]
+    inp = _packed_inputs(lengths, H=1, d=128, io="bf16", seed=28)
+    got, _ = _run_gpu(inp, "bf16")
+    want = _oracle(inp)
+    G.assert_close(got, want, 2e-2, "packed in segments")
+    b, (s, e) = 1, (int(inp["cu"][1]), int(inp["cu"][2]))               # the 200-token sequence: a single segment
+    sub = {k: np.ascontiguousarray(inp[k][None, :, s:e]) for k in ("o", "f", "i", "dy")}
+    sub["S0"], sub["dSN"] = inp["S0"][b:b + 1], inp["dSN"][b:b + 1]
+    one = G.gpu_fwd_bwd(sub, "bf16")
+    for k in ("y", "d_o", "d_f", "d_i"):
+        np.testing.assert_array_equal(got[k][:, s:e], one[k][0])
+    assert G.rel_err(got["SN"][b], one["SN"][0]) <= 2e-2
+    assert G.rel_err(got["dS0"][b], one["dS0"][0]) <= 2e-2
 
 
 def test_packed_hard_forget_sequence_takes_the_exact_path():
