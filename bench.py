@@ -17,8 +17,10 @@ Timing.  The step loop is timed in batches of exactly K steps (CUDA events on th
 barrier and a device synchronise on both sides, max over ranks); batches are repeated until at least
 --min-seconds of device time have been spent, so that the SM clock is sampled under a sustained load, and
 the MEDIAN batch is reported (`value`, `ms_per_step`; the spread is in `timing`).  `roofline.kernels` and the
-dominant-kernel figures come from separate loops of one kernel alone (forward only, backward only); those
-find different data in L2 than the alternating step does, so their sum differs from the step by a few %.
+dominant-kernel figures come from separate loops of one kernel alone (forward only, backward only), K launches
+each, taken BEFORE the long step loop: a few milliseconds on a board that has not reached its power cap (boost
+clock), whereas the step loop settles at the capped clock it reports; they also find different data in L2 than
+the alternating step does.  So their sum is below the step's time, by the clock ratio and a few %.
 """
 from __future__ import annotations
 
@@ -573,6 +575,10 @@ def run_cuda(args):
     torch.cuda.synchronize()
     assert binding.hgrn2_poll(ws) == 0, "device-side error during warm-up"
 
+    # isolated kernel loops, before the long step loop (see the module docstring)
+    ms_fwd = max_over_ranks(timed(fwd, K))
+    ms_bwd = max_over_ranks(timed(bwd, K))
+
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
     if rank == 0:
         sampler.start()
@@ -588,9 +594,6 @@ def run_cuda(args):
         sampler.stop()
     clocks = sampler.summary()
     ms_total = statistics.median(batch_ms)
-    # isolated kernel loops (their own L2 state: see the module docstring)
-    ms_fwd = max_over_ranks(timed(fwd, K))
-    ms_bwd = max_over_ranks(timed(bwd, K))
     for _ in range(2):
         e2e_step()
     torch.cuda.synchronize()
